@@ -1,0 +1,162 @@
+// Internal declarations shared by the translation units of libcerb.so.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "cerb.h"
+
+#define CERB_CUDA_OK(expr)                         \
+  do {                                             \
+    cudaError_t e__ = (expr);                      \
+    if (e__ != cudaSuccess) return CERB_E_CUDA;    \
+  } while (0)
+
+#define CERB_TRY(expr)                 \
+  do {                                 \
+    int rc__ = (expr);                 \
+    if (rc__ != CERB_OK) return rc__;  \
+  } while (0)
+
+#define CERB_LAUNCH_CHECK(c)                                   \
+  do {                                                         \
+    if (c) (c)->launches++;                                    \
+    if (cudaGetLastError() != cudaSuccess) return CERB_E_CUDA; \
+  } while (0)
+
+namespace cerb {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int kPathMax = CERB_MAX_DEPTH + 1;
+constexpr int kGemmRowsPerPass = 256;   // activation rows one tcgen05 pass covers (the MMA's N extent)
+constexpr int kGemmMaxSplit = 16;
+
+// Device-side copy of a tree, living in the workspace.
+struct TreeDev {
+  int32_t* parent;   // [CERB_MAX_NODES]
+  int32_t* depth;
+  int32_t* head_of;
+  int32_t* rank_of;
+  uint64_t* anc;     // [CERB_MAX_NODES][2]
+};
+constexpr size_t kTreeSlotBytes = 4 * CERB_MAX_NODES * sizeof(int32_t) + CERB_MAX_NODES * 2 * sizeof(uint64_t);
+
+// Tensor maps for one activation buffer used as the MMA's B operand, one per row bucket.
+constexpr int kRowBuckets = 5;          // 16, 32, 64, 128, 256 rows
+struct ActMaps {
+  CUtensorMap m[kRowBuckets];
+};
+
+}  // namespace cerb
+
+struct cerb_tree {
+  int32_t n;
+  int32_t slot;
+  int32_t max_depth;
+  cerb::TreeDev dev;
+  std::vector<int32_t> parent, depth;
+};
+
+struct cerb_ctx {
+  cerb_config cfg;
+  bool bf16;
+  size_t esize;                       // bytes per model element
+  int Mmax;                           // max rows of one forward (max_batch * max_nodes)
+  int max_pos;                        // 16 * max_pages
+  int head_w[CERB_MAX_HEADS][CERB_MAX_LEVELS + 1];   // state width entering each level
+  int head_wmax;
+
+  // weights (device pointers, host arrays)
+  const void *embed, *final_norm, *lm_head;
+  std::vector<const void*> attn_norm, wqkv, wo, mlp_norm, wgu, wd, head_W, head_b, head_fc;
+  char *k_pool, *v_pool;
+  size_t pool_layer_bytes;
+  const int32_t* page_table;
+
+  // tensor maps (bf16 only)
+  std::vector<CUtensorMap> tm_wqkv, tm_wo, tm_wgu, tm_wd;
+  CUtensorMap tm_lm_head;
+  cerb::ActMaps tm_xn, tm_attn, tm_act, tm_hidden, tm_hlast;
+  std::vector<CUtensorMap> tm_kpool, tm_vpool;        // per layer
+
+  // workspace carve-out
+  int32_t *d_len, *d_len_old, *d_root, *d_nactive, *d_status, *d_lens_in, *d_mode, *d_naccept;
+  int32_t *d_path, *d_outtok, *d_argmax, *d_treetok, *d_topk;
+  float* d_S;
+  void *d_hlast, *d_x, *d_xn, *d_q, *d_attn, *d_act, *d_hidden;
+  float *d_part, *d_logits, *d_hlogits;
+  size_t part_floats;
+  float* d_hstate[2];
+  float2* d_rope;
+  char* d_attn_scratch;
+  size_t attn_scratch_bytes;
+  char* d_tree_store;
+  bool tree_used[CERB_MAX_TREES];
+  cerb_tree* chain;                   // chain tree of max_nodes for the prefill
+  cerb_tree* single;                  // one-node tree for auto-regressive steps
+
+  // pinned host staging
+  int32_t* h_stage;                   // [8 * CERB_MAX_BATCH]
+
+  // host-side state
+  int B;
+  int h_len[CERB_MAX_BATCH];          // upper bound of the committed length per sequence
+  const cerb_tree* verified_tree;     // tree of the last cerb_verify not yet accepted
+  int64_t launches;
+  int sm_count;
+};
+
+namespace cerb {
+
+inline int row_bucket(int rows) {
+  int b = 0, r = 16;
+  while (r < rows && b < kRowBuckets - 1) { r <<= 1; ++b; }
+  return b;
+}
+inline int bucket_rows(int b) { return 16 << b; }
+
+// ---- launch wrappers implemented across the .cu files (all asynchronous on `st`) ----
+
+// glue.cu
+int launch_rope_table(cerb_ctx* c, cudaStream_t st);
+int launch_embed(cerb_ctx* c, const int32_t* tok, int tok_stride, int tok_off, int B, int n, cudaStream_t st);
+int launch_rmsnorm(cerb_ctx* c, const void* x, const void* gain, void* out, int rows, cudaStream_t st);
+int launch_rope_append(cerb_ctx* c, int layer, const TreeDev& t, const float* part, int nsplit, size_t split_stride,
+                       int B, int n, cudaStream_t st);
+int launch_residual(cerb_ctx* c, void* x, const float* part, int nsplit, size_t split_stride, int rows, int N,
+                    cudaStream_t st);
+int launch_swiglu(cerb_ctx* c, const float* part, int nsplit, size_t split_stride, void* act, int rows, cudaStream_t st);
+int launch_argmax_rows(cerb_ctx* c, const float* logits, int rows, int V, int32_t* out, cudaStream_t st);
+int launch_set_nactive(cerb_ctx* c, int mode, int a, int b, cudaStream_t st);
+int launch_prefill_commit(cerb_ctx* c, int n, cudaStream_t st);
+
+// gemm_f32.cu / gemm_bf16.cu : out[split][M][N] fp32 partial sums of X[M][K] . W[N][K]^T
+int launch_gemm_f32(cerb_ctx* c, const float* X, const float* W, float* out, int M, int N, int K, cudaStream_t st);
+int gemm_plan_split(int sm_count, int M, int N, int K);
+int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, float* out, int M, int N, int K,
+                     int nsplit, int32_t* status, cudaStream_t st);
+int make_weight_map(CUtensorMap* out, const void* W, int N, int K);
+int make_act_maps(ActMaps* out, const void* X, int rows_alloc, int K);
+int init_driver_api();
+
+// attention.cu
+size_t attn_scratch_bytes(int B, int n, int H, int Dh);
+int make_pool_map(CUtensorMap* out, const void* pool, int n_pool_pages, int H, int Dh);
+int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMap* tmK, const CUtensorMap* tmV,
+                          int sm_count, int32_t* status, cudaStream_t st);
+
+// heads.cu
+int launch_heads(cerb_ctx* c, const cerb_tree* tree, int32_t* tree_tok, const int32_t* plant, int32_t* topk_out,
+                 float* logits_out, cudaStream_t st);
+
+// gate_accept.cu
+int launch_gate(cerb_ctx* c, float T, float* S, int32_t* mode, int32_t* nactive_or_null, int n_par, cudaStream_t st);
+int launch_accept(cerb_ctx* c, const cerb_tree* tree, const int32_t* tree_tok, const int32_t* n_active,
+                  const int32_t* node_argmax, int32_t* n_accept, int32_t* path, int32_t* out_tok, cudaStream_t st);
+
+}  // namespace cerb
