@@ -1,0 +1,528 @@
+// Tree-verification attention (Sections 1 and 3.1: all candidates are verified in one pass with
+// tree attention).  Query i of a sequence sees every committed prefix key and those tree keys j
+// that are its ancestors (bit j of anc[i]), nothing else.
+//
+// bf16 path: one CTA per (split, head, sequence).  A producer warp streams 64-key tiles (four
+// 16-token pages of one head, K and V) into shared memory with TMA, 128-byte swizzled, through an
+// mbarrier ring; compute warps run QK^T and PV on tensor cores (warp-level MMA, fp32 accumulate)
+// with an online softmax in registers.  Warps are arranged WQ x WK: WQ blocks of 16 query rows,
+// WK slices of each key tile, so small trees still use every warp.  Long contexts are split along
+// the keys; each split writes an unnormalised partial (m, l, O) and the last CTA to finish for a
+// (sequence, head) merges the partials in split order, so the result does not depend on timing.
+//
+// fp32 path (CERB_F32 models): plain FMA arithmetic, one CTA per (node, head, sequence).
+#include "cerb_internal.cuh"
+
+namespace cerb {
+
+namespace {
+
+constexpr int TILE = 64;                  // keys per pipeline stage = 4 pages
+constexpr int PAGES_PER_TILE = TILE / CERB_PAGE;
+constexpr int kTargetCtas = 296;          // two CTAs per SM on a 148-SM part
+constexpr int kMaxSplit = 32;
+constexpr int kMaxPagesPerCta = 1024;
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr size_t kCounterBytes = 4096;    // one ticket counter per (sequence, head)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* aborted, int32_t* status) {
+  uint32_t limit = *aborted ? 256u : kSpinLimit;
+  for (uint32_t i = 0; i < limit; ++i)
+    if (mbar_try_wait(bar, parity)) return;
+  *aborted = 1;
+  atomicExch(status, CERB_E_TIMEOUT);
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"((uint64_t)map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ void compute_bar(int nthreads) { asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory"); }
+
+struct AttnParams {
+  const bf16* q;
+  const int32_t* page_table;
+  const int32_t* len;
+  const int32_t* n_active;
+  const uint64_t* anc;
+  bf16* out;
+  float* lse;
+  float* partial;           // [B*H][nsplit][NQ][DH+2]
+  unsigned int* counters;   // [B*H]
+  int32_t* status;
+  int n, H, max_pages, nsplit, oob_row;
+  float scale_log2;
+};
+
+template <int DH, int WQ, int WK, int STAGES>
+__global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(const __grid_constant__ CUtensorMap tmK,
+                                                                          const __grid_constant__ CUtensorMap tmV,
+                                                                          const AttnParams p) {
+  constexpr int NW = WQ * WK;               // compute warps
+  constexpr int NQ = WQ * 16;               // query rows of this CTA
+  constexpr int KW = TILE / WK;             // keys per warp per tile
+  constexpr int NT = KW / 8;                // 8-key score tiles per warp
+  constexpr int HALVES = DH / 64;
+  constexpr uint32_t HALF_BYTES = TILE * 128;
+  constexpr uint32_t KV_BYTES = HALVES * HALF_BYTES;      // one of K or V for a stage
+  constexpr uint32_t STAGE_BYTES = 2 * KV_BYTES;
+  constexpr int ROWF = DH + 2;                            // merge row: O[DH], m, l
+  static_assert(NQ * ROWF * 4 <= STAGES * STAGE_BYTES, "merge buffer must fit in the stage ring");
+
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[STAGES];
+  __shared__ __align__(8) uint64_t empty_bar[STAGES];
+  __shared__ int page_list[kMaxPagesPerCta];
+  __shared__ int aborted_s;
+  __shared__ unsigned int ticket_s;
+  volatile int* aborted = &aborted_s;
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int L = p.len[b];
+  const int nq = p.n_active ? min(p.n_active[b], p.n) : p.n;
+  if (nq <= 0) return;
+  const int kv_total = L + nq;
+  const int tiles = (kv_total + TILE - 1) / TILE;
+  const int per = (tiles + p.nsplit - 1) / p.nsplit;
+  const int t0 = min(tiles, split * per), t1 = min(tiles, t0 + per);
+  const bool too_long = per * PAGES_PER_TILE > kMaxPagesPerCta;
+
+  if (threadIdx.x == 0) {
+    aborted_s = 0;
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), NW);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (too_long) atomicExch(p.status, CERB_E_SHAPE);
+  }
+  __syncthreads();
+  const int t_end = too_long ? t0 : t1;
+
+  float* mrg = reinterpret_cast<float*>(smem_gen);   // [NQ][ROWF], used after the key loop
+
+  if (warp == NW) {
+    // ---------------- producer warp ----------------
+    const int32_t* pt = p.page_table + (size_t)b * p.max_pages;
+    const int n_pages = (t_end - t0) * PAGES_PER_TILE;
+    for (int i = lane; i < n_pages; i += 32) {
+      int lp = t0 * PAGES_PER_TILE + i;
+      page_list[i] = (lp * CERB_PAGE < kv_total && lp < p.max_pages) ? (pt[lp] * p.H + h) * CERB_PAGE : p.oob_row;
+    }
+    __syncwarp();
+    if (lane == 0) {
+      for (int t = t0, i = 0; t < t_end; ++t, ++i) {
+        int s = i % STAGES;
+        uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+        mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, aborted, p.status);
+        uint32_t fb = smem_u32(&full_bar[s]);
+        mbar_expect_tx(fb, STAGE_BYTES);
+        uint32_t kdst = smem_base + (uint32_t)s * STAGE_BYTES, vdst = kdst + KV_BYTES;
+#pragma unroll
+        for (int pg = 0; pg < PAGES_PER_TILE; ++pg) {
+          int row = page_list[i * PAGES_PER_TILE + pg];      // out-of-range rows are zero-filled by TMA
+#pragma unroll
+          for (int hf = 0; hf < HALVES; ++hf) {
+            uint32_t off = (uint32_t)hf * HALF_BYTES + (uint32_t)pg * (CERB_PAGE * 128);
+            tma_load_2d(kdst + off, &tmK, hf * 64, row, fb);
+            tma_load_2d(vdst + off, &tmV, hf * 64, row, fb);
+          }
+        }
+      }
+    }
+  } else {
+    // ---------------- compute warps ----------------
+    const int qi = warp % WQ, ki = warp / WQ;
+    const int g = lane >> 2, tq = lane & 3;
+    const int r0 = qi * 16 + g, r1 = r0 + 8;                // this thread's two query rows
+    // Q fragments straight from global memory (A operand of m16n8k16, one per 16 head-dim elements)
+    uint32_t qa[DH / 16][4];
+    {
+      const bf16* q0 = p.q + (((size_t)b * p.n + r0) * p.H + h) * DH;
+      const bf16* q1 = p.q + (((size_t)b * p.n + r1) * p.H + h) * DH;
+#pragma unroll
+      for (int kk = 0; kk < DH / 16; ++kk) {
+        int c = kk * 16 + tq * 2;
+        qa[kk][0] = r0 < nq ? *reinterpret_cast<const uint32_t*>(q0 + c) : 0u;
+        qa[kk][1] = r1 < nq ? *reinterpret_cast<const uint32_t*>(q1 + c) : 0u;
+        qa[kk][2] = r0 < nq ? *reinterpret_cast<const uint32_t*>(q0 + c + 8) : 0u;
+        qa[kk][3] = r1 < nq ? *reinterpret_cast<const uint32_t*>(q1 + c + 8) : 0u;
+      }
+    }
+    uint64_t anc0[2] = {0, 0}, anc1[2] = {0, 0};
+    if (r0 < nq) { anc0[0] = p.anc[r0 * 2]; anc0[1] = p.anc[r0 * 2 + 1]; }
+    if (r1 < nq) { anc1[0] = p.anc[r1 * 2]; anc1[1] = p.anc[r1 * 2 + 1]; }
+
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+    float o[DH / 8][4];
+#pragma unroll
+    for (int i = 0; i < DH / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
+
+    for (int t = t0, it = 0; t < t_end; ++t, ++it) {
+      const int s = it % STAGES;
+      const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
+      mbar_wait(smem_u32(&full_bar[s]), ph, aborted, p.status);
+      const uint32_t kbase = smem_base + (uint32_t)s * STAGE_BYTES, vbase = kbase + KV_BYTES;
+      const int key_tile0 = t * TILE;
+      if (key_tile0 + TILE > kv_total) {
+        // last, partial tile: rows past the end may hold anything (stale pool memory); zero V there so
+        // that a zero probability times a non-finite value cannot poison the sum.
+        const int first_bad = kv_total - key_tile0;
+        uint8_t* vgen = smem_gen + (size_t)s * STAGE_BYTES + KV_BYTES;
+        for (int idx = warp * 32 + lane; idx < (TILE - first_bad) * HALVES * 8; idx += NW * 32) {
+          int row = first_bad + idx / (HALVES * 8), rem = idx % (HALVES * 8);
+          *reinterpret_cast<uint4*>(vgen + (size_t)(rem / 8) * HALF_BYTES + row * 128 + (rem % 8) * 16) = make_uint4(0, 0, 0, 0);
+        }
+        compute_bar(NW * 32);
+      }
+
+      // ---- S = Q K^T for this warp's key slice ----
+      float sc[NT][4];
+#pragma unroll
+      for (int i = 0; i < NT; ++i) { sc[i][0] = sc[i][1] = sc[i][2] = sc[i][3] = 0.f; }
+      const int mat = lane >> 3, lr = lane & 7;
+#pragma unroll
+      for (int kk = 0; kk < DH / 16; ++kk) {
+#pragma unroll
+        for (int nt = 0; nt < NT; nt += 2) {
+          int key = ki * KW + nt * 8 + (mat >> 1) * 8 + lr;
+          int chunk = kk * 2 + (mat & 1);
+          uint32_t addr = kbase + (uint32_t)(chunk >> 3) * HALF_BYTES + (uint32_t)key * 128 + (uint32_t)(((chunk & 7) ^ (key & 7)) << 4);
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4(addr, b0, b1, b2, b3);
+          mma_bf16(sc[nt], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b0, b1);
+          mma_bf16(sc[nt + 1], qa[kk][0], qa[kk][1], qa[kk][2], qa[kk][3], b2, b3);
+        }
+      }
+
+      // ---- mask, online softmax ----
+      const bool need_mask = key_tile0 + TILE > L;
+      float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float v = sc[nt][e] * p.scale_log2;
+          if (need_mask) {
+            int kpos = key_tile0 + ki * KW + nt * 8 + tq * 2 + (e & 1);
+            bool vis = kpos < L;
+            if (!vis && kpos < kv_total) {
+              int j = kpos - L;
+              const uint64_t* a = (e < 2) ? anc0 : anc1;
+              vis = (a[j >> 6] >> (j & 63)) & 1ull;
+            }
+            if (!vis) v = -INFINITY;
+          }
+          sc[nt][e] = v;
+          if (e < 2) mx0 = fmaxf(mx0, v); else mx1 = fmaxf(mx1, v);
+        }
+      }
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+      mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+      mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+      const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+      const float mu0 = mn0 == -INFINITY ? 0.f : mn0, mu1 = mn1 == -INFINITY ? 0.f : mn1;
+      const float al0 = exp2f(m0 - mu0), al1 = exp2f(m1 - mu1);
+      m0 = mn0; m1 = mn1;
+      float rs0 = 0.f, rs1 = 0.f;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        sc[nt][0] = exp2f(sc[nt][0] - mu0); sc[nt][1] = exp2f(sc[nt][1] - mu0);
+        sc[nt][2] = exp2f(sc[nt][2] - mu1); sc[nt][3] = exp2f(sc[nt][3] - mu1);
+        rs0 += sc[nt][0] + sc[nt][1];
+        rs1 += sc[nt][2] + sc[nt][3];
+      }
+      l0 = l0 * al0 + rs0;
+      l1 = l1 * al1 + rs1;
+#pragma unroll
+      for (int i = 0; i < DH / 8; ++i) { o[i][0] *= al0; o[i][1] *= al0; o[i][2] *= al1; o[i][3] *= al1; }
+
+      // ---- O += P V ----
+#pragma unroll
+      for (int j = 0; j < KW / 16; ++j) {
+        uint32_t a0 = pack_bf16(sc[2 * j][0], sc[2 * j][1]);
+        uint32_t a1 = pack_bf16(sc[2 * j][2], sc[2 * j][3]);
+        uint32_t a2 = pack_bf16(sc[2 * j + 1][0], sc[2 * j + 1][1]);
+        uint32_t a3 = pack_bf16(sc[2 * j + 1][2], sc[2 * j + 1][3]);
+#pragma unroll
+        for (int dn = 0; dn < DH / 8; dn += 2) {
+          int key = ki * KW + j * 16 + (mat & 1) * 8 + lr;
+          int chunk = dn + (mat >> 1);
+          uint32_t addr = vbase + (uint32_t)(chunk >> 3) * HALF_BYTES + (uint32_t)key * 128 + (uint32_t)(((chunk & 7) ^ (key & 7)) << 4);
+          uint32_t b0, b1, b2, b3;
+          ldsm_x4_t(addr, b0, b1, b2, b3);
+          mma_bf16(o[dn], a0, a1, a2, a3, b0, b1);
+          mma_bf16(o[dn + 1], a0, a1, a2, a3, b2, b3);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&empty_bar[s]));
+    }
+
+    // ---- combine the WK key slices of each query block, through shared memory ----
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+    compute_bar(NW * 32);                       // every warp is done with the stage ring
+    for (int kslice = 0; kslice < WK; ++kslice) {
+      if (ki == kslice) {
+        float* row0 = mrg + (size_t)r0 * ROWF;
+        float* row1 = mrg + (size_t)r1 * ROWF;
+        if (kslice == 0) {
+#pragma unroll
+          for (int i = 0; i < DH / 8; ++i) {
+            int c = i * 8 + tq * 2;
+            row0[c] = o[i][0]; row0[c + 1] = o[i][1]; row1[c] = o[i][2]; row1[c + 1] = o[i][3];
+          }
+          if (tq == 0) { row0[DH] = m0; row0[DH + 1] = l0; row1[DH] = m1; row1[DH + 1] = l1; }
+        } else {
+          float pm0 = row0[DH], pl0 = row0[DH + 1], pm1 = row1[DH], pl1 = row1[DH + 1];
+          float n0 = fmaxf(pm0, m0), n1 = fmaxf(pm1, m1);
+          float u0 = n0 == -INFINITY ? 0.f : n0, u1 = n1 == -INFINITY ? 0.f : n1;
+          float wa0 = exp2f(pm0 - u0), wb0 = exp2f(m0 - u0), wa1 = exp2f(pm1 - u1), wb1 = exp2f(m1 - u1);
+#pragma unroll
+          for (int i = 0; i < DH / 8; ++i) {
+            int c = i * 8 + tq * 2;
+            row0[c] = row0[c] * wa0 + o[i][0] * wb0; row0[c + 1] = row0[c + 1] * wa0 + o[i][1] * wb0;
+            row1[c] = row1[c] * wa1 + o[i][2] * wb1; row1[c + 1] = row1[c + 1] * wa1 + o[i][3] * wb1;
+          }
+          __syncwarp();
+          if (tq == 0) {
+            row0[DH] = n0; row0[DH + 1] = pl0 * wa0 + l0 * wb0;
+            row1[DH] = n1; row1[DH + 1] = pl1 * wa1 + l1 * wb1;
+          }
+        }
+      }
+      compute_bar(NW * 32);
+    }
+
+    // ---- output: final, or partial + fixed-order merge by the last CTA of this (sequence, head) ----
+    const int ct = warp * 32 + lane, nct = NW * 32;
+    const float LN2 = 0.6931471805599453f;
+    if (p.nsplit == 1) {
+      for (int idx = ct; idx < nq * DH; idx += nct) {
+        int r = idx / DH, c = idx % DH;
+        float l = mrg[(size_t)r * ROWF + DH + 1];
+        p.out[(((size_t)b * p.n + r) * p.H + h) * DH + c] = __float2bfloat16_rn(mrg[(size_t)r * ROWF + c] / l);
+      }
+      if (p.lse)
+        for (int r = ct; r < nq; r += nct)
+          p.lse[((size_t)b * p.H + h) * p.n + r] = (mrg[(size_t)r * ROWF + DH] + log2f(mrg[(size_t)r * ROWF + DH + 1])) * LN2;
+    } else {
+      float* part = p.partial + (((size_t)b * p.H + h) * p.nsplit) * (size_t)(NQ * ROWF);
+      float* mine = part + (size_t)split * (NQ * ROWF);
+      for (int idx = ct; idx < nq * ROWF; idx += nct) __stcg(mine + idx, mrg[idx]);
+      __threadfence();
+      compute_bar(NW * 32);
+      if (ct == 0) ticket_s = atomicAdd(&p.counters[b * p.H + h], 1u);
+      compute_bar(NW * 32);
+      if (ticket_s == (unsigned)p.nsplit - 1) {
+        __threadfence();
+        for (int idx = ct; idx < nq * DH; idx += nct) {
+          int r = idx / DH, c = idx % DH;
+          float M = -INFINITY;
+          for (int s2 = 0; s2 < p.nsplit; ++s2) M = fmaxf(M, __ldcg(part + (size_t)s2 * (NQ * ROWF) + r * ROWF + DH));
+          float Lsum = 0.f, acc = 0.f;
+          for (int s2 = 0; s2 < p.nsplit; ++s2) {
+            const float* pr = part + (size_t)s2 * (NQ * ROWF) + r * ROWF;
+            float w = exp2f(__ldcg(pr + DH) - M);
+            Lsum += __ldcg(pr + DH + 1) * w;
+            acc += __ldcg(pr + c) * w;
+          }
+          p.out[(((size_t)b * p.n + r) * p.H + h) * DH + c] = __float2bfloat16_rn(acc / Lsum);
+          if (c == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
+        }
+        if (ct == 0) p.counters[b * p.H + h] = 0u;       // ready for the next launch
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// fp32 path
+// ---------------------------------------------------------------------------------------------
+template <int DH>
+__global__ void __launch_bounds__(128) tree_attn_f32_kernel(const float* __restrict__ q, const float* __restrict__ kpool,
+                                                            const float* __restrict__ vpool,
+                                                            const int32_t* __restrict__ page_table,
+                                                            const int32_t* __restrict__ len,
+                                                            const int32_t* __restrict__ n_active,
+                                                            const uint64_t* __restrict__ anc, float* __restrict__ out,
+                                                            float* __restrict__ lse, int n, int H, int max_pages,
+                                                            float scale) {
+  constexpr int E = DH / 32;
+  __shared__ float s_o[4][DH];
+  __shared__ float s_m[4], s_l[4];
+  const int i = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int nq = n_active ? min(n_active[b], n) : n;
+  if (i >= nq) return;
+  const int L = len[b], warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint64_t a0 = anc[i * 2], a1 = anc[i * 2 + 1];
+  float qv[E], acc[E];
+  const float* qp = q + (((size_t)b * n + i) * H + h) * DH;
+  for (int e = 0; e < E; ++e) { qv[e] = qp[lane + 32 * e]; acc[e] = 0.f; }
+  float m = -INFINITY, l = 0.f;
+  for (int kpos = warp; kpos < L + nq; kpos += 4) {
+    if (kpos >= L) {
+      int j = kpos - L;
+      if (!(((j < 64 ? a0 : a1) >> (j & 63)) & 1ull)) continue;
+    }
+    int page = page_table[(size_t)b * max_pages + kpos / CERB_PAGE];
+    size_t off = (((size_t)page * H + h) * CERB_PAGE + kpos % CERB_PAGE) * DH;
+    float s = 0.f;
+    for (int e = 0; e < E; ++e) s += qv[e] * kpool[off + lane + 32 * e];
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    s *= scale;
+    float mn = fmaxf(m, s), al = expf(m - mn), pw = expf(s - mn);
+    l = l * al + pw;
+    for (int e = 0; e < E; ++e) acc[e] = acc[e] * al + pw * vpool[off + lane + 32 * e];
+    m = mn;
+  }
+  for (int e = 0; e < E; ++e) s_o[warp][lane + 32 * e] = acc[e];
+  if (lane == 0) { s_m[warp] = m; s_l[warp] = l; }
+  __syncthreads();
+  float M = fmaxf(fmaxf(s_m[0], s_m[1]), fmaxf(s_m[2], s_m[3]));
+  float Ls = 0.f;
+  for (int w = 0; w < 4; ++w) Ls += s_m[w] == -INFINITY ? 0.f : s_l[w] * expf(s_m[w] - M);
+  for (int c = threadIdx.x; c < DH; c += 128) {
+    float a = 0.f;
+    for (int w = 0; w < 4; ++w) a += s_m[w] == -INFINITY ? 0.f : s_o[w][c] * expf(s_m[w] - M);
+    out[(((size_t)b * n + i) * H + h) * DH + c] = a / Ls;
+  }
+  if (threadIdx.x == 0 && lse) lse[((size_t)b * H + h) * n + i] = M + logf(Ls);
+}
+
+int plan_nsplit(int B, int H, int max_len) {
+  int tiles = (max_len + TILE - 1) / TILE;
+  if (tiles < 1) tiles = 1;
+  int want = (kTargetCtas + B * H - 1) / (B * H);
+  if (want > kMaxSplit) want = kMaxSplit;
+  if (want > tiles) want = tiles;
+  if (want < 1) want = 1;
+  int per = (tiles + want - 1) / want;
+  if (per * PAGES_PER_TILE > kMaxPagesPerCta) return -1;       // more than 16K keys per split
+  return (tiles + per - 1) / per;
+}
+
+inline int nq_pad(int n) { return n <= 16 ? 16 : n <= 32 ? 32 : n <= 64 ? 64 : 128; }
+
+template <int DH, int WQ, int WK, int STAGES>
+int launch_cfg(const AttnParams& p, const CUtensorMap* tmK, const CUtensorMap* tmV, int B, cudaStream_t st) {
+  constexpr size_t smem = (size_t)STAGES * 2 * (DH / 64) * TILE * 128 + 1024;
+  static bool configured = false;
+  if (!configured) {
+    CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_bf16_kernel<DH, WQ, WK, STAGES>,
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    configured = true;
+  }
+  dim3 grid(p.nsplit, p.H, B);
+  tree_attn_bf16_kernel<DH, WQ, WK, STAGES><<<grid, (WQ * WK + 1) * 32, smem, st>>>(*tmK, *tmV, p);
+  return CERB_OK;
+}
+
+}  // namespace
+
+size_t attn_scratch_bytes(int B, int n, int H, int Dh) {
+  size_t rows = (size_t)(kTargetCtas + B * H + kMaxSplit);
+  return kCounterBytes + rows * (size_t)nq_pad(n) * (size_t)(Dh + 2) * sizeof(float);
+}
+
+int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMap* tmK, const CUtensorMap* tmV,
+                          int sm_count, int32_t* status, cudaStream_t st) {
+  (void)sm_count;
+  if (a->dtype == CERB_F32) {
+    dim3 grid(a->n, a->n_heads, a->B);
+    if (a->head_dim == 64)
+      tree_attn_f32_kernel<64><<<grid, 128, 0, st>>>((const float*)a->q, (const float*)a->k_pool, (const float*)a->v_pool,
+                                                     a->page_table, a->len, a->n_active, a->anc, (float*)a->out, a->lse,
+                                                     a->n, a->n_heads, a->max_pages, a->scale);
+    else if (a->head_dim == 128)
+      tree_attn_f32_kernel<128><<<grid, 128, 0, st>>>((const float*)a->q, (const float*)a->k_pool, (const float*)a->v_pool,
+                                                      a->page_table, a->len, a->n_active, a->anc, (float*)a->out, a->lse,
+                                                      a->n, a->n_heads, a->max_pages, a->scale);
+    else
+      return CERB_E_SHAPE;
+    CERB_LAUNCH_CHECK(c);
+    return CERB_OK;
+  }
+  if (a->B * a->n_heads > (int)(kCounterBytes / sizeof(unsigned int))) return CERB_E_SHAPE;
+  AttnParams p;
+  p.q = (const bf16*)a->q;
+  p.page_table = a->page_table;
+  p.len = a->len;
+  p.n_active = a->n_active;
+  p.anc = a->anc;
+  p.out = (bf16*)a->out;
+  p.lse = a->lse;
+  p.counters = (unsigned int*)a->scratch;
+  p.partial = (float*)((char*)a->scratch + kCounterBytes);
+  p.status = status;
+  p.n = a->n;
+  p.H = a->n_heads;
+  p.max_pages = a->max_pages;
+  p.nsplit = plan_nsplit(a->B, a->n_heads, a->max_len);
+  if (p.nsplit < 1) return CERB_E_SHAPE;
+  p.oob_row = a->n_pool_pages * a->n_heads * CERB_PAGE;
+  p.scale_log2 = a->scale * 1.4426950408889634f;
+  if (a->scratch_bytes < attn_scratch_bytes(a->B, a->n, a->n_heads, a->head_dim)) return CERB_E_NOMEM;
+  int np = nq_pad(a->n), rc = CERB_E_SHAPE;
+  if (a->head_dim == 128) {
+    if (np == 16) rc = launch_cfg<128, 1, 4, 3>(p, tmK, tmV, a->B, st);
+    else if (np == 32) rc = launch_cfg<128, 2, 4, 3>(p, tmK, tmV, a->B, st);
+    else if (np == 64) rc = launch_cfg<128, 4, 2, 3>(p, tmK, tmV, a->B, st);
+    else rc = launch_cfg<128, 8, 1, 3>(p, tmK, tmV, a->B, st);
+  } else if (a->head_dim == 64) {
+    if (np == 16) rc = launch_cfg<64, 1, 4, 4>(p, tmK, tmV, a->B, st);
+    else if (np == 32) rc = launch_cfg<64, 2, 4, 4>(p, tmK, tmV, a->B, st);
+    else if (np == 64) rc = launch_cfg<64, 4, 2, 4>(p, tmK, tmV, a->B, st);
+    else rc = launch_cfg<64, 8, 1, 4>(p, tmK, tmV, a->B, st);
+  }
+  if (rc != CERB_OK) return rc;
+  CERB_LAUNCH_CHECK(c);
+  return CERB_OK;
+}
+
+}  // namespace cerb

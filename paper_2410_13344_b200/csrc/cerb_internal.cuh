@@ -131,7 +131,8 @@ int launch_rope_append(cerb_ctx* c, int layer, const TreeDev& t, const float* pa
 int launch_residual(cerb_ctx* c, void* x, const float* part, int nsplit, size_t split_stride, int rows, int N,
                     cudaStream_t st);
 int launch_swiglu(cerb_ctx* c, const float* part, int nsplit, size_t split_stride, void* act, int rows, cudaStream_t st);
-int launch_argmax_rows(cerb_ctx* c, const float* logits, int rows, int V, int32_t* out, cudaStream_t st);
+int launch_argmax_rows(cerb_ctx* c, const float* part, int nsplit, size_t split_stride, int rows, int V, int32_t* out,
+                       float* summed, cudaStream_t st);
 int launch_set_nactive(cerb_ctx* c, int mode, int a, int b, cudaStream_t st);
 int launch_prefill_commit(cerb_ctx* c, int n, cudaStream_t st);
 

@@ -123,14 +123,19 @@ __global__ void swiglu_kernel(const float* __restrict__ part, int nsplit, size_t
   stf(act + i, g / (1.0f + expf(-g)) * u);
 }
 
-__global__ void argmax_rows_kernel(const float* __restrict__ logits, int V, int32_t* __restrict__ out) {
+// Row argmax over logits given as split-K partial sums; ties go to the lower index.  When
+// `summed` is not null the summed logits are also written there ([rows][V]).
+__global__ void argmax_rows_kernel(const float* __restrict__ part, int nsplit, size_t split_stride, int V,
+                                   int32_t* __restrict__ out, float* __restrict__ summed) {
   __shared__ float sv[32];
   __shared__ int si[32];
-  const float* r = logits + (size_t)blockIdx.x * V;
+  const float* r = part + (size_t)blockIdx.x * V;
   float best = -INFINITY;
   int bi = 0x7fffffff;
   for (int j = threadIdx.x; j < V; j += blockDim.x) {
-    float v = r[j];
+    float v = 0.f;
+    for (int s = 0; s < nsplit; ++s) v += r[s * split_stride + j];
+    if (summed) summed[(size_t)blockIdx.x * V + j] = v;
     if (v > best || (v == best && j < bi)) { best = v; bi = j; }
   }
   for (int o = 16; o > 0; o >>= 1) {
@@ -237,8 +242,9 @@ int launch_swiglu(cerb_ctx* c, const float* part, int nsplit, size_t split_strid
   return CERB_OK;
 }
 
-int launch_argmax_rows(cerb_ctx* c, const float* logits, int rows, int V, int32_t* out, cudaStream_t st) {
-  argmax_rows_kernel<<<rows, 1024, 0, st>>>(logits, V, out);
+int launch_argmax_rows(cerb_ctx* c, const float* part, int nsplit, size_t split_stride, int rows, int V, int32_t* out,
+                       float* summed, cudaStream_t st) {
+  argmax_rows_kernel<<<rows, 1024, 0, st>>>(part, nsplit, split_stride, V, out, summed);
   CERB_LAUNCH_CHECK(c);
   return CERB_OK;
 }
