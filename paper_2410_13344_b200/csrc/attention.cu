@@ -488,7 +488,7 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
     CERB_LAUNCH_CHECK(c);
     return CERB_OK;
   }
-  if (a->B * a->n_heads > (int)(kCounterBytes / sizeof(unsigned int))) return CERB_E_SHAPE;
+  if (a->B * a->n_heads > (int)(kCounterBytes / sizeof(unsigned int)) - 4) return CERB_E_SHAPE;   // last 16 bytes: status word
   AttnParams p;
   p.q = (const bf16*)a->q;
   p.page_table = a->page_table;

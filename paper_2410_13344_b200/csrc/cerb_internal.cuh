@@ -86,7 +86,7 @@ struct cerb_ctx {
 
   // workspace carve-out
   int32_t *d_len, *d_len_old, *d_root, *d_nactive, *d_status, *d_lens_in, *d_mode, *d_naccept;
-  int32_t *d_path, *d_outtok, *d_argmax, *d_treetok, *d_topk;
+  int32_t *d_path, *d_outtok, *d_argmax, *d_treetok, *d_topk, *d_kper;
   float* d_S;
   void *d_hlast, *d_x, *d_xn, *d_q, *d_attn, *d_act, *d_hidden;
   float *d_part, *d_logits, *d_hlogits;
