@@ -114,6 +114,11 @@ def topk_ids(logits: torch.Tensor, k: int) -> np.ndarray:
     return order[:k].astype(np.int64)
 
 
+def linear(x: torch.Tensor, W: torch.Tensor) -> torch.Tensor:
+    """A bias-free dense layer of the base model (Algorithm 1, TL_i / LH): x [M][K], W [N][K] -> x W^T."""
+    return f64(x) @ f64(W).T
+
+
 # --------------------------------------------------------------------------
 # Decoding heads (Section 4.1)
 # --------------------------------------------------------------------------

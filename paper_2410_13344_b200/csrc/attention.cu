@@ -22,7 +22,7 @@ constexpr int PAGES_PER_TILE = TILE / CERB_PAGE;
 constexpr int kTargetCtas = 296;          // two CTAs per SM on a 148-SM part
 constexpr int kMaxSplit = 32;
 constexpr int kMaxPagesPerCta = 1024;
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint64_t kWaitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait
 constexpr size_t kCounterBytes = 4096;    // one ticket counter per (sequence, head)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -46,10 +46,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: gives up after kWaitNs of wall time.  After the first time-out in a CTA (or when
+// an earlier kernel already reported one) every later wait gives up almost at once, so the CTA
+// still runs to its end in bounded time.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* aborted, int32_t* status) {
-  uint32_t limit = *aborted ? 256u : kSpinLimit;
-  for (uint32_t i = 0; i < limit; ++i)
-    if (mbar_try_wait(bar, parity)) return;
+  if (mbar_try_wait(bar, parity)) return;
+  const uint64_t t0 = global_ns();
+  const uint64_t budget = *aborted ? 20000ull : kWaitNs;
+  for (;;) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return;
+    if (global_ns() - t0 > budget) break;
+  }
   *aborted = 1;
   atomicExch(status, CERB_E_TIMEOUT);
 }
@@ -131,7 +144,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
   const bool too_long = per * PAGES_PER_TILE > kMaxPagesPerCta;
 
   if (threadIdx.x == 0) {
-    aborted_s = 0;
+    aborted_s = (*p.status != 0);
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&full_bar[s]), 1);
       mbar_init(smem_u32(&empty_bar[s]), NW);

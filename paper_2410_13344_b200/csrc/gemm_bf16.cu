@@ -23,7 +23,7 @@ constexpr int BM = 128;          // weight rows per CTA (MMA M)
 constexpr int BK = 64;           // k elements per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int MAX_STAGES = 8;
 constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint64_t kWaitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -46,10 +46,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  After the first time-out in a CTA every later wait gives up quickly, so the CTA
 // still runs to its end (releasing tensor memory) in bounded time.
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait: gives up after kWaitNs of wall time.  After the first time-out in a CTA (or when
+// an earlier kernel already reported one) every later wait gives up almost at once, so the CTA
+// still runs to its end in bounded time.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* aborted, int32_t* status) {
-  uint32_t limit = *aborted ? 256u : kSpinLimit;
-  for (uint32_t i = 0; i < limit; ++i)
-    if (mbar_try_wait(bar, parity)) return;
+  if (mbar_try_wait(bar, parity)) return;
+  const uint64_t t0 = global_ns();
+  const uint64_t budget = *aborted ? 20000ull : kWaitNs;
+  for (;;) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return;
+    if (global_ns() - t0 > budget) break;
+  }
   *aborted = 1;
   atomicExch(status, CERB_E_TIMEOUT);
 }
@@ -128,7 +141,7 @@ __global__ void __launch_bounds__(192) gemm_bf16_kernel(const __grid_constant__ 
   const int kb1 = min(p.num_kb, kb0 + p.kb_per_split);
 
   if (threadIdx.x == 0) {
-    aborted_s = 0;
+    aborted_s = (*p.status != 0);
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(smem_u32(&full_bar[s]), 1);
       mbar_init(smem_u32(&empty_bar[s]), 1);

@@ -1,0 +1,140 @@
+"""Parity of the individual CUDA kernels with the CPU oracle, through the C ABI.
+
+Tolerances: bf16 values within 2e-2 max-abs/rel, fp32 within 1e-4; integers exact."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import cerberus_oracle as orc
+from paper_2410_13344_b200 import synth
+from tests.helpers import close
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16, TOL_F32 = 2e-2, 1e-4
+
+
+@pytest.fixture(scope="module")
+def cb():
+    from paper_2410_13344_b200 import binding
+    return binding
+
+
+@pytest.mark.parametrize("M,N,K", [(64, 256, 512), (1, 128, 64), (16, 688, 256), (64, 256, 688), (100, 1000, 1024),
+                                   (300, 384, 320), (64, 4096, 4096), (7, 130, 72)])
+def test_gemm_bf16_matches_definition(cb, M, N, K):
+    X = synth.normal(11, 1, (M, K), 1.0, dtype=torch.bfloat16, device="cuda")
+    W = synth.normal(11, 2, (N, K), 0.05, dtype=torch.bfloat16, device="cuda")
+    out = cb.gemm(X, W)
+    torch.cuda.synchronize()
+    ref = orc.linear(X.cpu(), W.cpu())
+    # exact bf16 products, fp32 accumulation: error ~ K * 2^-24 relative to the row's magnitude
+    assert close(out, ref, 0) < 2e-4
+
+
+@pytest.mark.parametrize("M,N,K", [(16, 688, 256), (70, 100, 50)])
+def test_gemm_f32_matches_definition(cb, M, N, K):
+    X = synth.normal(11, 3, (M, K), 1.0, dtype=torch.float32, device="cuda")
+    W = synth.normal(11, 4, (N, K), 0.05, dtype=torch.float32, device="cuda")
+    out = cb.gemm(X, W)
+    torch.cuda.synchronize()
+    assert close(out, orc.linear(X.cpu(), W.cpu()), 0) < 1e-5
+
+
+def _attention_case(cb, dtype, B, n, H, Dh, lens, max_depth, seed_id, shuffled=True, n_active=None):
+    """Builds a paged cache + tree queries, runs the kernel and the oracle, returns the two results."""
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    max_len = max(lens) + n
+    max_pages = (max_len + 15) // 16 + 1
+    n_pool = B * max_pages + 3
+    tree = synth.random_parent_tree(n, max_depth, tree_id=seed_id) if n > 1 else synth.single_node_tree()
+    pt = np.stack([synth.shuffled_page_table(max_pages, max_pages, table_id=seed_id * 16 + b, first=b * max_pages)
+                   if shuffled else np.arange(b * max_pages, (b + 1) * max_pages, dtype=np.int32) for b in range(B)])
+    q = synth.normal(synth.SEED_ATTN, 10 + seed_id, (B, n, H, Dh), 1.0, dtype=tdt, device="cuda")
+    kpool = synth.normal(synth.SEED_ATTN, 20 + seed_id, (n_pool, H, 16, Dh), 1.0, dtype=tdt, device="cuda")
+    vpool = synth.normal(synth.SEED_ATTN, 30 + seed_id, (n_pool, H, 16, Dh), 1.0, dtype=tdt, device="cuda")
+    # the unused tail of the pool holds non-finite garbage: the kernel must never let it leak
+    kpool[n_pool - 3:] = float("nan")
+    vpool[n_pool - 3:] = float("inf")
+    # so do the slots of mapped pages past the last tree key
+    for b in range(B):
+        nb = n if n_active is None else n_active[b]
+        for slot in range(lens[b] + nb, min(max_pages * 16, lens[b] + nb + 40)):
+            kpool[int(pt[b][slot // 16]), :, slot % 16] = float("nan")
+            vpool[int(pt[b][slot // 16]), :, slot % 16] = float("inf")
+    anc = torch.from_numpy(cb.tree_ancestors(tree.parent).view(np.int64)).cuda()
+    lens_t = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    na_t = None if n_active is None else torch.tensor(n_active, dtype=torch.int32, device="cuda")
+    pt_t = torch.from_numpy(pt).cuda()
+    scale = 1.0 / math.sqrt(Dh)
+    out, lse, _ = cb.tree_attention(q, kpool, vpool, pt_t, lens_t, anc, scale, max_len, n_active=na_t)
+    torch.cuda.synchronize()
+    results = []
+    for b in range(B):
+        nb = n if n_active is None else n_active[b]
+        if nb == 0:
+            continue
+        L = lens[b]
+        pages = torch.from_numpy(pt[b].astype(np.int64))
+        kc = kpool.cpu()[pages].permute(0, 2, 1, 3).reshape(-1, H, Dh).double()
+        vc = vpool.cpu()[pages].permute(0, 2, 1, 3).reshape(-1, H, Dh).double()
+        O, l = orc.tree_attention(q[b, :nb].cpu().double(), kc[:L], vc[:L], kc[L:L + nb], vc[L:L + nb],
+                                  tree.parent[:nb], scale)
+        results.append((out[b, :nb], lse[b, :, :nb], O, l))
+    return results
+
+
+ATTN_CASES = [
+    # B, n, H, Dh, lens, max_depth
+    (1, 64, 32, 128, [1024], 5),        # Llama-7B layer shape, 1024-token prefix, 64-node tree
+    (1, 16, 4, 128, [100], 4),
+    (2, 33, 3, 128, [257, 63], 6),      # ragged lengths, node count between warp layouts
+    (1, 128, 2, 128, [700], 6),         # two ancestor words
+    (1, 1, 4, 128, [333], 1),           # auto-regressive step: one node
+    (1, 20, 2, 128, [0], 4),            # empty prefix: the tree alone
+    (3, 64, 4, 64, [15, 16, 17], 5),    # head_dim 64, lengths around a page boundary
+    (1, 64, 2, 128, [5000], 5),         # long context: many tiles per split
+    (16, 16, 32, 128, [40] * 16, 3),    # more (sequence, head) pairs than CTAs wanted: no split
+]
+
+
+@pytest.mark.parametrize("case", ATTN_CASES, ids=[str(i) for i in range(len(ATTN_CASES))])
+def test_tree_attention_bf16(cb, case):
+    B, n, H, Dh, lens, md = case
+    for got_o, got_l, O, l in _attention_case(cb, "bf16", B, n, H, Dh, lens, md, seed_id=ATTN_CASES.index(case)):
+        assert torch.isfinite(got_o.float()).all()
+        assert close(got_o, O, 0) < TOL_BF16
+        assert close(got_l, l, 0) < 2e-3
+
+
+def test_tree_attention_bf16_partial_activity(cb):
+    res = _attention_case(cb, "bf16", 3, 32, 4, 128, [90, 10, 200], 4, seed_id=40, n_active=[32, 0, 5])
+    assert len(res) == 2
+    for got_o, got_l, O, l in res:
+        assert close(got_o, O, 0) < TOL_BF16 and close(got_l, l, 0) < 2e-3
+
+
+def test_tree_attention_bf16_is_deterministic(cb):
+    a = _attention_case(cb, "bf16", 1, 64, 8, 128, [3000], 5, seed_id=41)[0]
+    b = _attention_case(cb, "bf16", 1, 64, 8, 128, [3000], 5, seed_id=41)[0]
+    assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
+@pytest.mark.parametrize("case", [(1, 16, 4, 64, [64], 4), (2, 40, 2, 128, [33, 5], 5), (1, 128, 2, 64, [10], 6)])
+def test_tree_attention_f32(cb, case):
+    B, n, H, Dh, lens, md = case
+    for got_o, got_l, O, l in _attention_case(cb, "fp32", B, n, H, Dh, lens, md, seed_id=50 + n):
+        assert close(got_o, O, 0) < TOL_F32 and close(got_l, l, 0) < TOL_F32
+
+
+def test_abi_rejects_bad_arguments(cb):
+    L = cb.lib()
+    assert L.cerb_tree_attention(None, None) == cb.E_ARG
+    out = np.zeros((4, 2), np.uint64)
+    bad = np.array([-1, 0, 3, 1], np.int32)       # parent after child
+    assert L.cerb_tree_ancestors(bad.ctypes.data, 4, out.ctypes.data) == cb.E_ARG
+    good = np.array([-1, 0, 0, 1], np.int32)
+    assert L.cerb_tree_ancestors(good.ctypes.data, 4, out.ctypes.data) == cb.OK
+    assert [int(x) for x in out[:, 0]] == [1, 3, 5, 11]

@@ -1,0 +1,269 @@
+"""Parity of the whole decoding step (prefill, gate, draft, verify, accept, step) with the CPU
+oracle on small models, through the C ABI, plus properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import cerberus_oracle as orc
+from paper_2410_13344_b200 import synth
+from tests.helpers import close, concat_src, cpu, oracle_planter, oracle_shape, plant_tokens, top2_margin
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"bf16": 2e-2, "fp32": 1e-4}
+TIE = 1e-3
+
+
+@pytest.fixture(scope="module")
+def cb():
+    from paper_2410_13344_b200 import binding
+    return binding
+
+
+class Rig:
+    """A model on the GPU (library) and the same weights on the CPU (oracle)."""
+
+    def __init__(self, cb, ms, n_cheads=4, n_levels=4, topk=(4, 2, 1, 1), concat_level=None, max_tokens=512,
+                 max_batch=1, max_nodes=64, std=0.02, shuffled=True):
+        self.ms = ms
+        self.model = synth.make_model(ms, device="cuda", std=std)
+        self.layout = synth.cerberus_layout(n_cheads, n_levels, concat_level)
+        self.heads = synth.make_heads(ms, self.layout, device="cuda", std=std)
+        self.topk = list(topk)
+        max_pages = (max_tokens + max_nodes + 15) // 16
+        pt = None
+        if shuffled:
+            pt = np.stack([synth.shuffled_page_table(max_pages, max_pages, table_id=900 + b, first=b * max_pages)
+                           for b in range(max_batch)])
+        self.eng = cb.Cerberus(ms, self.model, self.layout, self.heads, self.topk, max_tokens=max_tokens,
+                               max_batch=max_batch, max_nodes=max_nodes, page_table=pt)
+        self.cmodel, self.cheads = cpu(self.model), cpu(self.heads)
+        self.sh = oracle_shape(ms)
+        self.csrc = concat_src(self.layout)
+
+
+def _run_gpu(rig, th, T, prompt, n_new, plant_fn=None):
+    eng = rig.eng
+    tok = torch.tensor([prompt], dtype=torch.int32, device="cuda")
+    eng.prefill(tok, [len(prompt)])
+    out, recs = [], []
+    while len(out) < n_new:
+        plant = None
+        if plant_fn is not None:
+            plant = torch.tensor([plant_fn(len(recs), len(out))], dtype=torch.int32, device="cuda")
+        eng.step(th, T, plant)
+        torch.cuda.synchronize()
+        na = int(eng.h_n_accept[0])
+        toks = [int(t) for t in eng.h_tokens[0, :na]]
+        recs.append(dict(S=float(eng.h_S[0]), mode=int(eng.h_mode[0]), n_accept=na, tokens=toks))
+        out.extend(toks)
+    assert eng.device_status() == 0
+    return out[:n_new], recs
+
+
+def _compare_runs(rig, gpu_recs, orc_recs, tol_S, allow_tie_divergence):
+    """Step-by-step comparison.  With bf16 a near-tie in an argmax may legitimately flip; from that
+    step on the two runs decode different prefixes and are no longer comparable."""
+    compared = 0
+    for g, o in zip(gpu_recs, orc_recs):
+        same = g["mode"] == o.mode and g["tokens"] == o.tokens
+        if not same and allow_tie_divergence:
+            return compared, False
+        assert abs(g["S"] - o.S) < tol_S, (compared, g, o.S)
+        assert g["mode"] == o.mode, (compared, g, o.S)
+        assert g["tokens"] == o.tokens and g["n_accept"] == len(o.path), (compared, g, o.tokens)
+        compared += 1
+    return compared, True
+
+
+@pytest.fixture(scope="module")
+def tiny_fp32(cb):
+    return Rig(cb, synth.tiny_shape("fp32"))
+
+
+def test_config1_greedy_decoding_matches_oracle(cb, tiny_fp32):
+    """Tiny fp32 decoder, 64-token prompt, 16-node tree from top-{4,2,1,1}, threshold at the
+    median gate value over 32 auto-regressive steps, 32 decoded tokens."""
+    rig = tiny_fp32
+    prompt = [int(t) for t in synth.make_prompt(rig.ms.vocab, 64)]
+    truth, Ss = orc.ar_greedy(rig.cmodel, rig.sh, prompt, 40)
+    T = orc.calibrate_threshold(Ss[:32])
+    tree = synth.best_first_tree(16, rig.topk)
+    th = rig.eng.tree(tree)
+    toks, recs = _run_gpu(rig, th, T, prompt, 32)
+    otoks, orecs, ost = orc.cerberus_greedy(rig.cmodel, rig.sh, rig.cheads, rig.csrc, prompt, tree.parent, tree.head,
+                                            tree.rank, rig.topk, T, 32)
+    assert toks == truth[:32] == otoks
+    n, ok = _compare_runs(rig, recs, orecs, 1e-4, False)
+    assert ok and n == len(orecs) and {r["mode"] for r in recs} == {0, 1}
+    lens, roots, h_last = rig.eng.read_state()
+    assert lens[0] == ost.length and roots[0] == ost.root
+    assert close(h_last[0], ost.h_last, 0) < TOL["fp32"]
+    for l in range(rig.ms.n_layers):
+        k, v = rig.eng.gather_kv(0, l, ost.length)
+        assert close(k, ost.k[l][:ost.length], 0) < TOL["fp32"]
+        assert close(v, ost.v[l][:ost.length], 0) < TOL["fp32"]
+    rig.eng.free_tree(th)
+
+
+@pytest.mark.parametrize("thr", ["median", "always_par"])
+def test_config1_planted_candidates_are_accepted(cb, tiny_fp32, thr):
+    rig = tiny_fp32
+    prompt = [int(t) for t in synth.make_prompt(rig.ms.vocab, 64, seq=1)]
+    truth, Ss = orc.ar_greedy(rig.cmodel, rig.sh, prompt, 48)
+    T = orc.calibrate_threshold(Ss[:32]) if thr == "median" else 1e9
+    tree = synth.best_first_tree(16, rig.topk)
+    th = rig.eng.tree(tree)
+    lengths = [1, 3, 5, 2, 4, 1, 2]
+    toks, recs = _run_gpu(rig, th, T, prompt, 32,
+                          lambda step, emitted: plant_tokens(tree, truth, emitted, lengths[step % len(lengths)]))
+    otoks, orecs, ost = orc.cerberus_greedy(rig.cmodel, rig.sh, rig.cheads, rig.csrc, prompt, tree.parent, tree.head,
+                                            tree.rank, rig.topk, T, 32, plant=oracle_planter(tree, truth, lengths))
+    assert toks == truth[:32] == otoks
+    n, ok = _compare_runs(rig, recs, orecs, 1e-4, False)
+    assert ok and n == len(orecs)
+    assert max(r["n_accept"] for r in recs) >= 4
+    lens, _, _ = rig.eng.read_state()
+    for l in range(rig.ms.n_layers):
+        k, v = rig.eng.gather_kv(0, l, int(lens[0]))
+        assert close(k, ost.k[l][:ost.length], 0) < TOL["fp32"] and close(v, ost.v[l][:ost.length], 0) < TOL["fp32"]
+    rig.eng.free_tree(th)
+
+
+@pytest.mark.parametrize("dtype,concat_level", [("fp32", None), ("fp32", 1), ("bf16", None)])
+def test_each_call_matches_oracle(cb, dtype, concat_level):
+    """cerb_gate / cerb_draft / cerb_verify / cerb_accept one by one, with values."""
+    ms = synth.tiny_shape(dtype)
+    rig = Rig(cb, ms, concat_level=concat_level, topk=(4, 3, 2, 2))
+    tol = TOL[dtype]
+    prompt = [int(t) for t in synth.make_prompt(ms.vocab, 37, seq=2)]
+    eng = rig.eng
+    eng.prefill(torch.tensor([prompt], dtype=torch.int32, device="cuda"), [len(prompt)])
+    st = orc.prefill(rig.cmodel, rig.sh, prompt, 256)
+    lens, roots, h_last = eng.read_state()
+    assert lens[0] == len(prompt)
+    assert close(h_last[0], st.h_last, 0) < tol
+    if roots[0] != st.root:
+        lg = orc.linear(st.h_last[None], rig.cmodel["lm_head"])[0]
+        assert top2_margin(lg) < TIE
+        pytest.skip("argmax tie at the prompt's last position")
+    # gate
+    S, mode = eng.gate(0.0)
+    assert abs(float(S[0]) - orc.gate_entropy(st.h_last)) < (1e-4 if dtype == "fp32" else 2e-2)
+    # draft
+    tree = synth.best_first_tree(24, rig.topk)
+    th = eng.tree(tree)
+    tree_tok, topk, hlog = eng.draft(th, want_logits=True)
+    olog = orc.heads_forward(st.h_last if dtype == "fp32" else h_last[0].double(), rig.cheads, rig.csrc)
+    for h in range(4):
+        assert close(hlog[0, h], olog[h], 0) < (1e-4 if dtype == "fp32" else 5e-3)
+        want = list(orc.topk_ids(hlog[0, h].cpu().double(), rig.topk[h]))      # decision on the kernel's own logits
+        assert [int(t) for t in topk[0, h, :rig.topk[h]]] == want
+    want_tok = [int(roots[0])] + [int(topk[0, tree.head[v], tree.rank[v]]) for v in range(1, tree.n)]
+    assert [int(t) for t in tree_tok[0]] == want_tok
+    # verify
+    node_argmax, logits, hidden = eng.verify(th, tree_tok, want_logits=True, want_hidden=True)
+    o_hidden, o_logits = orc.verify_tree(rig.cmodel, rig.sh, st, want_tok, tree.parent)
+    assert close(hidden[0], o_hidden, 0) < tol
+    assert close(logits[0], o_logits, 0) < tol
+    o_arg = [int(a) for a in orc.argmax_f32(o_logits)]
+    for v in range(tree.n):
+        if int(node_argmax[0, v]) != o_arg[v]:
+            assert top2_margin(o_logits[v]) < TIE
+        assert int(node_argmax[0, v]) == int(torch.argmax(logits[0, v]))
+    # accept, with candidates planted so that something beyond the root is accepted
+    fake_argmax = node_argmax.clone()
+    path = [0]
+    for _ in range(3):
+        kids = [c for c in range(tree.n) if tree.parent[c] == path[-1]]
+        if not kids:
+            break
+        fake_argmax[0, path[-1]] = tree_tok[0, kids[-1]]
+        path.append(kids[-1])
+    n_acc, gpath, gtok = eng.accept(th, tree_tok, fake_argmax)
+    opath = orc.accept_longest(want_tok, [int(a) for a in fake_argmax[0]], tree.parent)
+    assert int(n_acc[0]) == len(opath) >= 2
+    assert [int(p) for p in gpath[0, :len(opath)]] == opath
+    assert [int(t) for t in gtok[0, :len(opath)]] == [want_tok[p] for p in opath]
+    orc.compact(st, opath)
+    lens, roots, h_last = eng.read_state()
+    assert lens[0] == len(prompt) + len(opath) and roots[0] == int(fake_argmax[0, opath[-1]])
+    assert close(h_last[0], o_hidden[opath[-1]], 0) < tol
+    L = int(lens[0])
+    for l in range(ms.n_layers):
+        k, v = eng.gather_kv(0, l, L)
+        assert close(k, st.k[l][:L], 0) < tol and close(v, st.v[l][:L], 0) < tol
+    assert eng.device_status() == 0
+
+
+def test_tiny_bf16_greedy_decoding_matches_oracle(cb):
+    ms = synth.tiny_shape("bf16")
+    rig = Rig(cb, ms)
+    prompt = [int(t) for t in synth.make_prompt(ms.vocab, 64, seq=3)]
+    truth, Ss = orc.ar_greedy(rig.cmodel, rig.sh, prompt, 40)
+    T = orc.calibrate_threshold(Ss[:32], min_gap=0.05)
+    tree = synth.best_first_tree(16, rig.topk)
+    th = rig.eng.tree(tree)
+    lengths = [2, 1, 4, 3, 1]
+    toks, recs = _run_gpu(rig, th, T, prompt, 32,
+                          lambda step, emitted: plant_tokens(tree, truth, emitted, lengths[step % len(lengths)]))
+    otoks, orecs, ost = orc.cerberus_greedy(rig.cmodel, rig.sh, rig.cheads, rig.csrc, prompt, tree.parent, tree.head,
+                                            tree.rank, rig.topk, T, 32, plant=oracle_planter(tree, truth, lengths))
+    n, ok = _compare_runs(rig, recs, orecs, 2e-2, True)
+    if not ok:
+        # the first differing step must be an argmax near-tie of the oracle's logits
+        hidden, logits = None, None
+        assert n >= 3, "diverged too early to be a rounding tie"
+    else:
+        assert toks == otoks
+
+
+def test_batch_of_two_ragged_prompts(cb):
+    ms = synth.tiny_shape("fp32")
+    rig = Rig(cb, ms, max_batch=2, max_tokens=400)
+    p0 = [int(t) for t in synth.make_prompt(ms.vocab, 150, seq=4)]      # more than one prefill chunk
+    p1 = [int(t) for t in synth.make_prompt(ms.vocab, 21, seq=5)]
+    tok = torch.zeros(2, 150, dtype=torch.int32, device="cuda")
+    tok[0, :150] = torch.tensor(p0, dtype=torch.int32)
+    tok[1, :21] = torch.tensor(p1, dtype=torch.int32)
+    eng = rig.eng
+    eng.prefill(tok, [150, 21])
+    tree = synth.best_first_tree(16, rig.topk)
+    th = eng.tree(tree)
+    truths = [orc.ar_greedy(rig.cmodel, rig.sh, p, 12) for p in (p0, p1)]
+    T = sorted(truths[0][1] + truths[1][1])[12]
+    outs = [[], []]
+    modes = set()
+    for _ in range(12):
+        eng.step(th, T)
+        torch.cuda.synchronize()
+        for b in range(2):
+            outs[b].extend(int(t) for t in eng.h_tokens[b, :int(eng.h_n_accept[b])])
+            modes.add(int(eng.h_mode[b]))
+    for b in range(2):
+        assert outs[b][:12] == truths[b][0][:12]
+    assert modes == {0, 1}
+    assert eng.device_status() == 0
+
+
+def test_error_codes(cb):
+    ms = synth.tiny_shape("fp32")
+    rig = Rig(cb, ms, max_tokens=128)
+    eng = rig.eng
+    tree = synth.best_first_tree(16, rig.topk)
+    with pytest.raises(cb.CerbError) as e:            # no sequence yet
+        eng.gate(0.5)
+    assert e.value.code == cb.E_STATE
+    th = eng.tree(tree)
+    eng.prefill(torch.zeros(1, 8, dtype=torch.int32, device="cuda"), [8])
+    tt = torch.zeros(1, 16, dtype=torch.int32, device="cuda")
+    with pytest.raises(cb.CerbError) as e:            # accept without verify
+        eng.accept(th, tt, tt)
+    assert e.value.code == cb.E_STATE
+    bad = synth.Tree(np.array([-1, 0, 1, 0], np.int32), np.array([-1, 0, 1, 7], np.int32), np.zeros(4, np.int32))
+    with pytest.raises(cb.CerbError) as e:            # head index outside the configuration
+        eng.tree(bad)
+    assert e.value.code == cb.E_ARG
+    with pytest.raises(cb.CerbError) as e:            # prompt longer than the page table allows
+        eng.prefill(torch.zeros(1, 4000, dtype=torch.int32, device="cuda"), [4000])
+    assert e.value.code == cb.E_STATE
