@@ -256,6 +256,18 @@ int cerb_read_state(cerb_ctx* ctx, int32_t* len_host, int32_t* root_host, void* 
  * function: CERB_OK, or CERB_E_TIMEOUT.  Synchronises `stream`. */
 int cerb_device_status(cerb_ctx* ctx, void* stream);
 
+/* Per-kernel-family device timing, for measurement only (the paper has no counterpart).  While
+ * enabled, the host controller brackets each family's launches with CUDA events on the caller's
+ * stream; cerb_profile_read synchronises the stream, adds up the elapsed times and launch-group
+ * counts per family since the last read, and clears them.  Families: 0 dense GEMMs, 1 tree
+ * attention, 2 decoding heads + top-k + tree fill, 3 element-wise glue (embedding, norms, RoPE
+ * and KV append, residual, SwiGLU, argmax), 4 gate, 5 acceptance + KV compaction.
+ * ms_out and groups_out are host arrays of CERB_PROF_KINDS entries.  Event recording costs a few
+ * microseconds per bracket, so time whole steps with profiling off. */
+#define CERB_PROF_KINDS 6
+int cerb_profile_enable(cerb_ctx* ctx, int32_t on);
+int cerb_profile_read(cerb_ctx* ctx, double* ms_out, int64_t* groups_out, void* stream);
+
 /* Number of kernel launches issued by this context since load (for accounting). */
 int64_t cerb_launch_count(const cerb_ctx* ctx);
 

@@ -29,7 +29,8 @@ EXPORTS = [
     "cerb_workspace_bytes", "cerb_load", "cerb_free", "cerb_tree_create", "cerb_tree_free", "cerb_reset",
     "cerb_prefill", "cerb_gate", "cerb_draft", "cerb_verify", "cerb_accept", "cerb_step",
     "cerb_attn_scratch_bytes", "cerb_tree_attention", "cerb_tree_ancestors", "cerb_gemm_scratch_bytes", "cerb_gemm",
-    "cerb_read_state", "cerb_device_status", "cerb_launch_count", "cerb_strerror",
+    "cerb_read_state", "cerb_device_status", "cerb_launch_count", "cerb_strerror", "cerb_profile_enable",
+    "cerb_profile_read",
 ]
 
 
@@ -113,6 +114,8 @@ def lib():
                                 C.c_void_p, C.c_size_t, C.c_void_p]
         L.cerb_read_state.argtypes = [C.c_void_p] * 5
         L.cerb_device_status.argtypes = [C.c_void_p, C.c_void_p]
+        L.cerb_profile_enable.argtypes = [C.c_void_p, C.c_int32]
+        L.cerb_profile_read.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -317,6 +320,18 @@ class Cerberus:
 
     def device_status(self) -> int:
         return lib().cerb_device_status(self.ctx, _stream())
+
+    PROF_KINDS = ("gemm", "attention", "heads", "glue", "gate", "accept")
+
+    def profile(self, on: bool):
+        _check(lib().cerb_profile_enable(self.ctx, 1 if on else 0), "cerb_profile_enable")
+
+    def profile_read(self):
+        """{family: (milliseconds, launch groups)} since the last read."""
+        ms = (C.c_double * 6)()
+        gr = (C.c_int64 * 6)()
+        _check(lib().cerb_profile_read(self.ctx, ms, gr, _stream()), "cerb_profile_read")
+        return {k: (ms[i], gr[i]) for i, k in enumerate(self.PROF_KINDS)}
 
     def launch_count(self) -> int:
         return lib().cerb_launch_count(self.ctx)

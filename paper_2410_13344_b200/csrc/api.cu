@@ -25,6 +25,32 @@ struct Bump {
 
 inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
+enum { K_GEMM = 0, K_ATTN = 1, K_HEADS = 2, K_GLUE = 3, K_GATE = 4, K_ACCEPT = 5 };
+constexpr size_t kProfMaxPairs = 1 << 15;
+
+// Brackets a group of launches with two events when profiling is on; free otherwise.
+struct ProfScope {
+  cerb_ctx* c;
+  cudaStream_t st;
+  long idx;
+  ProfScope(cerb_ctx* c_, int kind, cudaStream_t st_) : c(c_), st(st_), idx(-1) {
+    if (!c->prof_on || c->prof_used >= kProfMaxPairs) return;
+    if (c->prof_used * 2 >= c->prof_ev.size()) {
+      cudaEvent_t a, b;
+      if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) return;
+      c->prof_ev.push_back(a);
+      c->prof_ev.push_back(b);
+      c->prof_kind.push_back(kind);
+    }
+    idx = (long)c->prof_used++;
+    c->prof_kind[idx] = kind;
+    cudaEventRecord(c->prof_ev[2 * idx], st);
+  }
+  ~ProfScope() {
+    if (idx >= 0) cudaEventRecord(c->prof_ev[2 * idx + 1], st);
+  }
+};
+
 int validate_config(const cerb_config* g) {
   if (!g) return CERB_E_ARG;
   if (g->dtype != CERB_F32 && g->dtype != CERB_BF16) return CERB_E_ARG;
@@ -193,7 +219,7 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
     if (c->h_len[b] + n > c->max_pos) return CERB_E_STATE;
     if (c->h_len[b] + n > max_len) max_len = c->h_len[b] + n;
   }
-  CERB_TRY(launch_embed(c, tok, tok_stride, tok_off, B, n, st));
+  { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_embed(c, tok, tok_stride, tok_off, B, n, st)); }
   cerb_attn_args a;
   memset(&a, 0, sizeof(a));
   a.dtype = g.dtype; a.B = B; a.n = n; a.n_heads = g.n_heads; a.head_dim = g.head_dim; a.max_pages = g.max_pages;
@@ -202,22 +228,28 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
   a.n_pool_pages = g.n_pool_pages; a.scratch = c->d_attn_scratch; a.scratch_bytes = c->attn_scratch_bytes;
   int ns = 1;
   for (int l = 0; l < g.n_layers; ++l) {
-    CERB_TRY(launch_rmsnorm(c, c->d_x, c->attn_norm[l], c->d_xn, M, st));
-    CERB_TRY(gemm(c, c->d_xn, &c->tm_xn, c->wqkv[l], c->bf16 ? &c->tm_wqkv[l] : nullptr, M, 3 * HD, d, &ns, st));
-    CERB_TRY(launch_rope_append(c, l, tree->dev, c->d_part, ns, (size_t)M * 3 * HD, B, n, st));
+    { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_rmsnorm(c, c->d_x, c->attn_norm[l], c->d_xn, M, st)); }
+    { ProfScope ps(c, K_GEMM, st);
+      CERB_TRY(gemm(c, c->d_xn, &c->tm_xn, c->wqkv[l], c->bf16 ? &c->tm_wqkv[l] : nullptr, M, 3 * HD, d, &ns, st)); }
+    { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_rope_append(c, l, tree->dev, c->d_part, ns, (size_t)M * 3 * HD, B, n, st)); }
     a.k_pool = c->k_pool + (size_t)l * c->pool_layer_bytes;
     a.v_pool = c->v_pool + (size_t)l * c->pool_layer_bytes;
-    CERB_TRY(launch_tree_attention(c, &a, c->bf16 ? &c->tm_kpool[l] : nullptr, c->bf16 ? &c->tm_vpool[l] : nullptr,
-                                   c->sm_count, c->d_status, st));
-    CERB_TRY(gemm(c, c->d_attn, &c->tm_attn, c->wo[l], c->bf16 ? &c->tm_wo[l] : nullptr, M, d, HD, &ns, st));
-    CERB_TRY(launch_residual(c, c->d_x, c->d_part, ns, (size_t)M * d, M, d, st));
-    CERB_TRY(launch_rmsnorm(c, c->d_x, c->mlp_norm[l], c->d_xn, M, st));
-    CERB_TRY(gemm(c, c->d_xn, &c->tm_xn, c->wgu[l], c->bf16 ? &c->tm_wgu[l] : nullptr, M, 2 * F, d, &ns, st));
-    CERB_TRY(launch_swiglu(c, c->d_part, ns, (size_t)M * 2 * F, c->d_act, M, st));
-    CERB_TRY(gemm(c, c->d_act, &c->tm_act, c->wd[l], c->bf16 ? &c->tm_wd[l] : nullptr, M, d, F, &ns, st));
-    CERB_TRY(launch_residual(c, c->d_x, c->d_part, ns, (size_t)M * d, M, d, st));
+    { ProfScope ps(c, K_ATTN, st);
+      CERB_TRY(launch_tree_attention(c, &a, c->bf16 ? &c->tm_kpool[l] : nullptr, c->bf16 ? &c->tm_vpool[l] : nullptr,
+                                     c->sm_count, c->d_status, st)); }
+    { ProfScope ps(c, K_GEMM, st);
+      CERB_TRY(gemm(c, c->d_attn, &c->tm_attn, c->wo[l], c->bf16 ? &c->tm_wo[l] : nullptr, M, d, HD, &ns, st)); }
+    { ProfScope ps(c, K_GLUE, st);
+      CERB_TRY(launch_residual(c, c->d_x, c->d_part, ns, (size_t)M * d, M, d, st));
+      CERB_TRY(launch_rmsnorm(c, c->d_x, c->mlp_norm[l], c->d_xn, M, st)); }
+    { ProfScope ps(c, K_GEMM, st);
+      CERB_TRY(gemm(c, c->d_xn, &c->tm_xn, c->wgu[l], c->bf16 ? &c->tm_wgu[l] : nullptr, M, 2 * F, d, &ns, st)); }
+    { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_swiglu(c, c->d_part, ns, (size_t)M * 2 * F, c->d_act, M, st)); }
+    { ProfScope ps(c, K_GEMM, st);
+      CERB_TRY(gemm(c, c->d_act, &c->tm_act, c->wd[l], c->bf16 ? &c->tm_wd[l] : nullptr, M, d, F, &ns, st)); }
+    { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_residual(c, c->d_x, c->d_part, ns, (size_t)M * d, M, d, st)); }
   }
-  CERB_TRY(launch_rmsnorm(c, c->d_x, c->final_norm, c->d_hidden, M, st));
+  { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_rmsnorm(c, c->d_x, c->final_norm, c->d_hidden, M, st)); }
   return CERB_OK;
 }
 
@@ -225,7 +257,9 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
 int lm_head_argmax(cerb_ctx* c, const void* X, const ActMaps* xm, int rows, int32_t* argmax_out, float* logits_out,
                    cudaStream_t st) {
   int ns = 1;
-  CERB_TRY(gemm(c, X, xm, c->lm_head, c->bf16 ? &c->tm_lm_head : nullptr, rows, c->cfg.vocab, c->cfg.d_model, &ns, st));
+  { ProfScope ps(c, K_GEMM, st);
+    CERB_TRY(gemm(c, X, xm, c->lm_head, c->bf16 ? &c->tm_lm_head : nullptr, rows, c->cfg.vocab, c->cfg.d_model, &ns, st)); }
+  ProfScope ps(c, K_GLUE, st);
   return launch_argmax_rows(c, c->d_part, ns, (size_t)rows * c->cfg.vocab, rows, c->cfg.vocab, argmax_out, logits_out, st);
 }
 
@@ -321,6 +355,8 @@ int cerb_load(const cerb_config* cfg, const cerb_weights* w, void* workspace_dev
   c->B = 0;
   c->verified_tree = nullptr;
   c->launches = 0;
+  c->prof_on = false;
+  c->prof_used = 0;
   memset(c->tree_used, 0, sizeof(c->tree_used));
   memset(c->h_len, 0, sizeof(c->h_len));
   c->chain = c->single = nullptr;
@@ -368,6 +404,7 @@ int cerb_load(const cerb_config* cfg, const cerb_weights* w, void* workspace_dev
 int cerb_free(cerb_ctx* c) {
   if (!c) return CERB_E_ARG;
   if (c->h_stage) cudaFreeHost(c->h_stage);
+  for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
   delete c->chain;
   delete c->single;
   delete c;
@@ -482,7 +519,7 @@ int cerb_step(cerb_ctx* c, const cerb_tree* tree, float T, const int32_t* plant_
   cudaStream_t st = (cudaStream_t)stream;
   const int B = c->B;
   // gate; it also writes each sequence's live node count (1 for an auto-regressive sequence)
-  CERB_TRY(launch_gate(c, T, out->S_dev, out->mode_dev, c->d_nactive, tree->n, st));
+  { ProfScope ps(c, K_GATE, st); CERB_TRY(launch_gate(c, T, out->S_dev, out->mode_dev, c->d_nactive, tree->n, st)); }
   int32_t* hs = c->h_stage;
   CERB_CUDA_OK(cudaMemcpyAsync(hs, out->mode_dev, B * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
   CERB_CUDA_OK(cudaMemcpyAsync(hs + CERB_MAX_BATCH, c->d_len, B * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
@@ -501,13 +538,15 @@ int cerb_step(cerb_ctx* c, const cerb_tree* tree, float T, const int32_t* plant_
   const cerb_tree* used = (any_par && tree->n > 1) ? tree : c->single;
   const int32_t* tok = c->d_root;                       // [B][1]: the root tokens
   if (used != c->single) {
+    ProfScope ps(c, K_HEADS, st);
     CERB_TRY(launch_heads(c, tree, c->d_treetok, plant_tok_dev, nullptr, nullptr, st));
     tok = c->d_treetok;
   }
   const int n = used->n, M = B * n;
   CERB_TRY(forward_rows(c, used, tok, n, 0, n, st));
   CERB_TRY(lm_head_argmax(c, c->d_hidden, &c->tm_hidden, M, c->d_argmax, nullptr, st));
-  CERB_TRY(launch_accept(c, used, tok, c->d_nactive, c->d_argmax, out->n_accept_dev, c->d_path, out->tokens_dev, st));
+  { ProfScope ps(c, K_ACCEPT, st);
+    CERB_TRY(launch_accept(c, used, tok, c->d_nactive, c->d_argmax, out->n_accept_dev, c->d_path, out->tokens_dev, st)); }
   for (int b = 0; b < B; ++b) c->h_len[b] += used->max_depth + 1;
   if (out->n_accept_host)
     CERB_CUDA_OK(cudaMemcpyAsync(out->n_accept_host, out->n_accept_dev, B * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
@@ -604,6 +643,26 @@ int cerb_device_status(cerb_ctx* c, void* stream) {
   CERB_CUDA_OK(cudaMemcpy(&s, c->d_status, sizeof(s), cudaMemcpyDeviceToHost));
   if (s != 0) CERB_CUDA_OK(cudaMemset(c->d_status, 0, sizeof(s)));
   return s;
+}
+
+int cerb_profile_enable(cerb_ctx* c, int32_t on) {
+  if (!c) return CERB_E_ARG;
+  c->prof_on = on != 0;
+  return CERB_OK;
+}
+
+int cerb_profile_read(cerb_ctx* c, double* ms_out, int64_t* groups_out, void* stream) {
+  if (!c || !ms_out || !groups_out) return CERB_E_ARG;
+  CERB_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
+  for (int k = 0; k < CERB_PROF_KINDS; ++k) { ms_out[k] = 0.0; groups_out[k] = 0; }
+  for (size_t i = 0; i < c->prof_used; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->prof_ev[2 * i], c->prof_ev[2 * i + 1]) != cudaSuccess) continue;
+    ms_out[c->prof_kind[i]] += ms;
+    groups_out[c->prof_kind[i]] += 1;
+  }
+  c->prof_used = 0;
+  return CERB_OK;
 }
 
 int64_t cerb_launch_count(const cerb_ctx* c) { return c ? c->launches : -1; }

@@ -100,7 +100,7 @@ struct AttnParams {
   const uint64_t* anc;
   bf16* out;
   float* lse;
-  float* partial;           // [B*H][nsplit][NQ][DH+2]
+  float* partial;           // [B*H][nsplit][NQ][DH+4]
   unsigned int* counters;   // [B*H]
   int32_t* status;
   int n, H, max_pages, nsplit, oob_row;
@@ -119,7 +119,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
   constexpr uint32_t HALF_BYTES = TILE * 128;
   constexpr uint32_t KV_BYTES = HALVES * HALF_BYTES;      // one of K or V for a stage
   constexpr uint32_t STAGE_BYTES = 2 * KV_BYTES;
-  constexpr int ROWF = DH + 2;                            // merge row: O[DH], m, l
+  constexpr int ROWF = DH + 4;                            // merge row: O[DH], m, l, pad (16-byte rows)
   static_assert(NQ * ROWF * 4 <= STAGES * STAGE_BYTES, "merge buffer must fit in the stage ring");
 
   extern __shared__ uint8_t smem_raw[];
@@ -374,19 +374,36 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
       compute_bar(NW * 32);
       if (ticket_s == (unsigned)p.nsplit - 1) {
         __threadfence();
-        for (int idx = ct; idx < nq * DH; idx += nct) {
-          int r = idx / DH, c = idx % DH;
+        // per-row merge weights first (one thread per row), then a wide, vectorised weighted sum
+        float* wts = mrg;                                   // [nsplit][NQ], the merge buffer is free again
+        for (int r = ct; r < nq; r += nct) {
           float M = -INFINITY;
           for (int s2 = 0; s2 < p.nsplit; ++s2) M = fmaxf(M, __ldcg(part + (size_t)s2 * (NQ * ROWF) + r * ROWF + DH));
-          float Lsum = 0.f, acc = 0.f;
+          float Lsum = 0.f;
           for (int s2 = 0; s2 < p.nsplit; ++s2) {
             const float* pr = part + (size_t)s2 * (NQ * ROWF) + r * ROWF;
             float w = exp2f(__ldcg(pr + DH) - M);
+            wts[s2 * NQ + r] = w;
             Lsum += __ldcg(pr + DH + 1) * w;
-            acc += __ldcg(pr + c) * w;
           }
-          p.out[(((size_t)b * p.n + r) * p.H + h) * DH + c] = __float2bfloat16_rn(acc / Lsum);
-          if (c == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
+          float inv = 1.0f / Lsum;
+          for (int s2 = 0; s2 < p.nsplit; ++s2) wts[s2 * NQ + r] *= inv;
+          if (p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
+        }
+        compute_bar(NW * 32);
+        constexpr int C4 = DH / 4;
+        for (int idx = ct; idx < nq * C4; idx += nct) {
+          const int r = idx / C4, c4 = idx % C4;
+          const float4* src = reinterpret_cast<const float4*>(part + (size_t)r * ROWF) + c4;
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+          for (int s2 = 0; s2 < p.nsplit; ++s2) {
+            float4 v = __ldcg(src + (size_t)s2 * (NQ * ROWF / 4));
+            float w = wts[s2 * NQ + r];
+            acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+          }
+          uint2 packed = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+          *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.n + r) * p.H + h) * DH + c4 * 4) = packed;
         }
         if (ct == 0) p.counters[b * p.H + h] = 0u;       // ready for the next launch
       }
@@ -448,10 +465,14 @@ __global__ void __launch_bounds__(128) tree_attn_f32_kernel(const float* __restr
   if (threadIdx.x == 0 && lse) lse[((size_t)b * H + h) * n + i] = M + logf(Ls);
 }
 
-int plan_nsplit(int B, int H, int max_len) {
+// A split reads `per` tiles of 64 keys and writes an n-row fp32 partial, so wide trees get fewer,
+// longer splits: at least n/8 tiles each keeps the partial traffic near one eighth of the K/V read.
+int plan_nsplit(int B, int H, int n, int max_len) {
   int tiles = (max_len + TILE - 1) / TILE;
   if (tiles < 1) tiles = 1;
   int want = (kTargetCtas + B * H - 1) / (B * H);
+  int min_tiles = n / 8 > 1 ? n / 8 : 1;
+  if (want > tiles / min_tiles) want = tiles / min_tiles;
   if (want > kMaxSplit) want = kMaxSplit;
   if (want > tiles) want = tiles;
   if (want < 1) want = 1;
@@ -480,7 +501,7 @@ int launch_cfg(const AttnParams& p, const CUtensorMap* tmK, const CUtensorMap* t
 
 size_t attn_scratch_bytes(int B, int n, int H, int Dh) {
   size_t rows = (size_t)(kTargetCtas + B * H + kMaxSplit);
-  return kCounterBytes + rows * (size_t)nq_pad(n) * (size_t)(Dh + 2) * sizeof(float);
+  return kCounterBytes + rows * (size_t)nq_pad(n) * (size_t)(Dh + 4) * sizeof(float);
 }
 
 int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMap* tmK, const CUtensorMap* tmV,
@@ -516,7 +537,7 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
   p.n = a->n;
   p.H = a->n_heads;
   p.max_pages = a->max_pages;
-  p.nsplit = plan_nsplit(a->B, a->n_heads, a->max_len);
+  p.nsplit = plan_nsplit(a->B, a->n_heads, nq_pad(a->n), a->max_len);
   if (p.nsplit < 1) return CERB_E_SHAPE;
   p.oob_row = a->n_pool_pages * a->n_heads * CERB_PAGE;
   p.scale_log2 = a->scale * 1.4426950408889634f;

@@ -109,6 +109,12 @@ struct cerb_ctx {
   const cerb_tree* verified_tree;     // tree of the last cerb_verify not yet accepted
   int64_t launches;
   int sm_count;
+
+  // optional per-family timing (cerb_profile_*)
+  bool prof_on;
+  std::vector<cudaEvent_t> prof_ev;   // begin/end pairs
+  std::vector<int> prof_kind;         // family of each pair
+  size_t prof_used;                   // pairs recorded since the last read
 };
 
 namespace cerb {

@@ -42,10 +42,11 @@ def oracle_planter(tree: synth.Tree, truth, lengths):
     return plant
 
 
-def close(a: torch.Tensor, b: torch.Tensor, tol: float) -> float:
-    """max |a-b| / max(1, |b|): the 'max-abs/rel' error; returns it."""
+def close(a: torch.Tensor, b: torch.Tensor, tol: float = 0.0) -> float:
+    """Combined absolute/relative error max |a-b| / (1 + |b|); "within tol" means
+    |a-b| <= tol + tol*|b| for every element (atol = rtol = tol)."""
     a, b = a.double().cpu(), b.double().cpu()
-    return float(((a - b).abs() / b.abs().clamp(min=1.0)).max())
+    return float(((a - b).abs() / (1.0 + b.abs())).max())
 
 
 def top2_margin(logits_row: torch.Tensor) -> float:
