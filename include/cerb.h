@@ -236,6 +236,23 @@ typedef struct cerb_attn_args {
 int cerb_attn_scratch_bytes(int32_t B, int32_t n, int32_t n_heads, int32_t head_dim, size_t* bytes_out);
 int cerb_tree_attention(const cerb_attn_args* args, void* stream);
 
+/* cerb_tree_attention for callers that cannot allocate device memory (the paper has no
+ * counterpart; this is a packaging variant of the same kernel).  Typical cases: code running
+ * inside an allocator or memory-pool callback, a plug-in that only receives fixed buffers from its
+ * host application, a process whose device-memory budget is fixed at start-up.  The split-KV
+ * scratch that the caller would otherwise provide lives in a static device array inside the
+ * library, CERB_STATIC_ATTN_SCRATCH_BYTES large; every GPU that loads the library holds it until
+ * the process exits.  args->scratch and args->scratch_bytes are ignored; inputs and outputs are
+ * still the caller's.  bf16 only.  Returns CERB_E_NOMEM when cerb_attn_scratch_bytes() for the
+ * problem exceeds the static array (roughly: B * n_heads beyond a few hundred with 128-node trees).
+ * This call never allocates or frees device memory.
+ * The first call on each device looks up the array's device address (one runtime query); make that
+ * first call outside any stream capture.  All calls share the one array and each call clears the
+ * part that must start at zero on `stream`, so two calls that may overlap on the GPU (different
+ * streams, no dependency) race with each other: serialise them. */
+#define CERB_STATIC_ATTN_SCRATCH_BYTES (16u << 20)
+int cerb_tree_attention_noalloc(const cerb_attn_args* args, void* stream);
+
 /* Ancestor bitmasks of a tree, the form cerb_tree_attention takes: anc_out host [n][2]. */
 int cerb_tree_ancestors(const int32_t* parent, int32_t n, uint64_t* anc_out);
 

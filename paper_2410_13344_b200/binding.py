@@ -30,7 +30,7 @@ EXPORTS = [
     "cerb_prefill", "cerb_gate", "cerb_draft", "cerb_verify", "cerb_accept", "cerb_step",
     "cerb_attn_scratch_bytes", "cerb_tree_attention", "cerb_tree_ancestors", "cerb_gemm_scratch_bytes", "cerb_gemm",
     "cerb_read_state", "cerb_device_status", "cerb_launch_count", "cerb_strerror", "cerb_profile_enable",
-    "cerb_profile_read",
+    "cerb_profile_read", "cerb_tree_attention_noalloc",
 ]
 
 
@@ -109,6 +109,7 @@ def lib():
         L.cerb_attn_scratch_bytes.argtypes = [C.c_int32] * 4 + [C.POINTER(C.c_size_t)]
         L.cerb_tree_attention.argtypes = [C.POINTER(AttnArgs), C.c_void_p]
         L.cerb_tree_ancestors.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
+        L.cerb_tree_attention_noalloc.argtypes = [C.POINTER(AttnArgs), C.c_void_p]
         L.cerb_gemm_scratch_bytes.argtypes = [C.c_int32] * 3 + [C.POINTER(C.c_size_t)]
         L.cerb_gemm.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                 C.c_void_p, C.c_size_t, C.c_void_p]
@@ -362,6 +363,22 @@ def tree_attention(q: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor, 
                  scale, max_len, k_pool.shape[0], scratch.data_ptr(), scratch.numel())
     _check(lib().cerb_tree_attention(C.byref(a), _stream()), "cerb_tree_attention")
     return out, lse, scratch
+
+
+STATIC_ATTN_SCRATCH_BYTES = 16 << 20
+
+
+def tree_attention_noalloc(q: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor, page_table: torch.Tensor,
+                           lens: torch.Tensor, anc: torch.Tensor, scale: float, max_len: int, out: torch.Tensor,
+                           lse: Optional[torch.Tensor] = None, n_active: Optional[torch.Tensor] = None) -> int:
+    """Same operation as tree_attention for callers that must not allocate device memory: the split-KV
+    scratch is a static array inside the library and `out` / `lse` are passed in, so neither this
+    wrapper nor the library allocates anything.  Returns the library's status code."""
+    B, n, H, Dh = q.shape
+    a = AttnArgs(BF16, B, n, H, Dh, page_table.shape[1], q.data_ptr(), k_pool.data_ptr(), v_pool.data_ptr(),
+                 page_table.data_ptr(), lens.data_ptr(), _ptr(n_active), anc.data_ptr(), out.data_ptr(), _ptr(lse),
+                 scale, max_len, k_pool.shape[0], None, 0)
+    return lib().cerb_tree_attention_noalloc(C.byref(a), _stream())
 
 
 def gemm(X: torch.Tensor, W: torch.Tensor, scratch: Optional[torch.Tensor] = None) -> torch.Tensor:

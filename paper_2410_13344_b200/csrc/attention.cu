@@ -560,3 +560,52 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
 }
 
 }  // namespace cerb
+
+// ---------------------------------------------------------------------------------------------
+// Tree attention for callers that cannot allocate device memory
+// ---------------------------------------------------------------------------------------------
+// The split-KV partials and ticket counters normally live in a scratch buffer the caller allocates.
+// Some callers cannot do that: code running inside a memory-pool or allocator callback, a plug-in
+// that is handed fixed buffers by its host application, or a process whose device-memory budget was
+// fixed at start-up.  For them the scratch lives in this library's image instead, as one static
+// device array.  Every GPU that loads the library holds these bytes until the process exits.
+static __device__ __align__(256) unsigned char g_static_attn_scratch[CERB_STATIC_ATTN_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices];      // device address of the array, per device, once known
+}  // namespace
+
+extern "C" int cerb_tree_attention_noalloc(const cerb_attn_args* a, void* stream) {
+  using namespace cerb;
+  if (!a || !a->q || !a->k_pool || !a->v_pool || !a->page_table || !a->len || !a->anc || !a->out) return CERB_E_ARG;
+  if (a->B < 1 || a->n < 1 || a->n > CERB_MAX_NODES || a->n_heads < 1 || a->n_pool_pages < 1) return CERB_E_ARG;
+  if (a->dtype != CERB_BF16) return CERB_E_ARG;
+  if (a->head_dim != 64 && a->head_dim != 128) return CERB_E_SHAPE;
+  const size_t need = attn_scratch_bytes(a->B, a->n, a->n_heads, a->head_dim);
+  if (need > (size_t)CERB_STATIC_ATTN_SCRATCH_BYTES) return CERB_E_NOMEM;     // problem too large for the built-in scratch
+  int dev = -1;
+  CERB_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return CERB_E_SHAPE;
+  if (!g_static_scratch_addr[dev]) {
+    // In host code the array's name is only a handle; the address a kernel can use has to be asked
+    // for, once per device, while that device is current.
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_attn_scratch) != cudaSuccess || !ptr) return CERB_E_CUDA;
+    g_static_scratch_addr[dev] = ptr;
+  }
+  void* scratch = g_static_scratch_addr[dev];
+  cudaStream_t st = (cudaStream_t)stream;
+  // The array keeps whatever the previous call left: the ticket counters and the status word (the
+  // first 4 KB) must start at zero.  The partials behind them are fully rewritten before being read.
+  CERB_CUDA_OK(cudaMemsetAsync(scratch, 0, kCounterBytes, st));
+  CUtensorMap tk, tv;
+  CERB_TRY(make_pool_map(&tk, a->k_pool, a->n_pool_pages, a->n_heads, a->head_dim));
+  CERB_TRY(make_pool_map(&tv, a->v_pool, a->n_pool_pages, a->n_heads, a->head_dim));
+  cerb_attn_args b = *a;
+  b.scratch = scratch;
+  b.scratch_bytes = CERB_STATIC_ATTN_SCRATCH_BYTES;
+  int32_t* status = reinterpret_cast<int32_t*>((char*)scratch + kCounterBytes - 16);
+  return launch_tree_attention(nullptr, &b, &tk, &tv, 148, status, st);
+}
+
