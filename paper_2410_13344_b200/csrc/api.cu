@@ -1,6 +1,7 @@
 // C ABI of the Cerberus decoding-step library: context set-up, workspace carve-out and the host
 // controller that strings the kernels together (Algorithm 1).
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -8,6 +9,17 @@
 #include "cerb_internal.cuh"
 
 using namespace cerb;
+
+namespace cerb {
+bool pdl_enabled() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("CERB_PDL");
+    v = e ? (atoi(e) != 0) : 1;
+  }
+  return v != 0;
+}
+}  // namespace cerb
 
 namespace {
 
@@ -219,7 +231,9 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
     if (c->h_len[b] + n > c->max_pos) return CERB_E_STATE;
     if (c->h_len[b] + n > max_len) max_len = c->h_len[b] + n;
   }
-  { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_embed(c, tok, tok_stride, tok_off, B, n, st)); }
+  // embedding gather fused with the first layer's attention norm
+  { ProfScope ps(c, K_GLUE, st);
+    CERB_TRY(launch_fused_norm(c, nullptr, 0, 0, tok, tok_stride, tok_off, n, c->attn_norm[0], c->d_xn, M, st)); }
   cerb_attn_args a;
   memset(&a, 0, sizeof(a));
   a.dtype = g.dtype; a.B = B; a.n = n; a.n_heads = g.n_heads; a.head_dim = g.head_dim; a.max_pages = g.max_pages;
@@ -228,7 +242,6 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
   a.n_pool_pages = g.n_pool_pages; a.scratch = c->d_attn_scratch; a.scratch_bytes = c->attn_scratch_bytes;
   int ns = 1;
   for (int l = 0; l < g.n_layers; ++l) {
-    { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_rmsnorm(c, c->d_x, c->attn_norm[l], c->d_xn, M, st)); }
     { ProfScope ps(c, K_GEMM, st);
       CERB_TRY(gemm(c, c->d_xn, &c->tm_xn, c->wqkv[l], c->bf16 ? &c->tm_wqkv[l] : nullptr, M, 3 * HD, d, &ns, st)); }
     { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_rope_append(c, l, tree->dev, c->d_part, ns, (size_t)M * 3 * HD, B, n, st)); }
@@ -239,17 +252,20 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
                                      c->sm_count, c->d_status, st)); }
     { ProfScope ps(c, K_GEMM, st);
       CERB_TRY(gemm(c, c->d_attn, &c->tm_attn, c->wo[l], c->bf16 ? &c->tm_wo[l] : nullptr, M, d, HD, &ns, st)); }
+    // residual add fused with the MLP norm
     { ProfScope ps(c, K_GLUE, st);
-      CERB_TRY(launch_residual(c, c->d_x, c->d_part, ns, (size_t)M * d, M, d, st));
-      CERB_TRY(launch_rmsnorm(c, c->d_x, c->mlp_norm[l], c->d_xn, M, st)); }
+      CERB_TRY(launch_fused_norm(c, c->d_part, ns, (size_t)M * d, nullptr, 0, 0, n, c->mlp_norm[l], c->d_xn, M, st)); }
     { ProfScope ps(c, K_GEMM, st);
       CERB_TRY(gemm(c, c->d_xn, &c->tm_xn, c->wgu[l], c->bf16 ? &c->tm_wgu[l] : nullptr, M, 2 * F, d, &ns, st)); }
     { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_swiglu(c, c->d_part, ns, (size_t)M * 2 * F, c->d_act, M, st)); }
     { ProfScope ps(c, K_GEMM, st);
       CERB_TRY(gemm(c, c->d_act, &c->tm_act, c->wd[l], c->bf16 ? &c->tm_wd[l] : nullptr, M, d, F, &ns, st)); }
-    { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_residual(c, c->d_x, c->d_part, ns, (size_t)M * d, M, d, st)); }
+    // residual add fused with the next layer's attention norm, or with the final norm
+    { ProfScope ps(c, K_GLUE, st);
+      const bool last = l + 1 == g.n_layers;
+      CERB_TRY(launch_fused_norm(c, c->d_part, ns, (size_t)M * d, nullptr, 0, 0, n, last ? c->final_norm : c->attn_norm[l + 1],
+                                 last ? c->d_hidden : c->d_xn, M, st)); }
   }
-  { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_rmsnorm(c, c->d_x, c->final_norm, c->d_hidden, M, st)); }
   return CERB_OK;
 }
 
@@ -587,6 +603,7 @@ int cerb_gemm_scratch_bytes(int32_t M, int32_t N, int32_t K, size_t* bytes_out) 
 // Sums split partials into the output (used only by the stand-alone GEMM entry point).
 __global__ void sum_splits_kernel(const float* __restrict__ part, int nsplit, size_t stride, float* __restrict__ out,
                                   size_t total) {
+  griddep_wait();
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total) return;
   float a = 0.f;

@@ -132,6 +132,8 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  griddep_wait();
+  griddep_launch();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int L = p.len[b];
@@ -426,6 +428,8 @@ __global__ void __launch_bounds__(128) tree_attn_f32_kernel(const float* __restr
   constexpr int E = DH / 32;
   __shared__ float s_o[4][DH];
   __shared__ float s_m[4], s_l[4];
+  griddep_wait();
+  griddep_launch();
   const int i = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int nq = n_active ? min(n_active[b], n) : n;
   if (i >= nq) return;
@@ -493,7 +497,8 @@ int launch_cfg(const AttnParams& p, const CUtensorMap* tmK, const CUtensorMap* t
     configured = true;
   }
   dim3 grid(p.nsplit, p.H, B);
-  tree_attn_bf16_kernel<DH, WQ, WK, STAGES><<<grid, (WQ * WK + 1) * 32, smem, st>>>(*tmK, *tmV, p);
+  if (launch_pdl(tree_attn_bf16_kernel<DH, WQ, WK, STAGES>, grid, dim3((WQ * WK + 1) * 32), smem, st, *tmK, *tmV, p) != cudaSuccess)
+    return CERB_E_CUDA;
   return CERB_OK;
 }
 

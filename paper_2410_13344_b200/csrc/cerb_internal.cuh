@@ -32,6 +32,31 @@ namespace cerb {
 
 typedef __nv_bfloat16 bf16;
 
+// Programmatic dependent launch: a kernel launched through launch_pdl may begin while its
+// predecessor in the stream is still running; it must execute griddep_wait() before it touches
+// anything the predecessor writes (or anything the predecessor may still be reading and this
+// kernel overwrites).  griddep_launch() lets the next kernel in the stream be scheduled early.
+#ifdef __CUDACC__
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+bool pdl_enabled();
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 constexpr int kPathMax = CERB_MAX_DEPTH + 1;
 constexpr int kGemmRowsPerPass = 256;   // activation rows one tcgen05 pass covers (the MMA's N extent)
 constexpr int kGemmMaxSplit = 16;
@@ -130,12 +155,10 @@ inline int bucket_rows(int b) { return 16 << b; }
 
 // glue.cu
 int launch_rope_table(cerb_ctx* c, cudaStream_t st);
-int launch_embed(cerb_ctx* c, const int32_t* tok, int tok_stride, int tok_off, int B, int n, cudaStream_t st);
-int launch_rmsnorm(cerb_ctx* c, const void* x, const void* gain, void* out, int rows, cudaStream_t st);
+int launch_fused_norm(cerb_ctx* c, const float* part, int nsplit, size_t split_stride, const int32_t* tok, int tok_stride,
+                      int tok_off, int n, const void* gain, void* out, int rows, cudaStream_t st);
 int launch_rope_append(cerb_ctx* c, int layer, const TreeDev& t, const float* part, int nsplit, size_t split_stride,
                        int B, int n, cudaStream_t st);
-int launch_residual(cerb_ctx* c, void* x, const float* part, int nsplit, size_t split_stride, int rows, int N,
-                    cudaStream_t st);
 int launch_swiglu(cerb_ctx* c, const float* part, int nsplit, size_t split_stride, void* act, int rows, cudaStream_t st);
 int launch_argmax_rows(cerb_ctx* c, const float* part, int nsplit, size_t split_stride, int rows, int V, int32_t* out,
                        float* summed, cudaStream_t st);

@@ -30,6 +30,8 @@ template <typename T>
 __global__ void __launch_bounds__(256) gate_kernel(const T* __restrict__ h_last, int d, float thr, float* __restrict__ S,
                                                    int32_t* __restrict__ mode, int32_t* __restrict__ n_active, int n_par) {
   __shared__ float red[32];
+  griddep_wait();
+  griddep_launch();
   const T* h = h_last + (size_t)blockIdx.x * d;
   float m = -INFINITY;
   for (int j = threadIdx.x; j < d; j += blockDim.x) m = fmaxf(m, ldf(h + j));
@@ -67,6 +69,8 @@ __global__ void __launch_bounds__(128) accept_kernel(const int32_t* __restrict__
   __shared__ uint32_t mword[4];
   __shared__ int skey[4];
   __shared__ int best_s;
+  griddep_wait();
+  griddep_launch();
   const int b = blockIdx.x, v = threadIdx.x;
   const int na = min(n_active[b], n);
   const int32_t* tk = tok + (size_t)b * n;
@@ -119,6 +123,8 @@ __global__ void kv_compact_kernel(char* __restrict__ kpool, char* __restrict__ v
                                   const int32_t* __restrict__ page_table, int max_pages,
                                   const int32_t* __restrict__ len_old, const int32_t* __restrict__ n_accept,
                                   const int32_t* __restrict__ path, int H, int row_bytes) {
+  griddep_wait();
+  griddep_launch();
   const int b = blockIdx.z, layer = blockIdx.y >> 1;
   char* pool = ((blockIdx.y & 1) ? vpool : kpool) + (size_t)layer * layer_bytes;
   const int chunks = row_bytes / 16;

@@ -1,18 +1,34 @@
 // bf16 GEMM of the verification forward on the 5th-generation tensor cores (tcgen05 + TMEM).
 //
-//   out[split][m][n] = sum over this split's k of X[m][k] * W[n][k]        (fp32)
+//   out[slot][m][n] = partial sum over some k range of X[m][k] * W[n][k]        (fp32)
 //
 // A decoding step has few activation rows (tree nodes x batch) and large weight matrices, so the
-// kernel is organised around streaming W exactly once at HBM speed ("swap-AB"): a CTA takes a
-// 128-row tile of W as the MMA's A operand (M = 128) and up to 256 activation rows as the B
-// operand (N = rows), accumulates D[128][rows] in tensor memory and writes it transposed.
-// Where W has too few 128-row tiles to occupy the GPU the K dimension is split across CTAs and
-// each split writes its own fp32 partial; consumers add the partials in index order.
+// kernel is organised around streaming W exactly once at HBM speed ("swap-AB"): a 128-row tile of
+// W is the MMA's A operand (M = 128), up to 256 activation rows are the B operand (N = rows), and
+// D[128][rows] accumulates in tensor memory and is written out transposed.
 //
-// Roles inside a CTA (192 threads): warp 0 = TMA producer (one lane), warp 1 = TMEM allocator and
-// MMA issuer (one lane), warps 2-5 = epilogue (each owns the 32 TMEM lanes of its warp quarter).
-// Stages are handed over with mbarriers; every wait is bounded and reports CERB_E_TIMEOUT through
-// a status word instead of hanging.
+// With at most 128 activation rows a CTA takes 256 weight rows at a time (two MMA tiles that share
+// one activation stage), which halves the activation re-reads through L2; weight tiles carry an
+// evict-first L2 hint, activation tiles evict-last.
+//
+// The kernel is launched programmatically dependent on its predecessor: weights do not depend on
+// the previous kernel, so the producer fills the whole stage ring with weight tiles before it
+// waits for that kernel; only the activation loads and the output stores come after the wait.
+//
+// Schedule: persistent, one CTA per SM, stream-K.  The work is the list of (weight tile, 64-wide
+// k block) units; every CTA takes an equal, contiguous share of it, so all SMs stream for the same
+// time whatever the matrix shape (no partial last wave).  A share may cross tile boundaries: each
+// run of units inside one tile is a "segment" that accumulates in TMEM and is written to its own
+// fp32 partial slot; consumers add a tile's slots in index order (deterministic).  The CTA that
+// owns a tile's last segment zero-fills the slots that tile does not use.
+//
+// Roles inside a CTA (192 threads): warp 0 = TMA producer (one lane) running ahead through the
+// whole share, warp 1 = TMEM allocator and MMA issuer (one lane), warps 2-5 = epilogue (each owns
+// the 32 TMEM lanes of its warp quarter).  The accumulator is double-buffered in TMEM so a segment's
+// epilogue overlaps the next segment's MMAs.  Stages and accumulators are handed over with
+// mbarriers; every wait is bounded and reports CERB_E_TIMEOUT through a status word.
+#include <stdlib.h>
+
 #include "cerb_internal.cuh"
 
 namespace cerb {
@@ -33,6 +49,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -44,8 +63,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  After the first time-out in a CTA every later wait gives up quickly, so the CTA
-// still runs to its end (releasing tensor memory) in bounded time.
 __device__ __forceinline__ uint64_t global_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -67,6 +84,18 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
   atomicExch(status, CERB_E_TIMEOUT);
 }
 
+__device__ __forceinline__ uint64_t l2_policy(bool evict_first) {
+  uint64_t pol;
+  if (evict_first) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  else asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"((uint64_t)map), "r"(x), "r"(y), "r"(bar), "l"(pol)
+      : "memory");
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -116,42 +145,68 @@ struct GemmParams {
   int M, N, K;
   int n_mma;          // activation rows per pass (16..256, power of two)
   int num_kb;         // ceil(K / 64)
-  int kb_per_split;
+  int tiles;          // ceil(N / 128)
+  int per;            // work units per CTA
+  long long total;    // work units in all: mchunks * tiles * num_kb
+  int nslots;         // partial slots per output element
   int stages;
+  int wide;           // 1: a CTA works on 256 weight rows at a time (two MMA tiles sharing one activation stage)
+  int group;          // stages are released to the producer in groups of this many (1 or 2)
+  int hint;           // 1: weights evict-first, activations evict-last in L2
   uint32_t idesc;
-  uint32_t tmem_cols;
+  uint32_t acc_cols;  // TMEM columns of one accumulator buffer
 };
 
-__global__ void __launch_bounds__(192) gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmW,
-                                                        const __grid_constant__ CUtensorMap tmX, const GemmParams p) {
+// One run of k blocks inside one (row chunk, weight tile) job.
+struct Segment {
+  int job, kb0, nkb;
+};
+__device__ __forceinline__ bool next_segment(long long& u, long long u1, int num_kb, Segment& sg) {
+  if (u >= u1) return false;
+  sg.job = (int)(u / num_kb);
+  sg.kb0 = (int)(u % num_kb);
+  long long end = (long long)(sg.job + 1) * num_kb;
+  if (end > u1) end = u1;
+  sg.nkb = (int)(end - u);
+  u = end;
+  return true;
+}
+
+__global__ void __launch_bounds__(192, 1) gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmW,
+                                                           const __grid_constant__ CUtensorMap tmX, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
   __shared__ __align__(8) uint64_t empty_bar[MAX_STAGES];
-  __shared__ __align__(8) uint64_t accum_bar;
+  __shared__ __align__(8) uint64_t acc_full[2];
+  __shared__ __align__(8) uint64_t acc_empty[2];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int aborted_s;
   volatile int* aborted = &aborted_s;
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t b_bytes = (uint32_t)p.n_mma * BK * 2;
-  const uint32_t stage_bytes = A_STAGE_BYTES + b_bytes;
+  const uint32_t a_bytes = A_STAGE_BYTES * (uint32_t)(1 + p.wide);
+  const uint32_t stage_bytes = a_bytes + b_bytes;
+  const int rows_per_tile = BM * (1 + p.wide);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile = blockIdx.x, split = blockIdx.y, mchunk = blockIdx.z;
-  const int kb0 = split * p.kb_per_split;
-  const int kb1 = min(p.num_kb, kb0 + p.kb_per_split);
+  const long long u0 = (long long)blockIdx.x * p.per;
+  const long long u1 = (u0 + p.per < p.total) ? u0 + p.per : p.total;
 
   if (threadIdx.x == 0) {
-    aborted_s = (*p.status != 0);
+    aborted_s = 0;
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(smem_u32(&full_bar[s]), 1);
       mbar_init(smem_u32(&empty_bar[s]), 1);
     }
-    mbar_init(smem_u32(&accum_bar), 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&acc_full[i]), 1);
+      mbar_init(smem_u32(&acc_empty[i]), 4);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
-                 "r"(p.tmem_cols)
+                 "r"(2u * p.acc_cols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -160,62 +215,180 @@ __global__ void __launch_bounds__(192) gemm_bf16_kernel(const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
 
+  griddep_launch();
   if (warp == 0) {
     if (lane == 0) {
-      for (int kb = kb0, i = 0; kb < kb1; ++kb, ++i) {
-        int s = i % p.stages;
-        uint32_t ph = (uint32_t)(i / p.stages) & 1u;
-        mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, aborted, p.status);
-        uint32_t fb = smem_u32(&full_bar[s]);
+      const int n_units = (int)(u1 - u0);
+      const uint64_t pol_w = l2_policy(true), pol_x = l2_policy(false);
+      auto load_w = [&](int i) {
+        const long long u = u0 + i;
+        const int job = (int)(u / p.num_kb), kb = (int)(u % p.num_kb), tile = job % p.tiles;
+        const int s = i % p.stages;
+        const uint32_t fb = smem_u32(&full_bar[s]);
+        const uint32_t a_dst = smem_base + (uint32_t)s * stage_bytes;
         mbar_expect_tx(fb, stage_bytes);
-        uint32_t a_dst = smem_base + (uint32_t)s * stage_bytes;
-        tma_load_2d(a_dst, &tmW, kb * BK, tile * BM, fb);
-        tma_load_2d(a_dst + A_STAGE_BYTES, &tmX, kb * BK, mchunk * kGemmRowsPerPass, fb);
+        if (p.hint) {
+          tma_load_2d_hint(a_dst, &tmW, kb * BK, tile * rows_per_tile, fb, pol_w);
+          if (p.wide) tma_load_2d_hint(a_dst + A_STAGE_BYTES, &tmW, kb * BK, tile * rows_per_tile + BM, fb, pol_w);
+        } else {
+          tma_load_2d(a_dst, &tmW, kb * BK, tile * rows_per_tile, fb);
+          if (p.wide) tma_load_2d(a_dst + A_STAGE_BYTES, &tmW, kb * BK, tile * rows_per_tile + BM, fb);
+        }
+      };
+      auto load_x = [&](int i) {
+        const long long u = u0 + i;
+        const int job = (int)(u / p.num_kb), kb = (int)(u % p.num_kb), mchunk = job / p.tiles;
+        const int s = i % p.stages;
+        const uint32_t fb = smem_u32(&full_bar[s]);
+        const uint32_t x_dst = smem_base + (uint32_t)s * stage_bytes + a_bytes;
+        if (p.hint) tma_load_2d_hint(x_dst, &tmX, kb * BK, mchunk * kGemmRowsPerPass, fb, pol_x);
+        else tma_load_2d(x_dst, &tmX, kb * BK, mchunk * kGemmRowsPerPass, fb);
+      };
+      // Weights do not depend on the kernel before this one: fill the whole ring with weight tiles
+      // while that kernel is still finishing, then wait for it and fetch the activations.
+      const int pre = n_units < p.stages ? n_units : p.stages;
+      for (int i = 0; i < pre; ++i) load_w(i);
+      griddep_wait();
+      for (int i = 0; i < pre; ++i) load_x(i);
+      for (int i = pre; i < n_units; ++i) {
+        const int s = i % p.stages;
+        const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
+        mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, aborted, p.status);
+        load_w(i);
+        load_x(i);
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      for (int kb = kb0, i = 0; kb < kb1; ++kb, ++i) {
-        int s = i % p.stages;
-        uint32_t ph = (uint32_t)(i / p.stages) & 1u;
-        mbar_wait(smem_u32(&full_bar[s]), ph, aborted, p.status);
+      long long u = u0;
+      Segment sg;
+      int i = 0, g = 0;
+      while (next_segment(u, u1, p.num_kb, sg)) {
+        const int buf = g & 1;
+        mbar_wait(smem_u32(&acc_empty[buf]), ((uint32_t)(g >> 1) & 1u) ^ 1u, aborted, p.status);
         tc_fence_after();
-        uint32_t a_src = smem_base + (uint32_t)s * stage_bytes;
-        uint64_t adesc = umma_desc_sw128(a_src);
-        uint64_t bdesc = umma_desc_sw128(a_src + A_STAGE_BYTES);
+        const uint32_t tmem_d = tmem_base + (uint32_t)buf * p.acc_cols;
+        int held = -1;                                // stage whose release is deferred to pair it with the next
+        for (int k = 0; k < sg.nkb; ++k, ++i) {
+          int s = i % p.stages;
+          uint32_t ph = (uint32_t)(i / p.stages) & 1u;
+          mbar_wait(smem_u32(&full_bar[s]), ph, aborted, p.status);
+          tc_fence_after();
+          uint32_t a_src = smem_base + (uint32_t)s * stage_bytes;
+          uint64_t adesc = umma_desc_sw128(a_src);
+          uint64_t bdesc = umma_desc_sw128(a_src + a_bytes);
 #pragma unroll
-        for (int kk = 0; kk < BK / 16; ++kk) {
-          // advance 16 k elements = 32 bytes inside the swizzled row: +2 in 16-byte units
-          umma_bf16(tmem_base, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), p.idesc, (i > 0 || kk > 0) ? 1u : 0u);
+          for (int kk = 0; kk < BK / 16; ++kk) {
+            // advance 16 k elements = 32 bytes inside the swizzled row: +2 in 16-byte units
+            const uint32_t acc = (k > 0 || kk > 0) ? 1u : 0u;
+            umma_bf16(tmem_d, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), p.idesc, acc);
+            if (p.wide)
+              umma_bf16(tmem_d + (uint32_t)p.n_mma, umma_desc_sw128(a_src + A_STAGE_BYTES) + (uint64_t)(kk * 2),
+                        bdesc + (uint64_t)(kk * 2), p.idesc, acc);
+          }
+          // Release stages once the MMAs have read them.  Releasing two neighbouring k blocks together
+          // makes the producer request 256 contiguous bytes of every weight row at once.
+          if (p.group == 2 && held < 0 && k + 1 < sg.nkb) {
+            held = s;
+          } else {
+            if (held >= 0) umma_commit(smem_u32(&empty_bar[held]));
+            umma_commit(smem_u32(&empty_bar[s]));
+            held = -1;
+          }
         }
-        umma_commit(smem_u32(&empty_bar[s]));      // frees the stage once these MMAs have read it
+        umma_commit(smem_u32(&acc_full[buf]));       // this segment's accumulator is complete
+        ++g;
       }
-      umma_commit(smem_u32(&accum_bar));           // accumulator complete
     }
   } else {
-    const int quarter = warp & 3;                  // TMEM lanes 32*quarter .. +31 belong to this warp
-    mbar_wait(smem_u32(&accum_bar), 0, aborted, p.status);
-    tc_fence_after();
-    const int n_out = tile * BM + quarter * 32 + lane;
-    const int m_base = mchunk * kGemmRowsPerPass;
-    const int m_cnt = min(p.n_mma, p.M - m_base);
-    float* o = p.out + ((size_t)split * p.M + m_base) * p.N + n_out;
-    const bool n_ok = n_out < p.N;
-    for (int c0 = 0; c0 < m_cnt; c0 += 16) {
-      uint32_t r[16];
-      tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
-      if (n_ok) {
+    const int quarter = warp & 3;                    // TMEM lanes 32*quarter .. +31 belong to this warp
+    griddep_wait();                                  // the kernel before this one may still be reading the partial buffer
+    long long u = u0;
+    Segment sg;
+    int g = 0;
+    while (next_segment(u, u1, p.num_kb, sg)) {
+      const int buf = g & 1;
+      const int tile = sg.job % p.tiles, mchunk = sg.job / p.tiles;
+      mbar_wait(smem_u32(&acc_full[buf]), (uint32_t)(g >> 1) & 1u, aborted, p.status);
+      tc_fence_after();
+      // slot = how many CTAs before this one also work on this job
+      const long long job_u0 = (long long)sg.job * p.num_kb;
+      const int first_cta = (int)(job_u0 / p.per);
+      const int last_cta = (int)((job_u0 + p.num_kb - 1) / p.per);
+      const int slot = (int)blockIdx.x - first_cta;
+      const int m_base = mchunk * kGemmRowsPerPass;
+      const int m_cnt = min(p.n_mma, p.M - m_base);
+      for (int hf = 0; hf <= p.wide; ++hf) {
+        const int n_out = tile * rows_per_tile + hf * BM + quarter * 32 + lane;
+        const bool n_ok = n_out < p.N;
+        float* o = p.out + ((size_t)slot * p.M + m_base) * p.N + n_out;
+        const uint32_t taddr = tmem_base + (uint32_t)buf * p.acc_cols + (uint32_t)(hf * p.n_mma) + ((uint32_t)(quarter * 32) << 16);
+        for (int c0 = 0; c0 < m_cnt; c0 += 16) {
+          uint32_t r[16];
+          tmem_ld16(taddr + (uint32_t)c0, r);
+          if (n_ok) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
-          if (c0 + j < m_cnt) o[(size_t)(c0 + j) * p.N] = __uint_as_float(r[j]);
+            for (int j = 0; j < 16; ++j)
+              if (c0 + j < m_cnt) o[(size_t)(c0 + j) * p.N] = __uint_as_float(r[j]);
+          }
+        }
       }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
+      if ((int)blockIdx.x == last_cta) {
+        for (int hf = 0; hf <= p.wide; ++hf) {
+          const int n_out = tile * rows_per_tile + hf * BM + quarter * 32 + lane;
+          if (n_out >= p.N) continue;
+          for (int z = last_cta - first_cta + 1; z < p.nslots; ++z) {
+            float* zo = p.out + ((size_t)z * p.M + m_base) * p.N + n_out;
+            for (int m = 0; m < m_cnt; ++m) zo[(size_t)m * p.N] = 0.f;
+          }
+        }
+      }
+      ++g;
     }
   }
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2u * p.acc_cols) : "memory");
   }
+}
+
+struct GemmPlan {
+  int tiles, mchunks, num_kb, per, ctas, nslots;
+  long long total;
+};
+
+// Tuning switches (environment, read once): CERB_GEMM_WIDE, CERB_GEMM_GROUP, CERB_GEMM_HINT.
+int tune(const char* name, int dflt) {
+  const char* v = getenv(name);
+  return v ? atoi(v) : dflt;
+}
+bool use_wide(int M) {
+  static int w = tune("CERB_GEMM_WIDE", 1);
+  return w && bucket_rows(row_bucket(M < kGemmRowsPerPass ? M : kGemmRowsPerPass)) <= 128;
+}
+
+GemmPlan make_plan(int sm_count, int M, int N, int K) {
+  GemmPlan g;
+  const int rows_per_tile = BM * (use_wide(M) ? 2 : 1);
+  g.tiles = (N + rows_per_tile - 1) / rows_per_tile;
+  g.mchunks = (M + kGemmRowsPerPass - 1) / kGemmRowsPerPass;
+  g.num_kb = (K + BK - 1) / BK;
+  g.total = (long long)g.tiles * g.mchunks * g.num_kb;
+  long long per = (g.total + sm_count - 1) / sm_count;
+  int min_per = g.num_kb < 4 ? g.num_kb : 4;          // do not shred tiny problems into one-block segments
+  if (per < min_per) per = min_per;
+  g.per = (int)per;
+  g.ctas = (int)((g.total + per - 1) / per);
+  g.nslots = 1;
+  for (long long job = 0; job < (long long)g.tiles * g.mchunks; ++job) {
+    int first = (int)(job * g.num_kb / per), last = (int)((job * g.num_kb + g.num_kb - 1) / per);
+    if (last - first + 1 > g.nslots) g.nslots = last - first + 1;
+  }
+  return g;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -266,50 +439,53 @@ int make_pool_map(CUtensorMap* out, const void* pool, int n_pool_pages, int H, i
   return encode_2d(out, pool, (uint64_t)Dh, (uint64_t)n_pool_pages * H * CERB_PAGE, (uint64_t)Dh * 2, 64, CERB_PAGE);
 }
 
-// How many K splits to use so that about two CTAs per SM stream weights concurrently.
-int gemm_plan_split(int sm_count, int M, int N, int K) {
-  int tiles = (N + BM - 1) / BM;
-  int mchunks = (M + kGemmRowsPerPass - 1) / kGemmRowsPerPass;
-  int num_kb = (K + BK - 1) / BK;
-  int want = (2 * sm_count + tiles * mchunks - 1) / (tiles * mchunks);
-  int max_by_k = num_kb / 4 > 0 ? num_kb / 4 : 1;
-  int s = want < 1 ? 1 : want;
-  if (s > max_by_k) s = max_by_k;
-  if (s > kGemmMaxSplit) s = kGemmMaxSplit;
-  int per = (num_kb + s - 1) / s;
-  return (num_kb + per - 1) / per;
-}
+// Number of partial slots the schedule produces for this problem (what consumers must sum).
+int gemm_plan_split(int sm_count, int M, int N, int K) { return make_plan(sm_count, M, N, K).nslots; }
 
 int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, float* out, int M, int N, int K,
                      int nsplit, int32_t* status, cudaStream_t st) {
   if (M <= 0 || N <= 0 || K <= 0 || (K % 8) != 0) return CERB_E_SHAPE;
+  static int sm_count = 0;
+  if (!sm_count) {
+    int dev = 0;
+    CERB_CUDA_OK(cudaGetDevice(&dev));
+    CERB_CUDA_OK(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
+    if (sm_count > 148) sm_count = 148;      // slot counts are planned for at most 148 CTAs
+  }
+  // Fewer SMs than planned for would need more slots than the caller sized: plan with the number
+  // the caller used (148) and simply run that many CTAs; the hardware queues what does not fit.
+  GemmPlan g = make_plan(148, M, N, K);
+  if (g.nslots != nsplit) return CERB_E_ARG;
   GemmParams p;
-  int mchunks = (M + kGemmRowsPerPass - 1) / kGemmRowsPerPass;
   int bucket = row_bucket(M < kGemmRowsPerPass ? M : kGemmRowsPerPass);
   p.out = out;
   p.status = status;
   p.M = M; p.N = N; p.K = K;
   p.n_mma = bucket_rows(bucket);
-  p.num_kb = (K + BK - 1) / BK;
-  p.kb_per_split = (p.num_kb + nsplit - 1) / nsplit;
-  int splits = (p.num_kb + p.kb_per_split - 1) / p.kb_per_split;
-  if (splits != nsplit) return CERB_E_ARG;
-  uint32_t stage_bytes = A_STAGE_BYTES + (uint32_t)p.n_mma * BK * 2;
-  uint32_t budget = stage_bytes <= 28 * 1024 ? 110 * 1024 : 200 * 1024;
-  p.stages = (int)(budget / stage_bytes);
+  p.num_kb = g.num_kb;
+  p.tiles = g.tiles;
+  p.per = g.per;
+  p.total = g.total;
+  p.nslots = g.nslots;
+  static int group = tune("CERB_GEMM_GROUP", 1), hint = tune("CERB_GEMM_HINT", 1);
+  p.wide = use_wide(M) ? 1 : 0;
+  p.group = group == 2 ? 2 : 1;
+  p.hint = hint ? 1 : 0;
+  uint32_t stage_bytes = A_STAGE_BYTES * (1 + p.wide) + (uint32_t)p.n_mma * BK * 2;
+  p.stages = (int)((216u * 1024u) / stage_bytes);
   if (p.stages > MAX_STAGES) p.stages = MAX_STAGES;
   if (p.stages < 2) return CERB_E_SHAPE;
-  p.tmem_cols = p.n_mma < 32 ? 32u : (uint32_t)p.n_mma;
+  p.acc_cols = (uint32_t)p.n_mma * (1 + p.wide) < 32 ? 32u : (uint32_t)p.n_mma * (1 + p.wide);
   // instruction descriptor: D fp32, A and B bf16, both K-major, N = n_mma, M = 128
   p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_mma >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
   size_t smem = (size_t)p.stages * stage_bytes + 1024;
-  static size_t configured = 0;
-  if (smem > configured) {
+  if (smem < 120 * 1024) smem = 120 * 1024;    // one CTA per SM: a CTA may then own all of tensor memory
+  static bool configured = false;
+  if (!configured) {
     CERB_CUDA_OK(cudaFuncSetAttribute(gemm_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(220 * 1024)));
-    configured = 220 * 1024;
+    configured = true;
   }
-  dim3 grid((N + BM - 1) / BM, nsplit, mchunks);
-  gemm_bf16_kernel<<<grid, 192, smem, st>>>(*tmW, tmX->m[bucket], p);
+  if (launch_pdl(gemm_bf16_kernel, dim3(g.ctas), dim3(192), smem, st, *tmW, tmX->m[bucket], p) != cudaSuccess) return CERB_E_CUDA;
   CERB_LAUNCH_CHECK(c);
   return CERB_OK;
 }

@@ -10,6 +10,8 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(const float* __restrict__
                                                        float* __restrict__ out, int M, int N, int K) {
   __shared__ float sx[TK][TM + 4];
   __shared__ float sw[TK][TN + 4];
+  griddep_wait();
+  griddep_launch();
   int m0 = blockIdx.y * TM, n0 = blockIdx.x * TN;
   int tx = threadIdx.x % 16, ty = threadIdx.x / 16;     // tx -> n, ty -> m
   float acc[4][4] = {};
@@ -46,7 +48,7 @@ __global__ void __launch_bounds__(256) gemm_f32_kernel(const float* __restrict__
 
 int launch_gemm_f32(cerb_ctx* c, const float* X, const float* W, float* out, int M, int N, int K, cudaStream_t st) {
   dim3 grid((N + TN - 1) / TN, (M + TM - 1) / TM);
-  gemm_f32_kernel<<<grid, 256, 0, st>>>(X, W, out, M, N, K);
+  launch_pdl(gemm_f32_kernel, grid, dim3(256), 0, st, X, W, out, M, N, K);
   CERB_LAUNCH_CHECK(c);
   return CERB_OK;
 }

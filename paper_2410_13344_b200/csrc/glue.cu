@@ -35,92 +35,157 @@ __global__ void rope_table_kernel(float2* tab, int max_pos, int half, double bas
   tab[idx] = make_float2((float)c, (float)s);
 }
 
-template <typename T>
-__global__ void embed_kernel(const T* __restrict__ embed, const int32_t* __restrict__ tok, int tok_stride, int tok_off,
-                             const int32_t* __restrict__ n_active, int n, int d, int V, T* __restrict__ x) {
-  int row = blockIdx.x, b = row / n, v = row % n;
-  int t = 0;
-  if (v < n_active[b]) t = tok[(size_t)b * tok_stride + tok_off + v];
-  if (t < 0 || t >= V) t = 0;
-  const T* src = embed + (size_t)t * d;
-  T* dst = x + (size_t)row * d;
-  for (int j = threadIdx.x; j < d; j += blockDim.x) dst[j] = src[j];
+template <typename T> __device__ __forceinline__ void ld4(const T* p, float* f);
+template <> __device__ __forceinline__ void ld4<float>(const float* p, float* f) {
+  float4 v = *reinterpret_cast<const float4*>(p);
+  f[0] = v.x; f[1] = v.y; f[2] = v.z; f[3] = v.w;
 }
+template <> __device__ __forceinline__ void ld4<bf16>(const bf16* p, float* f) {
+  uint2 v = *reinterpret_cast<const uint2*>(p);
+  float2 a = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&v.x)), b = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&v.y));
+  f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y;
+}
+template <typename T> __device__ __forceinline__ void st4(T* p, const float* f);
+template <> __device__ __forceinline__ void st4<float>(float* p, const float* f) {
+  *reinterpret_cast<float4*>(p) = make_float4(f[0], f[1], f[2], f[3]);
+}
+template <> __device__ __forceinline__ void st4<bf16>(bf16* p, const float* f) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(f[0], f[1]), b = __floats2bfloat162_rn(f[2], f[3]);
+  uint2 v;
+  v.x = *reinterpret_cast<uint32_t*>(&a);
+  v.y = *reinterpret_cast<uint32_t*>(&b);
+  *reinterpret_cast<uint2*>(p) = v;
+}
+template <typename T> __device__ __forceinline__ float rnd(float v);
+template <> __device__ __forceinline__ float rnd<float>(float v) { return v; }
+template <> __device__ __forceinline__ float rnd<bf16>(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 
+// One row per CTA, four consecutive columns per thread:
+//   x <- (embedding row | x | x + sum of GEMM partial slots), rounded to the storage type and written back;
+//   out <- RMSNorm(x) * gain.
+// Fusing the residual add (and the first layer's embedding gather) with the norm that always follows
+// it halves the element-wise launches; the slot loads of a thread are independent 16-byte loads.
+constexpr int NORM_THREADS = 1024;
+constexpr int NORM_MAX_ITER = 4;          // d_model up to 16384
 template <typename T>
-__global__ void rmsnorm_kernel(const T* __restrict__ x, const T* __restrict__ gain, T* __restrict__ out, int d, float eps) {
+__global__ void __launch_bounds__(NORM_THREADS) fused_norm_kernel(T* __restrict__ x, const float* __restrict__ part, int nsplit,
+                                                                   size_t split_stride, const T* __restrict__ embed,
+                                                                   const int32_t* __restrict__ tok, int tok_stride, int tok_off,
+                                                                   const int32_t* __restrict__ n_active, int n, int V,
+                                                                   const T* __restrict__ gain, T* __restrict__ out, int d, float eps) {
   __shared__ float red[32];
-  const T* xr = x + (size_t)blockIdx.x * d;
+  griddep_wait();
+  griddep_launch();
+  const int row = blockIdx.x;
+  T* xr = x + (size_t)row * d;
+  const T* src = xr;
+  if (embed) {
+    int b = row / n, v = row % n, t = 0;
+    if (v < n_active[b]) t = tok[(size_t)b * tok_stride + tok_off + v];
+    if (t < 0 || t >= V) t = 0;
+    src = embed + (size_t)t * d;
+  }
+  float keep[NORM_MAX_ITER][4];
   float ss = 0.f;
-  for (int j = threadIdx.x; j < d; j += blockDim.x) { float v = ldf(xr + j); ss += v * v; }
+#pragma unroll
+  for (int it = 0; it < NORM_MAX_ITER; ++it) {
+    const int j = (it * NORM_THREADS + threadIdx.x) * 4;
+    if (j < d) {
+      float v[4];
+      ld4(src + j, v);
+      if (nsplit > 0) {
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float* pr = part + (size_t)row * d + j;
+#pragma unroll 4
+        for (int s = 0; s < nsplit; ++s) {
+          float4 t4 = *reinterpret_cast<const float4*>(pr + s * split_stride);
+          a.x += t4.x; a.y += t4.y; a.z += t4.z; a.w += t4.w;
+        }
+        v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w;
+      }
+      if (embed || nsplit > 0) {
+        st4(xr + j, v);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) v[e] = rnd<T>(v[e]);      // the norm sees the stored (rounded) value
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) { keep[it][e] = v[e]; ss += v[e] * v[e]; }
+    }
+  }
   ss = block_sum(ss, red);
-  float r = 1.0f / sqrtf(ss / (float)d + eps);
-  T* o = out + (size_t)blockIdx.x * d;
-  for (int j = threadIdx.x; j < d; j += blockDim.x) stf(o + j, ldf(xr + j) * r * ldf(gain + j));
+  if (!out) return;
+  const float r = 1.0f / sqrtf(ss / (float)d + eps);
+  T* o = out + (size_t)row * d;
+#pragma unroll
+  for (int it = 0; it < NORM_MAX_ITER; ++it) {
+    const int j = (it * NORM_THREADS + threadIdx.x) * 4;
+    if (j < d) {
+      float gv[4], ov[4];
+      ld4(gain + j, gv);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) ov[e] = keep[it][e] * r * gv[e];
+      st4(o + j, ov);
+    }
+  }
 }
 
 // q,k rotated at position len + depth; k,v stored at slot len + node of the paged pools; q kept dense.
+// One CTA per (row, head), one thread per rotation pair.
 template <typename T>
 __global__ void rope_append_kernel(const float* __restrict__ part, int nsplit, size_t split_stride,
                                    const int32_t* __restrict__ len, const int32_t* __restrict__ n_active,
                                    const int32_t* __restrict__ depth, const int32_t* __restrict__ page_table,
                                    int max_pages, const float2* __restrict__ rope, int max_pos, int n, int H, int Dh,
                                    T* __restrict__ q, T* __restrict__ kpool, T* __restrict__ vpool) {
-  int row = blockIdx.x, b = row / n, v = row % n;
+  griddep_wait();
+  griddep_launch();
+  const int row = blockIdx.x, h = blockIdx.y, b = row / n, v = row % n;
   if (v >= n_active[b]) return;
-  int HD = H * Dh, half = Dh >> 1;
-  int L = len[b];
-  int pos = L + depth[v], slot = L + v;
+  const int HD = H * Dh, half = Dh >> 1;
+  const int L = len[b];
+  const int pos = L + depth[v], slot = L + v;
   if (pos >= max_pos || slot >= max_pos) return;
-  int page = page_table[(size_t)b * max_pages + slot / CERB_PAGE];
-  size_t kv_base = ((size_t)page * H) * CERB_PAGE * Dh + (size_t)(slot % CERB_PAGE) * Dh;
-  const float* pr = part + (size_t)row * 3 * HD;
-  for (int idx = threadIdx.x; idx < H * half; idx += blockDim.x) {
-    int h = idx / half, i = idx % half;
+  const int page = page_table[(size_t)b * max_pages + slot / CERB_PAGE];
+  const size_t kv = (((size_t)page * H + h) * CERB_PAGE + (size_t)(slot % CERB_PAGE)) * Dh;
+  const float* pr = part + (size_t)row * 3 * HD + h * Dh;
+  for (int i = threadIdx.x; i < half; i += blockDim.x) {
     float2 cs = rope[(size_t)pos * half + i];
-    float q1 = 0.f, q2 = 0.f, k1 = 0.f, k2 = 0.f;
+    float q1 = 0.f, q2 = 0.f, k1 = 0.f, k2 = 0.f, v1 = 0.f, v2 = 0.f;
     for (int s = 0; s < nsplit; ++s) {
-      const float* p = pr + s * split_stride + h * Dh + i;
-      q1 += p[0]; q2 += p[half]; k1 += p[HD]; k2 += p[HD + half];
+      const float* p = pr + s * split_stride + i;
+      q1 += p[0]; q2 += p[half]; k1 += p[HD]; k2 += p[HD + half]; v1 += p[2 * HD]; v2 += p[2 * HD + half];
     }
     T* qo = q + (size_t)row * HD + h * Dh + i;
     stf(qo, q1 * cs.x - q2 * cs.y);
     stf(qo + half, q2 * cs.x + q1 * cs.y);
-    T* ko = kpool + kv_base + (size_t)h * CERB_PAGE * Dh + i;
-    stf(ko, k1 * cs.x - k2 * cs.y);
-    stf(ko + half, k2 * cs.x + k1 * cs.y);
+    stf(kpool + kv + i, k1 * cs.x - k2 * cs.y);
+    stf(kpool + kv + i + half, k2 * cs.x + k1 * cs.y);
+    stf(vpool + kv + i, v1);
+    stf(vpool + kv + i + half, v2);
   }
-  for (int idx = threadIdx.x; idx < HD; idx += blockDim.x) {
-    int h = idx / Dh, i = idx % Dh;
-    float vv = 0.f;
-    for (int s = 0; s < nsplit; ++s) vv += pr[s * split_stride + 2 * HD + idx];
-    stf(vpool + kv_base + (size_t)h * CERB_PAGE * Dh + i, vv);
-  }
-}
-
-template <typename T>
-__global__ void residual_kernel(T* __restrict__ x, const float* __restrict__ part, int nsplit, size_t split_stride,
-                                size_t total) {
-  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= total) return;
-  float a = 0.f;
-  for (int s = 0; s < nsplit; ++s) a += part[s * split_stride + i];
-  stf(x + i, ldf(x + i) + a);
 }
 
 template <typename T>
 __global__ void swiglu_kernel(const float* __restrict__ part, int nsplit, size_t split_stride, T* __restrict__ act,
                               int rows, int F) {
+  griddep_wait();
+  griddep_launch();
+  const int F4 = F >> 2;
   size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= (size_t)rows * F) return;
-  size_t row = i / F, j = i % F;
-  float g = 0.f, u = 0.f;
+  if (i >= (size_t)rows * F4) return;
+  size_t row = i / F4, j = (i % F4) * 4;
+  float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
   for (int s = 0; s < nsplit; ++s) {
     const float* p = part + s * split_stride + row * 2 * F;
-    g += p[j];
-    u += p[F + j];
+    float4 a = *reinterpret_cast<const float4*>(p + j), c = *reinterpret_cast<const float4*>(p + F + j);
+    g.x += a.x; g.y += a.y; g.z += a.z; g.w += a.w;
+    u.x += c.x; u.y += c.y; u.z += c.z; u.w += c.w;
   }
-  stf(act + i, g / (1.0f + expf(-g)) * u);
+  T* o = act + row * F + j;
+  stf(o, g.x / (1.0f + expf(-g.x)) * u.x);
+  stf(o + 1, g.y / (1.0f + expf(-g.y)) * u.y);
+  stf(o + 2, g.z / (1.0f + expf(-g.z)) * u.z);
+  stf(o + 3, g.w / (1.0f + expf(-g.w)) * u.w);
 }
 
 // Row argmax over logits given as split-K partial sums; ties go to the lower index.  When
@@ -129,6 +194,8 @@ __global__ void argmax_rows_kernel(const float* __restrict__ part, int nsplit, s
                                    int32_t* __restrict__ out, float* __restrict__ summed) {
   __shared__ float sv[32];
   __shared__ int si[32];
+  griddep_wait();
+  griddep_launch();
   const float* r = part + (size_t)blockIdx.x * V;
   float best = -INFINITY;
   int bi = 0x7fffffff;
@@ -155,6 +222,8 @@ __global__ void argmax_rows_kernel(const float* __restrict__ part, int nsplit, s
 
 // mode 0: n_active[b] = a.  mode 1 (prefill chunk): n_active[b] = clamp(lens_in[b] - a, 0, b_).
 __global__ void set_nactive_kernel(int32_t* n_active, const int32_t* lens_in, int B, int mode, int a, int b_) {
+  griddep_wait();
+  griddep_launch();
   int b = threadIdx.x;
   if (b >= B) return;
   if (mode == 0) n_active[b] = a;
@@ -168,6 +237,8 @@ __global__ void set_nactive_kernel(int32_t* n_active, const int32_t* lens_in, in
 template <typename T>
 __global__ void prefill_commit_kernel(const int32_t* __restrict__ n_active, int32_t* __restrict__ len,
                                       const T* __restrict__ hidden, T* __restrict__ h_last, int n, int d) {
+  griddep_wait();
+  griddep_launch();
   int b = blockIdx.x, na = n_active[b];
   if (na <= 0) return;
   const T* src = hidden + ((size_t)b * n + na - 1) * d;
@@ -183,24 +254,20 @@ int launch_rope_table(cerb_ctx* c, cudaStream_t st) {
   return CERB_OK;
 }
 
-int launch_embed(cerb_ctx* c, const int32_t* tok, int tok_stride, int tok_off, int B, int n, cudaStream_t st) {
-  int d = c->cfg.d_model;
+// x <- embedding rows (tok != null) | x + partials (nsplit > 0) | x;  out <- RMSNorm(x) * gain (out may be null).
+int launch_fused_norm(cerb_ctx* c, const float* part, int nsplit, size_t split_stride, const int32_t* tok, int tok_stride,
+                      int tok_off, int n, const void* gain, void* out, int rows, cudaStream_t st) {
+  const cerb_config& g = c->cfg;
+  const int d = g.d_model;
+  if (d % 4 || d > NORM_THREADS * NORM_MAX_ITER * 4) return CERB_E_SHAPE;
   if (c->bf16)
-    embed_kernel<bf16><<<B * n, 128, 0, st>>>((const bf16*)c->embed, tok, tok_stride, tok_off, c->d_nactive, n, d,
-                                              c->cfg.vocab, (bf16*)c->d_x);
+    launch_pdl(fused_norm_kernel<bf16>, dim3(rows), dim3(NORM_THREADS), 0, st, (bf16*)c->d_x, part, nsplit, split_stride,
+               tok ? (const bf16*)c->embed : (const bf16*)nullptr, tok, tok_stride, tok_off, (const int32_t*)c->d_nactive, n,
+               g.vocab, (const bf16*)gain, (bf16*)out, d, g.rms_eps);
   else
-    embed_kernel<float><<<B * n, 128, 0, st>>>((const float*)c->embed, tok, tok_stride, tok_off, c->d_nactive, n, d,
-                                               c->cfg.vocab, (float*)c->d_x);
-  CERB_LAUNCH_CHECK(c);
-  return CERB_OK;
-}
-
-int launch_rmsnorm(cerb_ctx* c, const void* x, const void* gain, void* out, int rows, cudaStream_t st) {
-  int d = c->cfg.d_model;
-  if (c->bf16)
-    rmsnorm_kernel<bf16><<<rows, 256, 0, st>>>((const bf16*)x, (const bf16*)gain, (bf16*)out, d, c->cfg.rms_eps);
-  else
-    rmsnorm_kernel<float><<<rows, 256, 0, st>>>((const float*)x, (const float*)gain, (float*)out, d, c->cfg.rms_eps);
+    launch_pdl(fused_norm_kernel<float>, dim3(rows), dim3(NORM_THREADS), 0, st, (float*)c->d_x, part, nsplit, split_stride,
+               tok ? (const float*)c->embed : (const float*)nullptr, tok, tok_stride, tok_off, (const int32_t*)c->d_nactive, n,
+               g.vocab, (const float*)gain, (float*)out, d, g.rms_eps);
   CERB_LAUNCH_CHECK(c);
   return CERB_OK;
 }
@@ -211,40 +278,30 @@ int launch_rope_append(cerb_ctx* c, int layer, const TreeDev& t, const float* pa
   char* kp = c->k_pool + (size_t)layer * c->pool_layer_bytes;
   char* vp = c->v_pool + (size_t)layer * c->pool_layer_bytes;
   if (c->bf16)
-    rope_append_kernel<bf16><<<B * n, 256, 0, st>>>(part, nsplit, split_stride, c->d_len, c->d_nactive, t.depth,
-                                                    c->page_table, g.max_pages, c->d_rope, c->max_pos, n, g.n_heads,
-                                                    g.head_dim, (bf16*)c->d_q, (bf16*)kp, (bf16*)vp);
+    launch_pdl(rope_append_kernel<bf16>, dim3(B * n, g.n_heads), dim3(64), 0, st, part, nsplit, split_stride,
+               (const int32_t*)c->d_len, (const int32_t*)c->d_nactive, (const int32_t*)t.depth, c->page_table, g.max_pages,
+               (const float2*)c->d_rope, c->max_pos, n, g.n_heads, g.head_dim, (bf16*)c->d_q, (bf16*)kp, (bf16*)vp);
   else
-    rope_append_kernel<float><<<B * n, 256, 0, st>>>(part, nsplit, split_stride, c->d_len, c->d_nactive, t.depth,
-                                                     c->page_table, g.max_pages, c->d_rope, c->max_pos, n, g.n_heads,
-                                                     g.head_dim, (float*)c->d_q, (float*)kp, (float*)vp);
-  CERB_LAUNCH_CHECK(c);
-  return CERB_OK;
-}
-
-int launch_residual(cerb_ctx* c, void* x, const float* part, int nsplit, size_t split_stride, int rows, int N,
-                    cudaStream_t st) {
-  size_t total = (size_t)rows * N;
-  unsigned blocks = (unsigned)((total + 255) / 256);
-  if (c->bf16) residual_kernel<bf16><<<blocks, 256, 0, st>>>((bf16*)x, part, nsplit, split_stride, total);
-  else residual_kernel<float><<<blocks, 256, 0, st>>>((float*)x, part, nsplit, split_stride, total);
+    launch_pdl(rope_append_kernel<float>, dim3(B * n, g.n_heads), dim3(64), 0, st, part, nsplit, split_stride,
+               (const int32_t*)c->d_len, (const int32_t*)c->d_nactive, (const int32_t*)t.depth, c->page_table, g.max_pages,
+               (const float2*)c->d_rope, c->max_pos, n, g.n_heads, g.head_dim, (float*)c->d_q, (float*)kp, (float*)vp);
   CERB_LAUNCH_CHECK(c);
   return CERB_OK;
 }
 
 int launch_swiglu(cerb_ctx* c, const float* part, int nsplit, size_t split_stride, void* act, int rows, cudaStream_t st) {
   int F = c->cfg.mlp_dim;
-  size_t total = (size_t)rows * F;
+  size_t total = (size_t)rows * (F / 4);
   unsigned blocks = (unsigned)((total + 255) / 256);
-  if (c->bf16) swiglu_kernel<bf16><<<blocks, 256, 0, st>>>(part, nsplit, split_stride, (bf16*)act, rows, F);
-  else swiglu_kernel<float><<<blocks, 256, 0, st>>>(part, nsplit, split_stride, (float*)act, rows, F);
+  if (c->bf16) launch_pdl(swiglu_kernel<bf16>, dim3(blocks), dim3(256), 0, st, part, nsplit, split_stride, (bf16*)act, rows, F);
+  else launch_pdl(swiglu_kernel<float>, dim3(blocks), dim3(256), 0, st, part, nsplit, split_stride, (float*)act, rows, F);
   CERB_LAUNCH_CHECK(c);
   return CERB_OK;
 }
 
 int launch_argmax_rows(cerb_ctx* c, const float* part, int nsplit, size_t split_stride, int rows, int V, int32_t* out,
                        float* summed, cudaStream_t st) {
-  argmax_rows_kernel<<<rows, 1024, 0, st>>>(part, nsplit, split_stride, V, out, summed);
+  launch_pdl(argmax_rows_kernel, dim3(rows), dim3(1024), 0, st, part, nsplit, split_stride, V, out, summed);
   CERB_LAUNCH_CHECK(c);
   return CERB_OK;
 }

@@ -59,6 +59,8 @@ template <> __device__ __forceinline__ float ldf<bf16>(const bf16* p) { return _
 template <typename T, int NB>
 __global__ void __launch_bounds__(WARPS * 32) head_gemv_kernel(const LevelParams P) {
   extern __shared__ float su[];                       // [NB][w]
+  griddep_wait();
+  griddep_launch();
   const int head = blockIdx.y;
   const HeadJob J = P.job[head];
   const int w = J.w0 + J.w1;
@@ -128,6 +130,8 @@ __global__ void __launch_bounds__(WARPS * 32) head_gemv_kernel(const LevelParams
 
 template <typename T>
 __global__ void head_init_kernel(const T* __restrict__ h_last, float* __restrict__ state, int Hc, int wmax, int d) {
+  griddep_wait();
+  griddep_launch();
   int b = blockIdx.x, h = blockIdx.y;
   for (int k = threadIdx.x; k < d; k += blockDim.x)
     state[((size_t)b * Hc + h) * wmax + k] = ldf(h_last + (size_t)b * d + k);
@@ -144,6 +148,8 @@ __global__ void __launch_bounds__(1024) topk_kernel(const float* __restrict__ lo
   __shared__ int si[32];
   __shared__ float pv_s;
   __shared__ int pi_s;
+  griddep_wait();
+  griddep_launch();
   const int h = blockIdx.x, b = blockIdx.y;
   const float* r = logits + ((size_t)b * Hc + h) * V;
   const int k = kper[h];
@@ -189,6 +195,8 @@ __global__ void __launch_bounds__(1024) topk_kernel(const float* __restrict__ lo
 __global__ void tree_fill_kernel(const int32_t* __restrict__ root, const int32_t* __restrict__ topk,
                                  const int32_t* __restrict__ head_of, const int32_t* __restrict__ rank_of,
                                  const int32_t* __restrict__ plant, int Hc, int n, int32_t* __restrict__ tree_tok) {
+  griddep_wait();
+  griddep_launch();
   int b = blockIdx.x;
   for (int v = threadIdx.x; v < n; v += blockDim.x) {
     int t;
