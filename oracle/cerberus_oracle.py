@@ -43,11 +43,10 @@ specification, not by code):
     argmax at the last accepted node becomes the next step's root.
   * RoPE position of a node = committed length + depth; its KV slot = committed
     length + node index; accepted nodes are moved to consecutive slots.
-  * bf16 models: values are rounded to bf16 exactly at: the residual stream
-    after each residual add, every norm output, q and k after RoPE, v, the
-    attention output, the SwiGLU output.  Everything else (accumulation,
-    softmax, logits, head states, entropy) is unrounded.  fp32 models: no
-    rounding at all (the oracle stays in float64).
+  * bf16 models: values are rounded to bf16 exactly at: every norm output, q and
+    k after RoPE, v, the attention output, the SwiGLU output.  Everything else
+    (the residual stream, accumulation, softmax, logits, head states, entropy)
+    is unrounded.  fp32 models: no rounding at all (the oracle stays in float64).
   * Integer decisions (argmax, top-k) are taken on logits cast to float32, the
     precision the kernels decide in; ties go to the lower token id.
 """
@@ -216,11 +215,11 @@ def _qkv(x, model, l, sh: Shape, pos):
 def _post_attention(x, a, model, l, sh: Shape):
     T = x.shape[0]
     F = sh.mlp_dim
-    x = rb(x + a.reshape(T, -1) @ f64(model[f"wo.{l}"]).T, sh.act)
+    x = x + a.reshape(T, -1) @ f64(model[f"wo.{l}"]).T
     xn = rb(rmsnorm(x, f64(model[f"mlp_norm.{l}"]), sh.rms_eps), sh.act)
     gu = xn @ f64(model[f"wgu.{l}"]).T
     m = rb(silu(gu[:, :F]) * gu[:, F:], sh.act)
-    return rb(x + m @ f64(model[f"wd.{l}"]).T, sh.act)
+    return x + m @ f64(model[f"wd.{l}"]).T
 
 
 def _final(x, model, sh: Shape, want_logits=True):
@@ -235,7 +234,7 @@ def forward_full(model, sh: Shape, tokens: Sequence[int]):
     tok = torch.as_tensor(list(tokens), dtype=torch.long)
     T = tok.shape[0]
     pos = list(range(T))
-    x = rb(f64(model["embed"][tok]), sh.act)
+    x = f64(model["embed"][tok])
     kv = []
     for l in range(sh.n_layers):
         q, k, v = _qkv(x, model, l, sh, pos)
@@ -309,7 +308,7 @@ def verify_tree(model, sh: Shape, st: State, tree_tok: Sequence[int], parent: Se
     n = len(tree_tok)
     tok = torch.as_tensor(list(tree_tok), dtype=torch.long)
     pos = [st.length + node_depth(parent, v) for v in range(n)]
-    x = rb(f64(model["embed"][tok]), sh.act)
+    x = f64(model["embed"][tok])
     L = st.length
     for l in range(sh.n_layers):
         q, k, v = _qkv(x, model, l, sh, pos)

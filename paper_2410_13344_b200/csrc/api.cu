@@ -132,7 +132,7 @@ size_t carve(cerb_ctx* c, char* base) {
   c->d_treetok = b.take<int32_t>(MB * CERB_MAX_NODES);
   c->d_topk = b.take<int32_t>(MB * CERB_MAX_HEADS * CERB_MAX_TOPK);
   c->d_hlast = b.take<char>((size_t)MB * g.d_model * es);
-  c->d_x = b.take<char>((size_t)Mr * g.d_model * es);
+  c->d_x = b.take<char>((size_t)Mr * g.d_model * sizeof(float));     // residual stream, always fp32
   c->d_xn = b.take<char>((size_t)Mr * g.d_model * es);
   c->d_hidden = b.take<char>((size_t)Mr * g.d_model * es);
   c->d_q = b.take<char>((size_t)Mr * HD * es);

@@ -56,19 +56,15 @@ template <> __device__ __forceinline__ void st4<bf16>(bf16* p, const float* f) {
   v.y = *reinterpret_cast<uint32_t*>(&b);
   *reinterpret_cast<uint2*>(p) = v;
 }
-template <typename T> __device__ __forceinline__ float rnd(float v);
-template <> __device__ __forceinline__ float rnd<float>(float v) { return v; }
-template <> __device__ __forceinline__ float rnd<bf16>(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
-
 // One row per CTA, four consecutive columns per thread:
-//   x <- (embedding row | x | x + sum of GEMM partial slots), rounded to the storage type and written back;
-//   out <- RMSNorm(x) * gain.
+//   x <- (embedding row | x | x + sum of GEMM partial slots), kept in fp32 (the residual stream is never rounded);
+//   out <- RMSNorm(x) * gain, in the model's storage type.
 // Fusing the residual add (and the first layer's embedding gather) with the norm that always follows
 // it halves the element-wise launches; the slot loads of a thread are independent 16-byte loads.
 constexpr int NORM_THREADS = 1024;
 constexpr int NORM_MAX_ITER = 4;          // d_model up to 16384
 template <typename T>
-__global__ void __launch_bounds__(NORM_THREADS) fused_norm_kernel(T* __restrict__ x, const float* __restrict__ part, int nsplit,
+__global__ void __launch_bounds__(NORM_THREADS) fused_norm_kernel(float* __restrict__ x, const float* __restrict__ part, int nsplit,
                                                                    size_t split_stride, const T* __restrict__ embed,
                                                                    const int32_t* __restrict__ tok, int tok_stride, int tok_off,
                                                                    const int32_t* __restrict__ n_active, int n, int V,
@@ -77,8 +73,8 @@ __global__ void __launch_bounds__(NORM_THREADS) fused_norm_kernel(T* __restrict_
   griddep_wait();
   griddep_launch();
   const int row = blockIdx.x;
-  T* xr = x + (size_t)row * d;
-  const T* src = xr;
+  float* xr = x + (size_t)row * d;
+  const T* src = nullptr;
   if (embed) {
     int b = row / n, v = row % n, t = 0;
     if (v < n_active[b]) t = tok[(size_t)b * tok_stride + tok_off + v];
@@ -92,7 +88,8 @@ __global__ void __launch_bounds__(NORM_THREADS) fused_norm_kernel(T* __restrict_
     const int j = (it * NORM_THREADS + threadIdx.x) * 4;
     if (j < d) {
       float v[4];
-      ld4(src + j, v);
+      if (src) ld4(src + j, v);
+      else ld4(xr + j, v);
       if (nsplit > 0) {
         float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
         const float* pr = part + (size_t)row * d + j;
@@ -103,11 +100,7 @@ __global__ void __launch_bounds__(NORM_THREADS) fused_norm_kernel(T* __restrict_
         }
         v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w;
       }
-      if (embed || nsplit > 0) {
-        st4(xr + j, v);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) v[e] = rnd<T>(v[e]);      // the norm sees the stored (rounded) value
-      }
+      if (embed || nsplit > 0) st4(xr + j, v);
 #pragma unroll
       for (int e = 0; e < 4; ++e) { keep[it][e] = v[e]; ss += v[e] * v[e]; }
     }
@@ -261,7 +254,7 @@ int launch_fused_norm(cerb_ctx* c, const float* part, int nsplit, size_t split_s
   const int d = g.d_model;
   if (d % 4 || d > NORM_THREADS * NORM_MAX_ITER * 4) return CERB_E_SHAPE;
   if (c->bf16)
-    launch_pdl(fused_norm_kernel<bf16>, dim3(rows), dim3(NORM_THREADS), 0, st, (bf16*)c->d_x, part, nsplit, split_stride,
+    launch_pdl(fused_norm_kernel<bf16>, dim3(rows), dim3(NORM_THREADS), 0, st, (float*)c->d_x, part, nsplit, split_stride,
                tok ? (const bf16*)c->embed : (const bf16*)nullptr, tok, tok_stride, tok_off, (const int32_t*)c->d_nactive, n,
                g.vocab, (const bf16*)gain, (bf16*)out, d, g.rms_eps);
   else
