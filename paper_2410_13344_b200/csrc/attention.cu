@@ -298,11 +298,19 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
 
       // ---- O += P V ----
 #pragma unroll
+      // Probabilities enter the tensor core as two bf16 terms, p = p_hi + p_lo (about 16 significant
+      // bits), so that the product is not limited by bf16's 8-bit significand: with near-uniform
+      // attention over many keys a single bf16 term costs as much accuracy as all other roundings together.
       for (int j = 0; j < KW / 16; ++j) {
-        uint32_t a0 = pack_bf16(sc[2 * j][0], sc[2 * j][1]);
-        uint32_t a1 = pack_bf16(sc[2 * j][2], sc[2 * j][3]);
-        uint32_t a2 = pack_bf16(sc[2 * j + 1][0], sc[2 * j + 1][1]);
-        uint32_t a3 = pack_bf16(sc[2 * j + 1][2], sc[2 * j + 1][3]);
+        uint32_t ah[4], al[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float p0 = sc[2 * j + (e >> 1)][(e & 1) * 2], p1 = sc[2 * j + (e >> 1)][(e & 1) * 2 + 1];
+          __nv_bfloat162 hi = __floats2bfloat162_rn(p0, p1);
+          float2 hf = __bfloat1622float2(hi);
+          ah[e] = *reinterpret_cast<uint32_t*>(&hi);
+          al[e] = pack_bf16(p0 - hf.x, p1 - hf.y);
+        }
 #pragma unroll
         for (int dn = 0; dn < DH / 8; dn += 2) {
           int key = ki * KW + j * 16 + (mat & 1) * 8 + lr;
@@ -310,8 +318,10 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
           uint32_t addr = vbase + (uint32_t)(chunk >> 3) * HALF_BYTES + (uint32_t)key * 128 + (uint32_t)(((chunk & 7) ^ (key & 7)) << 4);
           uint32_t b0, b1, b2, b3;
           ldsm_x4_t(addr, b0, b1, b2, b3);
-          mma_bf16(o[dn], a0, a1, a2, a3, b0, b1);
-          mma_bf16(o[dn + 1], a0, a1, a2, a3, b2, b3);
+          mma_bf16(o[dn], ah[0], ah[1], ah[2], ah[3], b0, b1);
+          mma_bf16(o[dn + 1], ah[0], ah[1], ah[2], ah[3], b2, b3);
+          mma_bf16(o[dn], al[0], al[1], al[2], al[3], b0, b1);
+          mma_bf16(o[dn + 1], al[0], al[1], al[2], al[3], b2, b3);
         }
       }
       __syncwarp();
