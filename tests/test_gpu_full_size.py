@@ -11,7 +11,7 @@ import torch
 
 from oracle import cerberus_oracle as orc
 from paper_2410_13344_b200 import synth
-from tests.helpers import assert_close_large, close, concat_src, cpu, oracle_shape, plant_tokens, top2_margin
+from tests.helpers import assert_close_large, close, concat_src, cpu, deepest_path, oracle_shape, top2_margin
 
 pytestmark = pytest.mark.gpu
 TOL = 2e-2
@@ -105,7 +105,8 @@ def _teacher_forced_steps(cb, eng, tree, prompts, n_steps, lengths):
       * every argmax is exact on the kernel's own logits; acceptance equals the oracle's rule applied to
         those argmaxes (exact);
       * compaction moves the accepted nodes' K/V bit-exactly; len and the next root follow.
-    Candidates are planted from an auto-regressive run so that paths of several tokens are accepted."""
+    Candidates are planted with the greedy continuation from the current state (obtained by chain-shaped
+    forwards) so that paths of several tokens are accepted."""
     B = len(prompts)
     tol = _depth_tol(eng.shape.n_layers)
     maxlen = max(len(p) for p in prompts)
@@ -114,14 +115,8 @@ def _teacher_forced_steps(cb, eng, tree, prompts, n_steps, lengths):
         tok[b, :len(p)] = torch.tensor(p, dtype=torch.int32)
     lens0 = [len(p) for p in prompts]
     th, th1 = eng.tree(tree), eng.tree(synth.single_node_tree())
-    eng.prefill(tok, lens0)
-    truth = [[] for _ in range(B)]
-    for _ in range(5 * n_steps + 4):
-        eng.step(th, -1.0)                       # the entropy is never below -1: every step is auto-regressive
-        torch.cuda.synchronize()
-        for b in range(B):
-            assert int(eng.h_mode[b]) == 1 and int(eng.h_n_accept[b]) == 1
-            truth[b].append(int(eng.h_tokens[b, 0]))
+    max_want = max(lengths)
+    chains = {j: eng.tree(synth.chain_tree(j)) for j in range(2, max_want)}
     eng.prefill(tok, lens0)
     layers = (0, eng.shape.n_layers - 1)
     emitted = [[] for _ in range(B)]
@@ -131,15 +126,20 @@ def _teacher_forced_steps(cb, eng, tree, prompts, n_steps, lengths):
         roots_t = torch.tensor(roots, dtype=torch.int32, device="cuda").reshape(B, 1)
         am1, lg1, _ = eng.verify(th1, roots_t, want_logits=True)
         kv1 = [[tuple(t[int(lens[b])].clone() for t in eng.gather_kv(b, l, int(lens[b]) + 1)) for l in layers] for b in range(B)]
+        # the greedy continuation from this state, by chain-shaped forwards of growing length
+        cont = [[int(roots[b]), int(am1[b, 0])] for b in range(B)]
+        for j in range(2, max_want):
+            ct = torch.tensor([c[:j] for c in cont], dtype=torch.int32, device="cuda")
+            amc, _, _ = eng.verify(chains[j], ct)
+            for b in range(B):
+                cont[b].append(int(amc[b, j - 1]))
         tree_tok, _, _ = eng.draft(th)
+        path = deepest_path(tree)
         for b in range(B):
             assert int(tree_tok[b, 0]) == int(roots[b])
-            # follow the auto-regressive continuation while this run has not left it
-            if emitted[b] == truth[b][:len(emitted[b])] and int(roots[b]) == truth[b][len(emitted[b])]:
-                ov = plant_tokens(tree, truth[b], len(emitted[b]), lengths[(step + b) % len(lengths)])
-                for v, t in enumerate(ov):
-                    if t >= 0:
-                        tree_tok[b, v] = t
+            want = lengths[(step + b) % len(lengths)]
+            for j, node in enumerate(path[1:want], start=1):
+                tree_tok[b, node] = cont[b][j]
         am, lg, _ = eng.verify(th, tree_tok, want_logits=True)
         torch.cuda.synchronize()
         snap = [[tuple(t[int(lens[b]):].clone() for t in eng.gather_kv(b, l, int(lens[b]) + tree.n)) for l in layers] for b in range(B)]
