@@ -11,6 +11,8 @@
 // (sequence, head) merges the partials in split order, so the result does not depend on timing.
 //
 // fp32 path (CERB_F32 models): plain FMA arithmetic, one CTA per (node, head, sequence).
+#include <stdlib.h>
+
 #include "cerb_internal.cuh"
 
 namespace cerb {
@@ -104,6 +106,8 @@ struct AttnParams {
   unsigned int* counters;   // [B*H]
   int32_t* status;
   int n, H, max_pages, nsplit, oob_row;
+  int rows_pad;             // rows per split in `partial` (16, 32, 64 or 128)
+  uint32_t v_lbo, v_sbo;    // byte offsets of the V operand's descriptor (tensor-core path)
   float scale_log2;
 };
 
@@ -424,6 +428,397 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
 }
 
 // ---------------------------------------------------------------------------------------------
+// bf16 path on the 5th-generation tensor cores (head_dim 128)
+// ---------------------------------------------------------------------------------------------
+// Same decomposition as above (one CTA per (split, head, sequence), 64-key tiles streamed by TMA),
+// but both products run as tcgen05 MMAs with their results in tensor memory:
+//   S[128 x 64]  = Q[128 x 128] . K_tile^T      (Q staged once in shared memory, zero rows past n)
+//   O[128 x 128] += P[128 x 64] . V_tile        (P = p_hi + p_lo, two bf16 terms, staged in shared memory)
+// Warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer, warps 2-5 = softmax: thread t owns
+// query row t (= TMEM lane t), reads its S row from TMEM, keeps the running maximum and sum in
+// registers, writes its P row (128-byte swizzled, the MMA's K-major A layout).  S is double-buffered
+// so the next tile's scores are computed while this tile's probabilities are formed.  O stays in
+// TMEM across tiles; it is only rescaled when a row's maximum grows by more than 2^8 (until then the
+// older maximum keeps being used, which is exact after the final normalisation).
+namespace {
+
+constexpr int TC_STAGES = 4;
+constexpr uint32_t TC_KV_BYTES = 16384;               // K (or V) of one 64-key tile, two 64-wide halves
+constexpr uint32_t TC_STAGE_BYTES = 2 * TC_KV_BYTES;
+constexpr uint32_t TC_Q_BYTES = 32768, TC_P_BYTES = 16384;
+constexpr size_t TC_SMEM = (size_t)TC_STAGES * TC_STAGE_BYTES + TC_Q_BYTES + 2 * TC_P_BYTES + 1024;
+constexpr int TC_DH = 128, TC_ROWF = TC_DH + 4;
+constexpr float TC_RESCALE = 8.0f;                    // log2 of the growth of a row maximum that forces a rescale
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ uint64_t desc_k_sw128(uint32_t saddr) {      // K-major rows of 128 bytes, 128-byte swizzle
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024u >> 4) << 32) | ((uint64_t)1 << 46) |
+         ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ uint64_t desc_mn_sw128(uint32_t saddr, uint32_t lbo, uint32_t sbo) {   // MN-major (V: [key][dh])
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | ((uint64_t)1 << 46) |
+         ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__global__ void __launch_bounds__(192, 1) tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK,
+                                                              const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+  constexpr int DH = TC_DH, ROWF = TC_ROWF, STAGES = TC_STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], s_full[2], s_free[2], q_ready, p_ready, pv_done;
+  __shared__ int page_list[kMaxPagesPerCta];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int aborted_s;
+  __shared__ unsigned int ticket_s;
+  volatile int* aborted = &aborted_s;
+
+  griddep_wait();
+  griddep_launch();
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t q_base = smem_base + STAGES * TC_STAGE_BYTES, ph_base = q_base + TC_Q_BYTES, pl_base = ph_base + TC_P_BYTES;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int L = p.len[b];
+  const int nq = p.n_active ? min(p.n_active[b], p.n) : p.n;
+  if (nq <= 0) return;
+  const int kv_total = L + nq;
+  const int tiles = (kv_total + TILE - 1) / TILE;
+  const int per = (tiles + p.nsplit - 1) / p.nsplit;
+  const int t0 = min(tiles, split * per), t1 = min(tiles, t0 + per);
+  const bool too_long = per * PAGES_PER_TILE > kMaxPagesPerCta;
+  const int T = too_long ? 0 : t1 - t0;
+
+  if (threadIdx.x == 0) {
+    aborted_s = (*p.status != 0);
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&s_full[i]), 1);
+      mbar_init(smem_u32(&s_free[i]), 4);
+    }
+    mbar_init(smem_u32(&q_ready), 4);
+    mbar_init(smem_u32(&p_ready), 4);
+    mbar_init(smem_u32(&pv_done), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (too_long) atomicExch(p.status, CERB_E_SHAPE);
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(256u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_slot;                 // columns 0-63 / 64-127: S buffers, 128-255: O
+  float* mrg = reinterpret_cast<float*>(smem_gen); // [128][ROWF] in the stage ring, once the key loop is over
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    const int32_t* pt = p.page_table + (size_t)b * p.max_pages;
+    const int n_pages = T * PAGES_PER_TILE;
+    for (int i = lane; i < n_pages; i += 32) {
+      int lp = t0 * PAGES_PER_TILE + i;
+      page_list[i] = (lp * CERB_PAGE < kv_total && lp < p.max_pages) ? (pt[lp] * p.H + h) * CERB_PAGE : p.oob_row;
+    }
+    __syncwarp();
+    if (lane == 0) {
+      for (int i = 0; i < T; ++i) {
+        const int s = i % STAGES;
+        mbar_wait(smem_u32(&empty_bar[s]), ((uint32_t)(i / STAGES) & 1u) ^ 1u, aborted, p.status);
+        const uint32_t fb = smem_u32(&full_bar[s]);
+        mbar_expect_tx(fb, TC_STAGE_BYTES);
+        const uint32_t kdst = smem_base + (uint32_t)s * TC_STAGE_BYTES, vdst = kdst + TC_KV_BYTES;
+#pragma unroll
+        for (int pg = 0; pg < PAGES_PER_TILE; ++pg) {
+          const int row = page_list[i * PAGES_PER_TILE + pg];       // out-of-range rows are zero-filled by TMA
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            const uint32_t off = (uint32_t)hf * 8192u + (uint32_t)pg * (CERB_PAGE * 128);
+            tma_load_2d(kdst + off, &tmK, hf * 64, row, fb);
+            tma_load_2d(vdst + off, &tmV, hf * 64, row, fb);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0 && T > 0) {
+      const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+      const uint32_t idesc_pv = idesc_s | (1u << 16);            // B operand (V) is MN-major
+      auto issue_s = [&](int i) {
+        const uint32_t kb = smem_base + (uint32_t)(i % STAGES) * TC_STAGE_BYTES;
+        const uint32_t d = tmem + (uint32_t)(i & 1) * 64u;
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk)
+            umma(d, desc_k_sw128(q_base + hf * 16384u) + (uint64_t)(kk * 2), desc_k_sw128(kb + hf * 8192u) + (uint64_t)(kk * 2),
+                 idesc_s, (hf | kk) ? 1u : 0u);
+        umma_commit(smem_u32(&s_full[i & 1]));
+      };
+      mbar_wait(smem_u32(&q_ready), 0, aborted, p.status);
+      mbar_wait(smem_u32(&full_bar[0]), 0, aborted, p.status);
+      tc_fence_after();
+      issue_s(0);
+      for (int i = 0; i < T; ++i) {
+        if (i + 1 < T) {
+          const int j = i + 1;
+          mbar_wait(smem_u32(&full_bar[j % STAGES]), (uint32_t)(j / STAGES) & 1u, aborted, p.status);
+          mbar_wait(smem_u32(&s_free[j & 1]), ((uint32_t)(j >> 1) & 1u) ^ 1u, aborted, p.status);
+          tc_fence_after();
+          issue_s(j);
+        }
+        mbar_wait(smem_u32(&p_ready), (uint32_t)i & 1u, aborted, p.status);
+        tc_fence_after();
+        const uint32_t vb = smem_base + (uint32_t)(i % STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+          for (int term = 0; term < 2; ++term)
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+              umma(tmem + 128u + hf * 64u, desc_k_sw128(term ? pl_base : ph_base) + (uint64_t)(ks * 2),
+                   desc_mn_sw128(vb + hf * 8192u + ks * 2048u, p.v_lbo, p.v_sbo), idesc_pv, (i == 0 && term == 0 && ks == 0) ? 0u : 1u);
+        umma_commit(smem_u32(&empty_bar[i % STAGES]));   // K and V of this tile are no longer needed
+        umma_commit(smem_u32(&pv_done));
+      }
+    }
+  } else {
+    // ---------------- softmax warps: thread <-> query row ----------------
+    const int row = (warp & 3) * 32 + lane;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const bool valid = row < nq;
+    {
+      // stage this row of Q (zeros past the last node) in the swizzled K-major layout
+      const uint4* src = reinterpret_cast<const uint4*>(p.q + (((size_t)b * p.n + (valid ? row : 0)) * p.H + h) * DH);
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        uint4 v = valid ? src[c] : make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(smem_gen + (q_base - smem_base) + (uint32_t)(c >> 3) * 16384u + (uint32_t)row * 128u +
+                                  (uint32_t)(((c & 7) ^ (row & 7)) << 4)) = v;
+      }
+      proxy_fence();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&q_ready));
+    }
+    uint64_t anc0 = 0, anc1 = 0;
+    if (valid) { anc0 = p.anc[row * 2]; anc1 = p.anc[row * 2 + 1]; }
+    float m_used = -INFINITY, l = 0.f;
+    for (int i = 0; i < T; ++i) {
+      const int buf = i & 1;
+      mbar_wait(smem_u32(&s_full[buf]), (uint32_t)(i >> 1) & 1u, aborted, p.status);
+      tc_fence_after();
+      float sc[64];
+#pragma unroll
+      for (int c0 = 0; c0 < 64; c0 += 16) tmem_ld16(tmem + lane_base + (uint32_t)(buf * 64 + c0), reinterpret_cast<uint32_t*>(sc + c0));
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&s_free[buf]));
+      const int key0 = (t0 + i) * TILE;
+      const bool need_mask = key0 + TILE > L;
+      float mx = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 64; ++j) {
+        float v = sc[j] * p.scale_log2;
+        if (need_mask) {
+          const int kpos = key0 + j;
+          bool vis = kpos < L;
+          if (!vis && kpos < kv_total) {
+            const int t = kpos - L;
+            vis = ((t < 64 ? anc0 : anc1) >> (t & 63)) & 1ull;
+          }
+          if (!vis) v = -INFINITY;
+        }
+        sc[j] = v;
+        mx = fmaxf(mx, v);
+      }
+      float alpha = 1.0f;
+      bool rescale = false;
+      if (m_used == -INFINITY) m_used = mx;                                   // nothing accumulated for this row yet
+      else if (mx > m_used + TC_RESCALE) { alpha = exp2f(m_used - mx); m_used = mx; rescale = true; }
+      const float mu = m_used == -INFINITY ? 0.f : m_used;
+      float rs = 0.f;
+#pragma unroll
+      for (int j = 0; j < 64; ++j) { sc[j] = exp2f(sc[j] - mu); rs += sc[j]; }
+      l = l * alpha + rs;
+      if (i > 0) {
+        mbar_wait(smem_u32(&pv_done), (uint32_t)(i - 1) & 1u, aborted, p.status);   // P buffers free, O at rest
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, rescale)) {
+#pragma unroll 1
+          for (int c0 = 0; c0 < DH; c0 += 16) {
+            uint32_t r[16];
+            tmem_ld16(tmem + lane_base + 128u + (uint32_t)c0, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
+            tmem_st16(tmem + lane_base + 128u + (uint32_t)c0, r);
+          }
+          tmem_st_wait();
+        }
+      }
+      if (key0 + TILE > kv_total) {
+        // last, partial tile: rows past the end may hold anything (stale pool memory); zero V there so
+        // that a zero probability times a non-finite value cannot poison the sum.  The tile has
+        // landed: its scores were computed from it.
+        const int first_bad = kv_total - key0;
+        uint8_t* vgen = smem_gen + (size_t)(i % STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
+        for (int idx = threadIdx.x - 64; idx < (TILE - first_bad) * 16; idx += 128) {
+          const int r = first_bad + (idx >> 4), c = idx & 15;
+          *reinterpret_cast<uint4*>(vgen + (size_t)(c >> 3) * 8192 + r * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
+        }
+      }
+      // probabilities as two bf16 terms, eight keys (16 bytes) per store
+      uint8_t* ph = smem_gen + (ph_base - smem_base) + (uint32_t)row * 128u;
+      uint8_t* pl = smem_gen + (pl_base - smem_base) + (uint32_t)row * 128u;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        uint32_t hi[4], lo[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float p0 = sc[c * 8 + 2 * e], p1 = sc[c * 8 + 2 * e + 1];
+          __nv_bfloat162 hb = __floats2bfloat162_rn(p0, p1);
+          float2 hf = __bfloat1622float2(hb);
+          hi[e] = *reinterpret_cast<uint32_t*>(&hb);
+          lo[e] = pack_bf16(p0 - hf.x, p1 - hf.y);
+        }
+        const uint32_t off = (uint32_t)((c ^ (row & 7)) << 4);
+        *reinterpret_cast<uint4*>(ph + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4*>(pl + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+      }
+      proxy_fence();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&p_ready));
+    }
+    // ---- this CTA's (m, l, O) rows into shared memory ----
+    if (T > 0) {
+      mbar_wait(smem_u32(&pv_done), (uint32_t)(T - 1) & 1u, aborted, p.status);
+      tc_fence_after();
+    }
+    compute_bar(128);                               // every MMA has retired: the stage ring can be reused
+    {
+      float* mr = mrg + (size_t)row * ROWF;
+#pragma unroll 1
+      for (int c0 = 0; c0 < DH; c0 += 16) {
+        uint32_t r[16];
+        if (T > 0) {
+          tmem_ld16(tmem + lane_base + 128u + (uint32_t)c0, r);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) r[j] = 0u;
+        }
+#pragma unroll
+        for (int j = 0; j < 16; j += 4)
+          *reinterpret_cast<float4*>(mr + c0 + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                                                __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+      }
+      mr[DH] = m_used;
+      mr[DH + 1] = l;
+    }
+    tc_fence_before();
+    compute_bar(128);
+
+    // ---- output: final, or partial + fixed-order merge by the last CTA of this (sequence, head) ----
+    const int ct = threadIdx.x - 64, nct = 128, RP = p.rows_pad;
+    const float LN2 = 0.6931471805599453f;
+    if (p.nsplit == 1) {
+      for (int idx = ct; idx < nq * (DH / 4); idx += nct) {
+        const int r = idx / (DH / 4), c4 = idx % (DH / 4);
+        const float inv = 1.0f / mrg[(size_t)r * ROWF + DH + 1];
+        const float4 v = *reinterpret_cast<const float4*>(mrg + (size_t)r * ROWF + c4 * 4);
+        *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.n + r) * p.H + h) * DH + c4 * 4) =
+            make_uint2(pack_bf16(v.x * inv, v.y * inv), pack_bf16(v.z * inv, v.w * inv));
+      }
+      if (p.lse)
+        for (int r = ct; r < nq; r += nct)
+          p.lse[((size_t)b * p.H + h) * p.n + r] = (mrg[(size_t)r * ROWF + DH] + log2f(mrg[(size_t)r * ROWF + DH + 1])) * LN2;
+    } else {
+      float* part = p.partial + (((size_t)b * p.H + h) * p.nsplit) * (size_t)(RP * ROWF);
+      float* mine = part + (size_t)split * (RP * ROWF);
+      for (int idx = ct; idx < nq * ROWF; idx += nct) __stcg(mine + idx, mrg[idx]);
+      __threadfence();
+      compute_bar(128);
+      if (ct == 0) ticket_s = atomicAdd(&p.counters[b * p.H + h], 1u);
+      compute_bar(128);
+      if (ticket_s == (unsigned)p.nsplit - 1) {
+        __threadfence();
+        float* wts = mrg;                                   // [nsplit][RP]
+        for (int r = ct; r < nq; r += nct) {
+          float M = -INFINITY;
+          for (int s2 = 0; s2 < p.nsplit; ++s2) M = fmaxf(M, __ldcg(part + (size_t)s2 * (RP * ROWF) + r * ROWF + DH));
+          float Lsum = 0.f;
+          for (int s2 = 0; s2 < p.nsplit; ++s2) {
+            const float* pr = part + (size_t)s2 * (RP * ROWF) + r * ROWF;
+            float w = exp2f(__ldcg(pr + DH) - M);
+            wts[s2 * RP + r] = w;
+            Lsum += __ldcg(pr + DH + 1) * w;
+          }
+          const float inv = 1.0f / Lsum;
+          for (int s2 = 0; s2 < p.nsplit; ++s2) wts[s2 * RP + r] *= inv;
+          if (p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
+        }
+        compute_bar(128);
+        for (int idx = ct; idx < nq * (DH / 4); idx += nct) {
+          const int r = idx / (DH / 4), c4 = idx % (DH / 4);
+          const float4* src = reinterpret_cast<const float4*>(part + (size_t)r * ROWF) + c4;
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+          for (int s2 = 0; s2 < p.nsplit; ++s2) {
+            const float4 v = __ldcg(src + (size_t)s2 * (RP * ROWF / 4));
+            const float w = wts[s2 * RP + r];
+            acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+          }
+          *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.n + r) * p.H + h) * DH + c4 * 4) =
+              make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+        }
+        if (ct == 0) p.counters[b * p.H + h] = 0u;          // ready for the next launch
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256u) : "memory");
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
 // fp32 path
 // ---------------------------------------------------------------------------------------------
 template <int DH>
@@ -481,10 +876,10 @@ __global__ void __launch_bounds__(128) tree_attn_f32_kernel(const float* __restr
 
 // A split reads `per` tiles of 64 keys and writes an n-row fp32 partial, so wide trees get fewer,
 // longer splits: at least n/8 tiles each keeps the partial traffic near one eighth of the K/V read.
-int plan_nsplit(int B, int H, int n, int max_len) {
+int plan_nsplit(int B, int H, int n, int max_len, int target_ctas) {
   int tiles = (max_len + TILE - 1) / TILE;
   if (tiles < 1) tiles = 1;
-  int want = (kTargetCtas + B * H - 1) / (B * H);
+  int want = (target_ctas + B * H - 1) / (B * H);
   int min_tiles = n / 8 > 1 ? n / 8 : 1;
   if (want > tiles / min_tiles) want = tiles / min_tiles;
   if (want > kMaxSplit) want = kMaxSplit;
@@ -552,13 +947,29 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
   p.n = a->n;
   p.H = a->n_heads;
   p.max_pages = a->max_pages;
-  p.nsplit = plan_nsplit(a->B, a->n_heads, nq_pad(a->n), a->max_len);
+  static const int legacy = getenv("CERB_ATTN_LEGACY") ? atoi(getenv("CERB_ATTN_LEGACY")) : 0;
+  static const int vswap = getenv("CERB_ATTN_VSWAP") ? atoi(getenv("CERB_ATTN_VSWAP")) : 0;
+  const bool tensor_path = a->head_dim == 128 && !legacy;
+  // the tensor-core kernel runs one CTA per SM, the warp-MMA kernel two
+  p.nsplit = plan_nsplit(a->B, a->n_heads, nq_pad(a->n), a->max_len, tensor_path ? 148 : kTargetCtas);
   if (p.nsplit < 1) return CERB_E_SHAPE;
   p.oob_row = a->n_pool_pages * a->n_heads * CERB_PAGE;
   p.scale_log2 = a->scale * 1.4426950408889634f;
+  p.rows_pad = nq_pad(a->n);
+  // V tile in shared memory: [half of head_dim][64 keys][128 bytes]; 8-key groups are 1024 bytes apart
+  p.v_lbo = vswap ? 1024u : 8192u;
+  p.v_sbo = vswap ? 8192u : 1024u;
   if (a->scratch_bytes < attn_scratch_bytes(a->B, a->n, a->n_heads, a->head_dim)) return CERB_E_NOMEM;
   int np = nq_pad(a->n), rc = CERB_E_SHAPE;
-  if (a->head_dim == 128) {
+  if (tensor_path) {
+    static bool configured = false;
+    if (!configured) {
+      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM));
+      configured = true;
+    }
+    rc = launch_pdl(tree_attn_tc_kernel, dim3(p.nsplit, p.H, a->B), dim3(192), TC_SMEM, st, *tmK, *tmV, p) == cudaSuccess
+             ? CERB_OK : CERB_E_CUDA;
+  } else if (a->head_dim == 128) {
     if (np == 16) rc = launch_cfg<128, 1, 4, 3>(p, tmK, tmV, a->B, st);
     else if (np == 32) rc = launch_cfg<128, 2, 4, 3>(p, tmK, tmV, a->B, st);
     else if (np == 64) rc = launch_cfg<128, 4, 2, 3>(p, tmK, tmV, a->B, st);
