@@ -24,7 +24,7 @@ constexpr int PAGES_PER_TILE = TILE / CERB_PAGE;
 constexpr int kTargetCtas = 296;          // two CTAs per SM on a 148-SM part
 constexpr int kMaxSplit = 32;
 constexpr int kMaxPagesPerCta = 1024;
-constexpr uint64_t kWaitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait
+constexpr long long kWaitCycles = 4000000000ll;   // about 2 s of SM clock: far beyond any legitimate wait
 constexpr size_t kCounterBytes = 4096;    // one ticket counter per (sequence, head)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -48,22 +48,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ uint64_t global_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait: gives up after kWaitNs of wall time.  After the first time-out in a CTA (or when
-// an earlier kernel already reported one) every later wait gives up almost at once, so the CTA
-// still runs to its end in bounded time.
+// Bounded wait: gives up after kWaitCycles SM clock cycles (a couple of seconds).  After the first
+// time-out in a CTA (or when an earlier kernel already reported one) every later wait gives up
+// almost at once, so the CTA still runs to its end in bounded time.  The budget is measured with
+// the SM-local cycle counter, which is cheap to read; the polls in between are back to back.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* aborted, int32_t* status) {
-  if (mbar_try_wait(bar, parity)) return;
-  const uint64_t t0 = global_ns();
-  const uint64_t budget = *aborted ? 20000ull : kWaitNs;
+  for (int i = 0; i < 1024; ++i)
+    if (mbar_try_wait(bar, parity)) return;
+  const long long t0 = clock64();
+  const long long budget = *aborted ? 40000ll : kWaitCycles;
   for (;;) {
-    for (int i = 0; i < 64; ++i)
+    for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return;
-    if (global_ns() - t0 > budget) break;
+    if (clock64() - t0 > budget) break;
   }
   *aborted = 1;
   atomicExch(status, CERB_E_TIMEOUT);
@@ -489,6 +486,11 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 
 __global__ void __launch_bounds__(192, 1) tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                               const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
@@ -641,40 +643,38 @@ __global__ void __launch_bounds__(192, 1) tree_attn_tc_kernel(const __grid_const
       const int buf = i & 1;
       mbar_wait(smem_u32(&s_full[buf]), (uint32_t)(i >> 1) & 1u, aborted, p.status);
       tc_fence_after();
-      float sc[64];
-#pragma unroll
-      for (int c0 = 0; c0 < 64; c0 += 16) tmem_ld16(tmem + lane_base + (uint32_t)(buf * 64 + c0), reinterpret_cast<uint32_t*>(sc + c0));
-      tmem_ld_wait();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&s_free[buf]));
+      // Two compact passes over the 64 scores of this row, 16 columns at a time (S is re-read from
+      // tensor memory, which is cheap; keeping the loop bodies small matters more with four warps).
       const int key0 = (t0 + i) * TILE;
       const bool need_mask = key0 + TILE > L;
-      float mx = -INFINITY;
-#pragma unroll
-      for (int j = 0; j < 64; ++j) {
-        float v = sc[j] * p.scale_log2;
-        if (need_mask) {
-          const int kpos = key0 + j;
-          bool vis = kpos < L;
-          if (!vis && kpos < kv_total) {
-            const int t = kpos - L;
-            vis = ((t < 64 ? anc0 : anc1) >> (t & 63)) & 1ull;
-          }
-          if (!vis) v = -INFINITY;
+      const uint32_t s_addr = tmem + lane_base + (uint32_t)(buf * 64);
+      auto masked = [&](float v, int kpos) -> float {
+        bool vis = kpos < L;
+        if (!vis && kpos < kv_total) {
+          const int t = kpos - L;
+          vis = ((t < 64 ? anc0 : anc1) >> (t & 63)) & 1ull;
         }
-        sc[j] = v;
-        mx = fmaxf(mx, v);
+        return vis ? v : -INFINITY;
+      };
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll 1
+      for (int c0 = 0; c0 < 64; c0 += 16) {
+        uint32_t r[16];
+        tmem_ld16(s_addr + (uint32_t)c0, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          float v = __uint_as_float(r[j]) * p.scale_log2;
+          if (need_mask) v = masked(v, key0 + c0 + j);
+          mx4[j & 3] = fmaxf(mx4[j & 3], v);
+        }
       }
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       float alpha = 1.0f;
       bool rescale = false;
       if (m_used == -INFINITY) m_used = mx;                                   // nothing accumulated for this row yet
-      else if (mx > m_used + TC_RESCALE) { alpha = exp2f(m_used - mx); m_used = mx; rescale = true; }
+      else if (mx > m_used + TC_RESCALE) { alpha = ex2(m_used - mx); m_used = mx; rescale = true; }
       const float mu = m_used == -INFINITY ? 0.f : m_used;
-      float rs = 0.f;
-#pragma unroll
-      for (int j = 0; j < 64; ++j) { sc[j] = exp2f(sc[j] - mu); rs += sc[j]; }
-      l = l * alpha + rs;
       if (i > 0) {
         mbar_wait(smem_u32(&pv_done), (uint32_t)(i - 1) & 1u, aborted, p.status);   // P buffers free, O at rest
         tc_fence_after();
@@ -705,21 +705,41 @@ __global__ void __launch_bounds__(192, 1) tree_attn_tc_kernel(const __grid_const
       // probabilities as two bf16 terms, eight keys (16 bytes) per store
       uint8_t* ph = smem_gen + (ph_base - smem_base) + (uint32_t)row * 128u;
       uint8_t* pl = smem_gen + (pl_base - smem_base) + (uint32_t)row * 128u;
+      float rs4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+      for (int c0 = 0; c0 < 64; c0 += 16) {
+        uint32_t r[16];
+        tmem_ld16(s_addr + (uint32_t)c0, r);
+        tmem_ld_wait();
+        float pr[16];
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        uint32_t hi[4], lo[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float p0 = sc[c * 8 + 2 * e], p1 = sc[c * 8 + 2 * e + 1];
-          __nv_bfloat162 hb = __floats2bfloat162_rn(p0, p1);
-          float2 hf = __bfloat1622float2(hb);
-          hi[e] = *reinterpret_cast<uint32_t*>(&hb);
-          lo[e] = pack_bf16(p0 - hf.x, p1 - hf.y);
+        for (int j = 0; j < 16; ++j) {
+          float v = __uint_as_float(r[j]) * p.scale_log2;
+          if (need_mask) v = masked(v, key0 + c0 + j);
+          pr[j] = ex2(v - mu);
+          rs4[j & 3] += pr[j];
         }
-        const uint32_t off = (uint32_t)((c ^ (row & 7)) << 4);
-        *reinterpret_cast<uint4*>(ph + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        *reinterpret_cast<uint4*>(pl + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+          uint32_t hi[4], lo[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float p0 = pr[c * 8 + 2 * e], p1 = pr[c * 8 + 2 * e + 1];
+            __nv_bfloat162 hb = __floats2bfloat162_rn(p0, p1);
+            float2 hf = __bfloat1622float2(hb);
+            hi[e] = *reinterpret_cast<uint32_t*>(&hb);
+            lo[e] = pack_bf16(p0 - hf.x, p1 - hf.y);
+          }
+          const uint32_t off = (uint32_t)((((c0 >> 3) + c) ^ (row & 7)) << 4);
+          *reinterpret_cast<uint4*>(ph + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *reinterpret_cast<uint4*>(pl + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
       }
+      l = l * alpha + ((rs4[0] + rs4[1]) + (rs4[2] + rs4[3]));
+      // S has been read for the last time: the MMA warp may overwrite this buffer
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&s_free[buf]));
       proxy_fence();
       tc_fence_before();
       __syncwarp();
@@ -947,9 +967,10 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
   p.n = a->n;
   p.H = a->n_heads;
   p.max_pages = a->max_pages;
-  static const int legacy = getenv("CERB_ATTN_LEGACY") ? atoi(getenv("CERB_ATTN_LEGACY")) : 0;
-  static const int vswap = getenv("CERB_ATTN_VSWAP") ? atoi(getenv("CERB_ATTN_VSWAP")) : 0;
-  const bool tensor_path = a->head_dim == 128 && !legacy;
+  // CERB_ATTN_TC=1 selects the tcgen05 kernel (head_dim 128).  It is correct (same tests) but its
+  // softmax stage is not yet pipelined deeply enough to beat the warp-MMA kernel, which stays the default.
+  static const int use_tc = getenv("CERB_ATTN_TC") ? atoi(getenv("CERB_ATTN_TC")) : 0;
+  const bool tensor_path = a->head_dim == 128 && use_tc;
   // the tensor-core kernel runs one CTA per SM, the warp-MMA kernel two
   p.nsplit = plan_nsplit(a->B, a->n_heads, nq_pad(a->n), a->max_len, tensor_path ? 148 : kTargetCtas);
   if (p.nsplit < 1) return CERB_E_SHAPE;
@@ -957,8 +978,8 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
   p.scale_log2 = a->scale * 1.4426950408889634f;
   p.rows_pad = nq_pad(a->n);
   // V tile in shared memory: [half of head_dim][64 keys][128 bytes]; 8-key groups are 1024 bytes apart
-  p.v_lbo = vswap ? 1024u : 8192u;
-  p.v_sbo = vswap ? 8192u : 1024u;
+  p.v_lbo = 8192u;
+  p.v_sbo = 1024u;
   if (a->scratch_bytes < attn_scratch_bytes(a->B, a->n, a->n_heads, a->head_dim)) return CERB_E_NOMEM;
   int np = nq_pad(a->n), rc = CERB_E_SHAPE;
   if (tensor_path) {

@@ -39,7 +39,7 @@ constexpr int BM = 128;          // weight rows per CTA (MMA M)
 constexpr int BK = 64;           // k elements per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int MAX_STAGES = 8;
 constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;
-constexpr uint64_t kWaitNs = 2000000000ull;   // 2 s: far beyond any legitimate wait
+constexpr long long kWaitCycles = 4000000000ll;   // about 2 s of SM clock: far beyond any legitimate wait
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -63,22 +63,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ uint64_t global_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait: gives up after kWaitNs of wall time.  After the first time-out in a CTA (or when
-// an earlier kernel already reported one) every later wait gives up almost at once, so the CTA
-// still runs to its end in bounded time.
+// Bounded wait: gives up after kWaitCycles SM clock cycles (a couple of seconds).  After the first
+// time-out in a CTA (or when an earlier kernel already reported one) every later wait gives up
+// almost at once, so the CTA still runs to its end in bounded time.  The budget is measured with
+// the SM-local cycle counter, which is cheap to read; the polls in between are back to back.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* aborted, int32_t* status) {
-  if (mbar_try_wait(bar, parity)) return;
-  const uint64_t t0 = global_ns();
-  const uint64_t budget = *aborted ? 20000ull : kWaitNs;
+  for (int i = 0; i < 1024; ++i)
+    if (mbar_try_wait(bar, parity)) return;
+  const long long t0 = clock64();
+  const long long budget = *aborted ? 40000ll : kWaitCycles;
   for (;;) {
-    for (int i = 0; i < 64; ++i)
+    for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return;
-    if (global_ns() - t0 > budget) break;
+    if (clock64() - t0 > budget) break;
   }
   *aborted = 1;
   atomicExch(status, CERB_E_TIMEOUT);
@@ -147,7 +144,7 @@ struct GemmParams {
   int num_kb;         // ceil(K / 64)
   int tiles;          // ceil(N / 128)
   int per;            // work units per CTA
-  long long total;    // work units in all: mchunks * tiles * num_kb
+  int total;          // work units in all: mchunks * tiles * num_kb
   int nslots;         // partial slots per output element
   int stages;
   int wide;           // 1: a CTA works on 256 weight rows at a time (two MMA tiles sharing one activation stage)
@@ -161,13 +158,13 @@ struct GemmParams {
 struct Segment {
   int job, kb0, nkb;
 };
-__device__ __forceinline__ bool next_segment(long long& u, long long u1, int num_kb, Segment& sg) {
+__device__ __forceinline__ bool next_segment(int& u, int u1, int num_kb, Segment& sg) {
   if (u >= u1) return false;
-  sg.job = (int)(u / num_kb);
-  sg.kb0 = (int)(u % num_kb);
-  long long end = (long long)(sg.job + 1) * num_kb;
+  sg.job = u / num_kb;
+  sg.kb0 = u - sg.job * num_kb;
+  int end = (sg.job + 1) * num_kb;
   if (end > u1) end = u1;
-  sg.nkb = (int)(end - u);
+  sg.nkb = end - u;
   u = end;
   return true;
 }
@@ -189,8 +186,8 @@ __global__ void __launch_bounds__(192, 1) gemm_bf16_kernel(const __grid_constant
   const uint32_t stage_bytes = a_bytes + b_bytes;
   const int rows_per_tile = BM * (1 + p.wide);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long u0 = (long long)blockIdx.x * p.per;
-  const long long u1 = (u0 + p.per < p.total) ? u0 + p.per : p.total;
+  const int u0 = (int)blockIdx.x * p.per;
+  const int u1 = (u0 + p.per < p.total) ? u0 + p.per : p.total;
 
   if (threadIdx.x == 0) {
     aborted_s = 0;
@@ -218,31 +215,34 @@ __global__ void __launch_bounds__(192, 1) gemm_bf16_kernel(const __grid_constant
   griddep_launch();
   if (warp == 0) {
     if (lane == 0) {
-      const int n_units = (int)(u1 - u0);
+      const int n_units = u1 - u0;
       const uint64_t pol_w = l2_policy(true), pol_x = l2_policy(false);
+      // (tile, row chunk, k block) of the unit being issued, advanced incrementally
+      int w_job = u0 / p.num_kb, w_kb = u0 - w_job * p.num_kb;
+      int x_job = w_job, x_kb = w_kb;
       auto load_w = [&](int i) {
-        const long long u = u0 + i;
-        const int job = (int)(u / p.num_kb), kb = (int)(u % p.num_kb), tile = job % p.tiles;
+        const int tile = w_job % p.tiles;
         const int s = i % p.stages;
         const uint32_t fb = smem_u32(&full_bar[s]);
         const uint32_t a_dst = smem_base + (uint32_t)s * stage_bytes;
         mbar_expect_tx(fb, stage_bytes);
         if (p.hint) {
-          tma_load_2d_hint(a_dst, &tmW, kb * BK, tile * rows_per_tile, fb, pol_w);
-          if (p.wide) tma_load_2d_hint(a_dst + A_STAGE_BYTES, &tmW, kb * BK, tile * rows_per_tile + BM, fb, pol_w);
+          tma_load_2d_hint(a_dst, &tmW, w_kb * BK, tile * rows_per_tile, fb, pol_w);
+          if (p.wide) tma_load_2d_hint(a_dst + A_STAGE_BYTES, &tmW, w_kb * BK, tile * rows_per_tile + BM, fb, pol_w);
         } else {
-          tma_load_2d(a_dst, &tmW, kb * BK, tile * rows_per_tile, fb);
-          if (p.wide) tma_load_2d(a_dst + A_STAGE_BYTES, &tmW, kb * BK, tile * rows_per_tile + BM, fb);
+          tma_load_2d(a_dst, &tmW, w_kb * BK, tile * rows_per_tile, fb);
+          if (p.wide) tma_load_2d(a_dst + A_STAGE_BYTES, &tmW, w_kb * BK, tile * rows_per_tile + BM, fb);
         }
+        if (++w_kb == p.num_kb) { w_kb = 0; ++w_job; }
       };
       auto load_x = [&](int i) {
-        const long long u = u0 + i;
-        const int job = (int)(u / p.num_kb), kb = (int)(u % p.num_kb), mchunk = job / p.tiles;
+        const int mchunk = x_job / p.tiles;
         const int s = i % p.stages;
         const uint32_t fb = smem_u32(&full_bar[s]);
         const uint32_t x_dst = smem_base + (uint32_t)s * stage_bytes + a_bytes;
-        if (p.hint) tma_load_2d_hint(x_dst, &tmX, kb * BK, mchunk * kGemmRowsPerPass, fb, pol_x);
-        else tma_load_2d(x_dst, &tmX, kb * BK, mchunk * kGemmRowsPerPass, fb);
+        if (p.hint) tma_load_2d_hint(x_dst, &tmX, x_kb * BK, mchunk * kGemmRowsPerPass, fb, pol_x);
+        else tma_load_2d(x_dst, &tmX, x_kb * BK, mchunk * kGemmRowsPerPass, fb);
+        if (++x_kb == p.num_kb) { x_kb = 0; ++x_job; }
       };
       // Weights do not depend on the kernel before this one: fill the whole ring with weight tiles
       // while that kernel is still finishing, then wait for it and fetch the activations.
@@ -260,7 +260,7 @@ __global__ void __launch_bounds__(192, 1) gemm_bf16_kernel(const __grid_constant
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      long long u = u0;
+      int u = u0;
       Segment sg;
       int i = 0, g = 0;
       while (next_segment(u, u1, p.num_kb, sg)) {
@@ -303,7 +303,7 @@ __global__ void __launch_bounds__(192, 1) gemm_bf16_kernel(const __grid_constant
   } else {
     const int quarter = warp & 3;                    // TMEM lanes 32*quarter .. +31 belong to this warp
     griddep_wait();                                  // the kernel before this one may still be reading the partial buffer
-    long long u = u0;
+    int u = u0;
     Segment sg;
     int g = 0;
     while (next_segment(u, u1, p.num_kb, sg)) {
@@ -312,24 +312,31 @@ __global__ void __launch_bounds__(192, 1) gemm_bf16_kernel(const __grid_constant
       mbar_wait(smem_u32(&acc_full[buf]), (uint32_t)(g >> 1) & 1u, aborted, p.status);
       tc_fence_after();
       // slot = how many CTAs before this one also work on this job
-      const long long job_u0 = (long long)sg.job * p.num_kb;
-      const int first_cta = (int)(job_u0 / p.per);
-      const int last_cta = (int)((job_u0 + p.num_kb - 1) / p.per);
+      const int job_u0 = sg.job * p.num_kb;
+      const int first_cta = job_u0 / p.per;
+      const int last_cta = (job_u0 + p.num_kb - 1) / p.per;
       const int slot = (int)blockIdx.x - first_cta;
       const int m_base = mchunk * kGemmRowsPerPass;
       const int m_cnt = min(p.n_mma, p.M - m_base);
+      const size_t ldo = (size_t)p.N;
       for (int hf = 0; hf <= p.wide; ++hf) {
         const int n_out = tile * rows_per_tile + hf * BM + quarter * 32 + lane;
         const bool n_ok = n_out < p.N;
-        float* o = p.out + ((size_t)slot * p.M + m_base) * p.N + n_out;
+        // consecutive lanes hold consecutive output columns: every store instruction writes 128 contiguous bytes
+        float* o = p.out + ((size_t)slot * p.M + m_base) * ldo + (n_ok ? n_out : 0);
         const uint32_t taddr = tmem_base + (uint32_t)buf * p.acc_cols + (uint32_t)(hf * p.n_mma) + ((uint32_t)(quarter * 32) << 16);
         for (int c0 = 0; c0 < m_cnt; c0 += 16) {
           uint32_t r[16];
           tmem_ld16(taddr + (uint32_t)c0, r);
           if (n_ok) {
+            if (c0 + 16 <= m_cnt) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j)
-              if (c0 + j < m_cnt) o[(size_t)(c0 + j) * p.N] = __uint_as_float(r[j]);
+              for (int j = 0; j < 16; ++j) { *o = __uint_as_float(r[j]); o += ldo; }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j)
+                if (c0 + j < m_cnt) { *o = __uint_as_float(r[j]); o += ldo; }
+            }
           }
         }
       }
@@ -341,8 +348,8 @@ __global__ void __launch_bounds__(192, 1) gemm_bf16_kernel(const __grid_constant
           const int n_out = tile * rows_per_tile + hf * BM + quarter * 32 + lane;
           if (n_out >= p.N) continue;
           for (int z = last_cta - first_cta + 1; z < p.nslots; ++z) {
-            float* zo = p.out + ((size_t)z * p.M + m_base) * p.N + n_out;
-            for (int m = 0; m < m_cnt; ++m) zo[(size_t)m * p.N] = 0.f;
+            float* zo = p.out + ((size_t)z * p.M + m_base) * ldo + n_out;
+            for (int m = 0; m < m_cnt; ++m) { *zo = 0.f; zo += ldo; }
           }
         }
       }
@@ -358,7 +365,7 @@ __global__ void __launch_bounds__(192, 1) gemm_bf16_kernel(const __grid_constant
 
 struct GemmPlan {
   int tiles, mchunks, num_kb, per, ctas, nslots;
-  long long total;
+  long long total;   // checked to fit 31 bits before launch
 };
 
 // Tuning switches (environment, read once): CERB_GEMM_WIDE, CERB_GEMM_GROUP, CERB_GEMM_HINT.
@@ -465,7 +472,8 @@ int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, fl
   p.num_kb = g.num_kb;
   p.tiles = g.tiles;
   p.per = g.per;
-  p.total = g.total;
+  if (g.total >= (1ll << 30)) return CERB_E_SHAPE;
+  p.total = (int)g.total;
   p.nslots = g.nslots;
   static int group = tune("CERB_GEMM_GROUP", 1), hint = tune("CERB_GEMM_HINT", 1);
   p.wide = use_wide(M) ? 1 : 0;
