@@ -23,7 +23,8 @@ def cb():
 
 
 @pytest.mark.parametrize("M,N,K", [(64, 256, 512), (1, 128, 64), (16, 688, 256), (64, 256, 688), (100, 1000, 1024),
-                                   (300, 384, 320), (64, 4096, 4096), (7, 130, 72)])
+                                   (300, 384, 320), (64, 4096, 4096), (7, 130, 72),
+                                   (2048, 640, 512), (1000, 11008, 256), (129, 256, 11008)])
 def test_gemm_bf16_matches_definition(cb, M, N, K):
     X = synth.normal(11, 1, (M, K), 1.0, dtype=torch.bfloat16, device="cuda")
     W = synth.normal(11, 2, (N, K), 0.05, dtype=torch.bfloat16, device="cuda")
@@ -97,6 +98,8 @@ ATTN_CASES = [
     (3, 64, 4, 64, [15, 16, 17], 5),    # head_dim 64, lengths around a page boundary
     (1, 64, 2, 128, [5000], 5),         # long context: many tiles per split
     (16, 16, 32, 128, [40] * 16, 3),    # more (sequence, head) pairs than CTAs wanted: no split
+    (16, 128, 2, 128, [8192 - 17 * i for i in range(16)], 6),   # sweep corner: batch 16, 128 nodes, 8K keys
+    (5, 32, 3, 128, [511, 512, 513, 2047, 1], 6),
 ]
 
 

@@ -246,6 +246,41 @@ def test_batch_of_two_ragged_prompts(cb):
     assert eng.device_status() == 0
 
 
+def test_batch_16_with_128_node_trees(cb):
+    """Sweep corner at small width: 16 ragged sequences, a 128-node tree (two ancestor words, 2048 rows
+    per forward), planted candidates; every sequence must emit its own auto-regressive continuation."""
+    ms = synth.tiny_shape("fp32")
+    rig = Rig(cb, ms, max_batch=16, max_tokens=400, max_nodes=128, topk=(10, 10, 10, 10))
+    B = 16
+    lens = [20 + 13 * b for b in range(B)]
+    prompts = [[int(t) for t in synth.make_prompt(ms.vocab, L, seq=30 + b)] for b, L in enumerate(lens)]
+    tok = torch.zeros(B, max(lens), dtype=torch.int32, device="cuda")
+    for b, p in enumerate(prompts):
+        tok[b, :len(p)] = torch.tensor(p, dtype=torch.int32)
+    eng = rig.eng
+    tree = synth.best_first_tree(128, rig.topk)
+    th = eng.tree(tree)
+    n_new = 8
+    truths = [orc.ar_greedy(rig.cmodel, rig.sh, p, n_new + 6)[0] for p in prompts]
+    eng.prefill(tok, lens)
+    outs = [[] for _ in range(B)]
+    best = 0
+    for step in range(n_new):
+        plant = torch.tensor([plant_tokens(tree, truths[b], len(outs[b]), 1 + (step + b) % 5) for b in range(B)],
+                             dtype=torch.int32, device="cuda")
+        eng.step(th, 1e9, plant)
+        torch.cuda.synchronize()
+        for b in range(B):
+            na = int(eng.h_n_accept[b])
+            best = max(best, na)
+            outs[b].extend(int(t) for t in eng.h_tokens[b, :na])
+    for b in range(B):
+        k = min(len(outs[b]), n_new + 6)
+        assert outs[b][:k] == truths[b][:k], b
+    assert best >= 4
+    assert eng.device_status() == 0
+
+
 def test_error_codes(cb):
     ms = synth.tiny_shape("fp32")
     rig = Rig(cb, ms, max_tokens=128)
