@@ -97,6 +97,31 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def init_dist():
+    """One process per GPU (replicas, no data-path collective).  NCCL when CUDA is there, gloo otherwise."""
+    import torch.distributed as dist
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    if torch.cuda.is_available():
+        dist.init_process_group("nccl", device_id=torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0))))
+    else:
+        dist.init_process_group("gloo")
+
+
+def max_over_ranks(value: float, world: int) -> float:
+    """The slowest rank's time: what the whole job waited for."""
+    if world <= 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device="cuda" if torch.cuda.is_available() else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t[0])
+
+
+def rank_prompt(vocab: int, prompt_len: int, rank: int) -> torch.Tensor:
+    """Every rank decodes its own sequence (weak scaling)."""
+    return synth.make_prompt(vocab, prompt_len, seq=rank).to(torch.int32)
+
+
 def percentile_threshold(values, q):
     """Threshold with a fraction q of the values at or below it (midpoint of neighbouring order statistics)."""
     s = sorted(values)
@@ -137,7 +162,7 @@ def run_cerb(args, rank, world):
     tree = synth.best_first_tree(n_nodes, topk)
     th = eng.tree(tree)
     # every rank decodes its own prompt (weak scaling: one sequence per GPU)
-    prompt = synth.make_prompt(ms.vocab, prompt_len, seq=rank).to(torch.int32)
+    prompt = rank_prompt(ms.vocab, prompt_len, rank)
     h_prompt = prompt.reshape(1, -1).contiguous().pin_memory()
     d_prompt = torch.empty_like(h_prompt, device="cuda")
 
@@ -212,12 +237,7 @@ def run_cerb(args, rank, world):
         out = decode(n_steps, **kw)
         e1.record()
         barrier()
-        ms_total = e0.elapsed_time(e1)
-        if world > 1:
-            import torch.distributed as dist
-            t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_total = float(t[0])
+        ms_total = max_over_ranks(e0.elapsed_time(e1), world)
         return ms_total, out, eng.launch_count() - l0
 
     # --- A: the headline run (device-resident inputs), natural acceptance
@@ -512,9 +532,7 @@ def main():
         run_kernel(args)
         return
     if world > 1:
-        import torch.distributed as dist
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=torch.device("cuda", int(os.environ.get("LOCAL_RANK", 0))))
+        init_dist()
     try:
         run_cerb(args, rank, world)
     finally:
