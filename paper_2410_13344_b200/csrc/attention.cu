@@ -65,6 +65,22 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatil
   *aborted = 1;
   atomicExch(status, CERB_E_TIMEOUT);
 }
+// Same bounded wait for a lane whose warp shares an issue port with busy warps: back off between polls.
+__device__ __forceinline__ void mbar_wait_polite(uint32_t bar, uint32_t parity, volatile int* aborted, int32_t* status) {
+  for (int i = 0; i < 4; ++i)
+    if (mbar_try_wait(bar, parity)) return;
+  const long long t0 = clock64();
+  const long long budget = *aborted ? 40000ll : kWaitCycles;
+  for (;;) {
+    for (int i = 0; i < 64; ++i) {
+      if (mbar_try_wait(bar, parity)) return;
+      __nanosleep(40);
+    }
+    if (clock64() - t0 > budget) break;
+  }
+  *aborted = 1;
+  atomicExch(status, CERB_E_TIMEOUT);
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -431,20 +447,25 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
 // but both products run as tcgen05 MMAs with their results in tensor memory:
 //   S[128 x 64]  = Q[128 x 128] . K_tile^T      (Q staged once in shared memory, zero rows past n)
 //   O[128 x 128] += P[128 x 64] . V_tile        (P = p_hi + p_lo, two bf16 terms, staged in shared memory)
-// Warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer, warps 2-5 = softmax: thread t owns
-// query row t (= TMEM lane t), reads its S row from TMEM, keeps the running maximum and sum in
-// registers, writes its P row (128-byte swizzled, the MMA's K-major A layout).  S is double-buffered
-// so the next tile's scores are computed while this tile's probabilities are formed.  O stays in
-// TMEM across tiles; it is only rescaled when a row's maximum grows by more than 2^8 (until then the
-// older maximum keeps being used, which is exact after the final normalisation).
+// Warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer, warps 2-5 and 6-9 = two softmax groups
+// that take alternate key tiles.  In a group thread t owns query row t (= TMEM lane t): it reads its
+// whole S row from tensor memory with back-to-back loads and ONE wait (a dependent TMEM round trip
+// costs ~600 cycles here, measured), keeps the running maximum and sum in registers and writes its P
+// row (128-byte swizzled, the MMA's K-major A layout).  Each group has its own S buffer, its own O
+// accumulator and its own P buffers, i.e. the two groups run two independent online-softmax streams
+// over the even and the odd tiles, merged once at the end; one group's TMEM latency and arithmetic
+// overlap the other's.  O stays in TMEM across tiles; it is only rescaled when a row's maximum grows
+// by more than 2^8 (until then the older maximum keeps being used, which is exact after the final
+// normalisation).
 namespace {
 
-constexpr int TC_STAGES = 4;
+constexpr int TC_STAGES = 3;
 constexpr uint32_t TC_KV_BYTES = 16384;               // K (or V) of one 64-key tile, two 64-wide halves
 constexpr uint32_t TC_STAGE_BYTES = 2 * TC_KV_BYTES;
-constexpr uint32_t TC_Q_BYTES = 32768, TC_P_BYTES = 16384;
-constexpr size_t TC_SMEM = (size_t)TC_STAGES * TC_STAGE_BYTES + TC_Q_BYTES + 2 * TC_P_BYTES + 1024;
+constexpr uint32_t TC_Q_BYTES = 32768, TC_P_BYTES = 16384;   // P: one term (hi or lo) of one softmax group
+constexpr size_t TC_SMEM = (size_t)TC_STAGES * TC_STAGE_BYTES + TC_Q_BYTES + 4 * TC_P_BYTES + 1024;
 constexpr int TC_DH = 128, TC_ROWF = TC_DH + 4;
+constexpr int TC_THREADS = 320;                       // producer warp, MMA warp, two softmax groups of four warps
 constexpr float TC_RESCALE = 8.0f;                    // log2 of the growth of a row maximum that forces a rescale
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -492,11 +513,11 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-__global__ void __launch_bounds__(192, 1) tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK,
-                                                              const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+__global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK,
+                                                                     const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
   constexpr int DH = TC_DH, ROWF = TC_ROWF, STAGES = TC_STAGES;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], s_full[2], s_free[2], q_ready, p_ready, pv_done;
+  __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], s_full[2], s_free[2], p_ready[2], pv_done[2], q_ready;
   __shared__ int page_list[kMaxPagesPerCta];
   __shared__ uint32_t tmem_slot;
   __shared__ int aborted_s;
@@ -507,7 +528,8 @@ __global__ void __launch_bounds__(192, 1) tree_attn_tc_kernel(const __grid_const
   griddep_launch();
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t q_base = smem_base + STAGES * TC_STAGE_BYTES, ph_base = q_base + TC_Q_BYTES, pl_base = ph_base + TC_P_BYTES;
+  const uint32_t q_base = smem_base + STAGES * TC_STAGE_BYTES;
+  const uint32_t p_base = q_base + TC_Q_BYTES;          // [group][hi, lo] x 16 KB
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int L = p.len[b];
@@ -526,26 +548,27 @@ __global__ void __launch_bounds__(192, 1) tree_attn_tc_kernel(const __grid_const
       mbar_init(smem_u32(&full_bar[s]), 1);
       mbar_init(smem_u32(&empty_bar[s]), 1);
     }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(smem_u32(&s_full[i]), 1);
-      mbar_init(smem_u32(&s_free[i]), 4);
+    for (int g = 0; g < 2; ++g) {
+      mbar_init(smem_u32(&s_full[g]), 1);
+      mbar_init(smem_u32(&s_free[g]), 4);
+      mbar_init(smem_u32(&p_ready[g]), 4);
+      mbar_init(smem_u32(&pv_done[g]), 1);
     }
     mbar_init(smem_u32(&q_ready), 4);
-    mbar_init(smem_u32(&p_ready), 4);
-    mbar_init(smem_u32(&pv_done), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     if (too_long) atomicExch(p.status, CERB_E_SHAPE);
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(256u)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(512u)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = tmem_slot;                 // columns 0-63 / 64-127: S buffers, 128-255: O
-  float* mrg = reinterpret_cast<float*>(smem_gen); // [128][ROWF] in the stage ring, once the key loop is over
+  // tensor memory: columns 0-63 / 64-127 = S of group 0 / 1, 128-255 / 256-383 = O of group 0 / 1
+  const uint32_t tmem = tmem_slot;
+  float* mrg = reinterpret_cast<float*>(smem_gen);   // [2][128][ROWF] over the whole buffer, once the key loop is over
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -559,7 +582,7 @@ __global__ void __launch_bounds__(192, 1) tree_attn_tc_kernel(const __grid_const
     if (lane == 0) {
       for (int i = 0; i < T; ++i) {
         const int s = i % STAGES;
-        mbar_wait(smem_u32(&empty_bar[s]), ((uint32_t)(i / STAGES) & 1u) ^ 1u, aborted, p.status);
+        mbar_wait_polite(smem_u32(&empty_bar[s]), ((uint32_t)(i / STAGES) & 1u) ^ 1u, aborted, p.status);
         const uint32_t fb = smem_u32(&full_bar[s]);
         mbar_expect_tx(fb, TC_STAGE_BYTES);
         const uint32_t kdst = smem_base + (uint32_t)s * TC_STAGE_BYTES, vdst = kdst + TC_KV_BYTES;
@@ -579,51 +602,51 @@ __global__ void __launch_bounds__(192, 1) tree_attn_tc_kernel(const __grid_const
     // ---------------- MMA issuer ----------------
     if (lane == 0 && T > 0) {
       const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
-      const uint32_t idesc_pv = idesc_s | (1u << 16);            // B operand (V) is MN-major
-      auto issue_s = [&](int i) {
-        const uint32_t kb = smem_base + (uint32_t)(i % STAGES) * TC_STAGE_BYTES;
-        const uint32_t d = tmem + (uint32_t)(i & 1) * 64u;
+      // PV: B operand (V) is MN-major, N = 128 (two 64-wide swizzle atoms, p.v_lbo bytes apart)
+      const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+      const uint64_t q_desc0 = desc_k_sw128(q_base), q_desc1 = desc_k_sw128(q_base + 16384u);
+      auto issue_pv = [&](int j) {
+        const int g = j & 1, k = j >> 1;
+        mbar_wait(smem_u32(&p_ready[g]), (uint32_t)k & 1u, aborted, p.status);
+        tc_fence_after();
+        const uint32_t vb = smem_base + (uint32_t)(j % STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
+        const uint32_t d = tmem + 128u + (uint32_t)g * 128u;
+        const uint64_t ph = desc_k_sw128(p_base + (uint32_t)g * 2u * TC_P_BYTES), pl = desc_k_sw128(p_base + (uint32_t)g * 2u * TC_P_BYTES + TC_P_BYTES);
 #pragma unroll
-        for (int hf = 0; hf < 2; ++hf)
-#pragma unroll
-          for (int kk = 0; kk < 4; ++kk)
-            umma(d, desc_k_sw128(q_base + hf * 16384u) + (uint64_t)(kk * 2), desc_k_sw128(kb + hf * 8192u) + (uint64_t)(kk * 2),
-                 idesc_s, (hf | kk) ? 1u : 0u);
-        umma_commit(smem_u32(&s_full[i & 1]));
+        for (int ks = 0; ks < 4; ++ks) {
+          const uint64_t vd = desc_mn_sw128(vb + ks * 2048u, p.v_lbo, p.v_sbo);
+          umma(d, ph + (uint64_t)(ks * 2), vd, idesc_pv, (k == 0 && ks == 0) ? 0u : 1u);
+          umma(d, pl + (uint64_t)(ks * 2), vd, idesc_pv, 1u);
+        }
+        umma_commit(smem_u32(&empty_bar[j % STAGES]));   // K and V of this tile are no longer needed
+        umma_commit(smem_u32(&pv_done[g]));
       };
       mbar_wait(smem_u32(&q_ready), 0, aborted, p.status);
-      mbar_wait(smem_u32(&full_bar[0]), 0, aborted, p.status);
-      tc_fence_after();
-      issue_s(0);
       for (int i = 0; i < T; ++i) {
-        if (i + 1 < T) {
-          const int j = i + 1;
-          mbar_wait(smem_u32(&full_bar[j % STAGES]), (uint32_t)(j / STAGES) & 1u, aborted, p.status);
-          mbar_wait(smem_u32(&s_free[j & 1]), ((uint32_t)(j >> 1) & 1u) ^ 1u, aborted, p.status);
-          tc_fence_after();
-          issue_s(j);
-        }
-        mbar_wait(smem_u32(&p_ready), (uint32_t)i & 1u, aborted, p.status);
+        const int g = i & 1, k = i >> 1;
+        mbar_wait(smem_u32(&full_bar[i % STAGES]), (uint32_t)(i / STAGES) & 1u, aborted, p.status);
+        mbar_wait(smem_u32(&s_free[g]), ((uint32_t)k & 1u) ^ 1u, aborted, p.status);
         tc_fence_after();
-        const uint32_t vb = smem_base + (uint32_t)(i % STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
+        const uint32_t kb = smem_base + (uint32_t)(i % STAGES) * TC_STAGE_BYTES;
+        const uint64_t k_desc0 = desc_k_sw128(kb), k_desc1 = desc_k_sw128(kb + 8192u);
+        const uint32_t d = tmem + (uint32_t)g * 64u;
 #pragma unroll
-        for (int hf = 0; hf < 2; ++hf)
+        for (int kk = 0; kk < 4; ++kk) umma(d, q_desc0 + (uint64_t)(kk * 2), k_desc0 + (uint64_t)(kk * 2), idesc_s, kk ? 1u : 0u);
 #pragma unroll
-          for (int term = 0; term < 2; ++term)
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks)
-              umma(tmem + 128u + hf * 64u, desc_k_sw128(term ? pl_base : ph_base) + (uint64_t)(ks * 2),
-                   desc_mn_sw128(vb + hf * 8192u + ks * 2048u, p.v_lbo, p.v_sbo), idesc_pv, (i == 0 && term == 0 && ks == 0) ? 0u : 1u);
-        umma_commit(smem_u32(&empty_bar[i % STAGES]));   // K and V of this tile are no longer needed
-        umma_commit(smem_u32(&pv_done));
+        for (int kk = 0; kk < 4; ++kk) umma(d, q_desc1 + (uint64_t)(kk * 2), k_desc1 + (uint64_t)(kk * 2), idesc_s, 1u);
+        umma_commit(smem_u32(&s_full[g]));
+        if (i >= 1) issue_pv(i - 1);
       }
+      issue_pv(T - 1);
     }
   } else {
-    // ---------------- softmax warps: thread <-> query row ----------------
-    const int row = (warp & 3) * 32 + lane;
+    // ---------------- softmax groups: thread <-> query row, group g takes tiles g, g+2, ... ----------------
+    const int g = (warp - 2) >> 2;
+    const int gt = (int)threadIdx.x - 64 - g * 128;           // thread index inside the group
+    const int row = (warp & 3) * 32 + lane;                    // = TMEM lane
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const bool valid = row < nq;
-    {
+    if (g == 0) {
       // stage this row of Q (zeros past the last node) in the swizzled K-major layout
       const uint4* src = reinterpret_cast<const uint4*>(p.q + (((size_t)b * p.n + (valid ? row : 0)) * p.H + h) * DH);
 #pragma unroll
@@ -638,35 +661,41 @@ __global__ void __launch_bounds__(192, 1) tree_attn_tc_kernel(const __grid_const
     }
     uint64_t anc0 = 0, anc1 = 0;
     if (valid) { anc0 = p.anc[row * 2]; anc1 = p.anc[row * 2 + 1]; }
+    const uint32_t s_addr = tmem + lane_base + (uint32_t)g * 64u;
+    const uint32_t o_addr = tmem + lane_base + 128u + (uint32_t)g * 128u;
+    uint8_t* ph = smem_gen + (p_base - smem_base) + (uint32_t)g * 2u * TC_P_BYTES + (uint32_t)row * 128u;
+    uint8_t* pl = ph + TC_P_BYTES;
     float m_used = -INFINITY, l = 0.f;
-    for (int i = 0; i < T; ++i) {
-      const int buf = i & 1;
-      mbar_wait(smem_u32(&s_full[buf]), (uint32_t)(i >> 1) & 1u, aborted, p.status);
+    int k = 0;
+    for (int i = g; i < T; i += 2, ++k) {
+      mbar_wait(smem_u32(&s_full[g]), (uint32_t)k & 1u, aborted, p.status);
       tc_fence_after();
-      // Two compact passes over the 64 scores of this row, 16 columns at a time (S is re-read from
-      // tensor memory, which is cheap; keeping the loop bodies small matters more with four warps).
-      const int key0 = (t0 + i) * TILE;
-      const bool need_mask = key0 + TILE > L;
-      const uint32_t s_addr = tmem + lane_base + (uint32_t)(buf * 64);
-      auto masked = [&](float v, int kpos) -> float {
-        bool vis = kpos < L;
-        if (!vis && kpos < kv_total) {
-          const int t = kpos - L;
-          vis = ((t < 64 ? anc0 : anc1) >> (t & 63)) & 1ull;
-        }
-        return vis ? v : -INFINITY;
-      };
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll 1
-      for (int c0 = 0; c0 < 64; c0 += 16) {
-        uint32_t r[16];
-        tmem_ld16(s_addr + (uint32_t)c0, r);
-        tmem_ld_wait();
+      float sc[64];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          float v = __uint_as_float(r[j]) * p.scale_log2;
-          if (need_mask) v = masked(v, key0 + c0 + j);
-          mx4[j & 3] = fmaxf(mx4[j & 3], v);
+      for (int c0 = 0; c0 < 64; c0 += 16) tmem_ld16(s_addr + (uint32_t)c0, reinterpret_cast<uint32_t*>(sc + c0));
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&s_free[g]));       // S is in registers: its buffer may be overwritten
+      const int key0 = (t0 + i) * TILE;
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      if (key0 + TILE > L) {
+#pragma unroll
+        for (int j = 0; j < 64; ++j) {
+          const int kpos = key0 + j;
+          bool vis = kpos < L;
+          if (!vis && kpos < kv_total) {
+            const int t = kpos - L;
+            vis = ((t < 64 ? anc0 : anc1) >> (t & 63)) & 1ull;
+          }
+          sc[j] = vis ? sc[j] * p.scale_log2 : -INFINITY;
+          mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 64; ++j) {
+          sc[j] *= p.scale_log2;
+          mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
         }
       }
       const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
@@ -675,18 +704,24 @@ __global__ void __launch_bounds__(192, 1) tree_attn_tc_kernel(const __grid_const
       if (m_used == -INFINITY) m_used = mx;                                   // nothing accumulated for this row yet
       else if (mx > m_used + TC_RESCALE) { alpha = ex2(m_used - mx); m_used = mx; rescale = true; }
       const float mu = m_used == -INFINITY ? 0.f : m_used;
-      if (i > 0) {
-        mbar_wait(smem_u32(&pv_done), (uint32_t)(i - 1) & 1u, aborted, p.status);   // P buffers free, O at rest
+      float rs4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int j = 0; j < 64; ++j) { sc[j] = ex2(sc[j] - mu); rs4[j & 3] += sc[j]; }
+      l = l * alpha + ((rs4[0] + rs4[1]) + (rs4[2] + rs4[3]));
+      if (k > 0) {
+        mbar_wait(smem_u32(&pv_done[g]), (uint32_t)(k - 1) & 1u, aborted, p.status);   // P buffers free, O at rest
         tc_fence_after();
         if (__any_sync(0xffffffffu, rescale)) {
 #pragma unroll 1
-          for (int c0 = 0; c0 < DH; c0 += 16) {
-            uint32_t r[16];
-            tmem_ld16(tmem + lane_base + 128u + (uint32_t)c0, r);
+          for (int c0 = 0; c0 < DH; c0 += 32) {
+            uint32_t r[32];
+            tmem_ld16(o_addr + (uint32_t)c0, r);
+            tmem_ld16(o_addr + (uint32_t)c0 + 16u, r + 16);
             tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 16; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
-            tmem_st16(tmem + lane_base + 128u + (uint32_t)c0, r);
+            for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
+            tmem_st16(o_addr + (uint32_t)c0, r);
+            tmem_st16(o_addr + (uint32_t)c0 + 16u, r + 16);
           }
           tmem_st_wait();
         }
@@ -697,74 +732,53 @@ __global__ void __launch_bounds__(192, 1) tree_attn_tc_kernel(const __grid_const
         // landed: its scores were computed from it.
         const int first_bad = kv_total - key0;
         uint8_t* vgen = smem_gen + (size_t)(i % STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
-        for (int idx = threadIdx.x - 64; idx < (TILE - first_bad) * 16; idx += 128) {
+        for (int idx = gt; idx < (TILE - first_bad) * 16; idx += 128) {
           const int r = first_bad + (idx >> 4), c = idx & 15;
           *reinterpret_cast<uint4*>(vgen + (size_t)(c >> 3) * 8192 + r * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
         }
       }
       // probabilities as two bf16 terms, eight keys (16 bytes) per store
-      uint8_t* ph = smem_gen + (ph_base - smem_base) + (uint32_t)row * 128u;
-      uint8_t* pl = smem_gen + (pl_base - smem_base) + (uint32_t)row * 128u;
-      float rs4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 1
-      for (int c0 = 0; c0 < 64; c0 += 16) {
-        uint32_t r[16];
-        tmem_ld16(s_addr + (uint32_t)c0, r);
-        tmem_ld_wait();
-        float pr[16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          float v = __uint_as_float(r[j]) * p.scale_log2;
-          if (need_mask) v = masked(v, key0 + c0 + j);
-          pr[j] = ex2(v - mu);
-          rs4[j & 3] += pr[j];
+      for (int c = 0; c < 8; ++c) {
+        uint32_t hi[4], lo[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float p0 = sc[c * 8 + 2 * e], p1 = sc[c * 8 + 2 * e + 1];
+          __nv_bfloat162 hb = __floats2bfloat162_rn(p0, p1);
+          float2 hf = __bfloat1622float2(hb);
+          hi[e] = *reinterpret_cast<uint32_t*>(&hb);
+          lo[e] = pack_bf16(p0 - hf.x, p1 - hf.y);
         }
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t hi[4], lo[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float p0 = pr[c * 8 + 2 * e], p1 = pr[c * 8 + 2 * e + 1];
-            __nv_bfloat162 hb = __floats2bfloat162_rn(p0, p1);
-            float2 hf = __bfloat1622float2(hb);
-            hi[e] = *reinterpret_cast<uint32_t*>(&hb);
-            lo[e] = pack_bf16(p0 - hf.x, p1 - hf.y);
-          }
-          const uint32_t off = (uint32_t)((((c0 >> 3) + c) ^ (row & 7)) << 4);
-          *reinterpret_cast<uint4*>(ph + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-          *reinterpret_cast<uint4*>(pl + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-        }
+        const uint32_t off = (uint32_t)((c ^ (row & 7)) << 4);
+        *reinterpret_cast<uint4*>(ph + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4*>(pl + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
       }
-      l = l * alpha + ((rs4[0] + rs4[1]) + (rs4[2] + rs4[3]));
-      // S has been read for the last time: the MMA warp may overwrite this buffer
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&s_free[buf]));
       proxy_fence();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&p_ready));
+      if (lane == 0) mbar_arrive(smem_u32(&p_ready[g]));
     }
-    // ---- this CTA's (m, l, O) rows into shared memory ----
-    if (T > 0) {
-      mbar_wait(smem_u32(&pv_done), (uint32_t)(T - 1) & 1u, aborted, p.status);
+    // ---- this group's (m, l, O) rows into shared memory ----
+    if (k > 0) {
+      mbar_wait(smem_u32(&pv_done[g]), (uint32_t)(k - 1) & 1u, aborted, p.status);
       tc_fence_after();
     }
-    compute_bar(128);                               // every MMA has retired: the stage ring can be reused
+    compute_bar(256);                               // every MMA has retired: all of shared memory can be reused
     {
-      float* mr = mrg + (size_t)row * ROWF;
+      float* mr = mrg + ((size_t)g * 128 + row) * ROWF;
 #pragma unroll 1
-      for (int c0 = 0; c0 < DH; c0 += 16) {
-        uint32_t r[16];
-        if (T > 0) {
-          tmem_ld16(tmem + lane_base + 128u + (uint32_t)c0, r);
+      for (int c0 = 0; c0 < DH; c0 += 32) {
+        uint32_t r[32];
+        if (k > 0) {
+          tmem_ld16(o_addr + (uint32_t)c0, r);
+          tmem_ld16(o_addr + (uint32_t)c0 + 16u, r + 16);
           tmem_ld_wait();
         } else {
 #pragma unroll
-          for (int j = 0; j < 16; ++j) r[j] = 0u;
+          for (int j = 0; j < 32; ++j) r[j] = 0u;
         }
 #pragma unroll
-        for (int j = 0; j < 16; j += 4)
+        for (int j = 0; j < 32; j += 4)
           *reinterpret_cast<float4*>(mr + c0 + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
                                                                 __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
       }
@@ -772,10 +786,28 @@ __global__ void __launch_bounds__(192, 1) tree_attn_tc_kernel(const __grid_const
       mr[DH + 1] = l;
     }
     tc_fence_before();
-    compute_bar(128);
+    compute_bar(256);
+    if (g == 0) {
+      // merge the two groups' streams, row by row, into group 0's rows
+      float* ra = mrg + (size_t)row * ROWF;
+      const float* rb = mrg + ((size_t)128 + row) * ROWF;
+      const float ma = ra[DH], mb = rb[DH];
+      const float M = fmaxf(ma, mb), u = M == -INFINITY ? 0.f : M;
+      const float wa = ex2(ma - u), wb = ex2(mb - u);
+#pragma unroll 4
+      for (int c = 0; c < DH; c += 4) {
+        float4 a = *reinterpret_cast<float4*>(ra + c);
+        const float4 bb = *reinterpret_cast<const float4*>(rb + c);
+        a.x = a.x * wa + bb.x * wb; a.y = a.y * wa + bb.y * wb; a.z = a.z * wa + bb.z * wb; a.w = a.w * wa + bb.w * wb;
+        *reinterpret_cast<float4*>(ra + c) = a;
+      }
+      ra[DH] = M;
+      ra[DH + 1] = ra[DH + 1] * wa + rb[DH + 1] * wb;
+    }
+    compute_bar(256);
 
     // ---- output: final, or partial + fixed-order merge by the last CTA of this (sequence, head) ----
-    const int ct = threadIdx.x - 64, nct = 128, RP = p.rows_pad;
+    const int ct = threadIdx.x - 64, nct = 256, RP = p.rows_pad;
     const float LN2 = 0.6931471805599453f;
     if (p.nsplit == 1) {
       for (int idx = ct; idx < nq * (DH / 4); idx += nct) {
@@ -793,9 +825,9 @@ __global__ void __launch_bounds__(192, 1) tree_attn_tc_kernel(const __grid_const
       float* mine = part + (size_t)split * (RP * ROWF);
       for (int idx = ct; idx < nq * ROWF; idx += nct) __stcg(mine + idx, mrg[idx]);
       __threadfence();
-      compute_bar(128);
+      compute_bar(256);
       if (ct == 0) ticket_s = atomicAdd(&p.counters[b * p.H + h], 1u);
-      compute_bar(128);
+      compute_bar(256);
       if (ticket_s == (unsigned)p.nsplit - 1) {
         __threadfence();
         float* wts = mrg;                                   // [nsplit][RP]
@@ -813,7 +845,7 @@ __global__ void __launch_bounds__(192, 1) tree_attn_tc_kernel(const __grid_const
           for (int s2 = 0; s2 < p.nsplit; ++s2) wts[s2 * RP + r] *= inv;
           if (p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
         }
-        compute_bar(128);
+        compute_bar(256);
         for (int idx = ct; idx < nq * (DH / 4); idx += nct) {
           const int r = idx / (DH / 4), c4 = idx % (DH / 4);
           const float4* src = reinterpret_cast<const float4*>(part + (size_t)r * ROWF) + c4;
@@ -833,7 +865,7 @@ __global__ void __launch_bounds__(192, 1) tree_attn_tc_kernel(const __grid_const
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256u) : "memory");
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
 }
 
 }  // namespace
@@ -988,7 +1020,7 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
       CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM));
       configured = true;
     }
-    rc = launch_pdl(tree_attn_tc_kernel, dim3(p.nsplit, p.H, a->B), dim3(192), TC_SMEM, st, *tmK, *tmV, p) == cudaSuccess
+    rc = launch_pdl(tree_attn_tc_kernel, dim3(p.nsplit, p.H, a->B), dim3(TC_THREADS), TC_SMEM, st, *tmK, *tmV, p) == cudaSuccess
              ? CERB_OK : CERB_E_CUDA;
   } else if (a->head_dim == 128) {
     if (np == 16) rc = launch_cfg<128, 1, 4, 3>(p, tmK, tmV, a->B, st);
