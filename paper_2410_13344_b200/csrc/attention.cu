@@ -465,7 +465,7 @@ constexpr uint32_t TC_STAGE_BYTES = 2 * TC_KV_BYTES;
 constexpr uint32_t TC_Q_BYTES = 32768, TC_P_BYTES = 16384;   // P: one term (hi or lo) of one softmax group
 constexpr size_t TC_SMEM = (size_t)TC_STAGES * TC_STAGE_BYTES + TC_Q_BYTES + 4 * TC_P_BYTES + 1024;
 constexpr int TC_DH = 128, TC_ROWF = TC_DH + 4;
-constexpr int TC_THREADS = 320;                       // producer warp, MMA warp, two softmax groups of four warps
+constexpr int TC_THREADS = 352;                       // producer, QK^T issuer, two softmax groups of four warps, PV issuer
 constexpr float TC_RESCALE = 8.0f;                    // log2 of the growth of a row maximum that forces a rescale
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -599,28 +599,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
+    // ---------------- QK^T issuer ----------------
+    // (issuing one tcgen05.mma costs this thread ~95 cycles whatever its size, measured, so the two
+    // products are issued by two different warps)
     if (lane == 0 && T > 0) {
       const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
-      // PV: B operand (V) is MN-major, N = 128 (two 64-wide swizzle atoms, p.v_lbo bytes apart)
-      const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
       const uint64_t q_desc0 = desc_k_sw128(q_base), q_desc1 = desc_k_sw128(q_base + 16384u);
-      auto issue_pv = [&](int j) {
-        const int g = j & 1, k = j >> 1;
-        mbar_wait(smem_u32(&p_ready[g]), (uint32_t)k & 1u, aborted, p.status);
-        tc_fence_after();
-        const uint32_t vb = smem_base + (uint32_t)(j % STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
-        const uint32_t d = tmem + 128u + (uint32_t)g * 128u;
-        const uint64_t ph = desc_k_sw128(p_base + (uint32_t)g * 2u * TC_P_BYTES), pl = desc_k_sw128(p_base + (uint32_t)g * 2u * TC_P_BYTES + TC_P_BYTES);
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-          const uint64_t vd = desc_mn_sw128(vb + ks * 2048u, p.v_lbo, p.v_sbo);
-          umma(d, ph + (uint64_t)(ks * 2), vd, idesc_pv, (k == 0 && ks == 0) ? 0u : 1u);
-          umma(d, pl + (uint64_t)(ks * 2), vd, idesc_pv, 1u);
-        }
-        umma_commit(smem_u32(&empty_bar[j % STAGES]));   // K and V of this tile are no longer needed
-        umma_commit(smem_u32(&pv_done[g]));
-      };
       mbar_wait(smem_u32(&q_ready), 0, aborted, p.status);
       for (int i = 0; i < T; ++i) {
         const int g = i & 1, k = i >> 1;
@@ -635,9 +619,31 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) umma(d, q_desc1 + (uint64_t)(kk * 2), k_desc1 + (uint64_t)(kk * 2), idesc_s, 1u);
         umma_commit(smem_u32(&s_full[g]));
-        if (i >= 1) issue_pv(i - 1);
       }
-      issue_pv(T - 1);
+    }
+  } else if (warp == 10) {
+    // ---------------- PV issuer ----------------
+    if (lane == 0) {
+      // B operand (V) is MN-major, N = 128 (two 64-wide swizzle atoms, p.v_lbo bytes apart)
+      const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+      for (int j = 0; j < T; ++j) {
+        const int g = j & 1, k = j >> 1;
+        mbar_wait(smem_u32(&p_ready[g]), (uint32_t)k & 1u, aborted, p.status);
+        tc_fence_after();
+        const uint32_t vb = smem_base + (uint32_t)(j % STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
+        const uint32_t d = tmem + 128u + (uint32_t)g * 128u;
+        const uint64_t ph = desc_k_sw128(p_base + (uint32_t)g * 2u * TC_P_BYTES), pl = desc_k_sw128(p_base + (uint32_t)g * 2u * TC_P_BYTES + TC_P_BYTES);
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+          const uint64_t vd = desc_mn_sw128(vb + ks * 2048u, p.v_lbo, p.v_sbo);
+          umma(d, ph + (uint64_t)(ks * 2), vd, idesc_pv, (k == 0 && ks == 0) ? 0u : 1u);
+          umma(d, pl + (uint64_t)(ks * 2), vd, idesc_pv, 1u);
+        }
+        // The scores of this tile were complete before its probabilities could be formed, so once
+        // these MMAs retire both K and V of the stage are free.
+        umma_commit(smem_u32(&empty_bar[j % STAGES]));
+        umma_commit(smem_u32(&pv_done[g]));
+      }
     }
   } else {
     // ---------------- softmax groups: thread <-> query row, group g takes tiles g, g+2, ... ----------------
@@ -999,10 +1005,13 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
   p.n = a->n;
   p.H = a->n_heads;
   p.max_pages = a->max_pages;
-  // CERB_ATTN_TC=1 selects the tcgen05 kernel (head_dim 128).  It is correct (same tests) but its
-  // softmax stage is not yet pipelined deeply enough to beat the warp-MMA kernel, which stays the default.
-  static const int use_tc = getenv("CERB_ATTN_TC") ? atoi(getenv("CERB_ATTN_TC")) : 0;
-  const bool tensor_path = a->head_dim == 128 && use_tc;
+  // The tcgen05 kernel's MMAs are 128 rows tall: it takes the 65..128-node trees, and the 33..64-node trees
+  // once there is enough work to amortise its longer set-up (measured cross-over: about 8K keys per head over
+  // the batch).  Narrow trees and one-node steps stay on the warp-MMA kernel.  CERB_ATTN_TC=0 / 1 forces one.
+  static const int force_tc = getenv("CERB_ATTN_TC") ? atoi(getenv("CERB_ATTN_TC")) : -1;
+  const int np_ = nq_pad(a->n);
+  const bool auto_tc = np_ == 128 || (np_ == 64 && (long long)a->B * a->max_len >= 8192);
+  const bool tensor_path = a->head_dim == 128 && (force_tc < 0 ? auto_tc : force_tc != 0);
   // the tensor-core kernel runs one CTA per SM, the warp-MMA kernel two
   p.nsplit = plan_nsplit(a->B, a->n_heads, nq_pad(a->n), a->max_len, tensor_path ? 148 : kTargetCtas);
   if (p.nsplit < 1) return CERB_E_SHAPE;
