@@ -100,6 +100,8 @@ ATTN_CASES = [
     (16, 16, 32, 128, [40] * 16, 3),    # more (sequence, head) pairs than CTAs wanted: no split
     (16, 128, 2, 128, [8192 - 17 * i for i in range(16)], 6),   # sweep corner: batch 16, 128 nodes, 8K keys
     (5, 32, 3, 128, [511, 512, 513, 2047, 1], 6),
+    (2, 64, 3, 128, [4100, 3991], 5),   # 64-node trees with enough keys to take the tcgen05 kernel
+    (3, 40, 2, 128, [3000, 2999, 1], 5),
 ]
 
 
