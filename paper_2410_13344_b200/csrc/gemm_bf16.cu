@@ -22,9 +22,9 @@
 // fp32 partial slot; consumers add a tile's slots in index order (deterministic).  The CTA that
 // owns a tile's last segment zero-fills the slots that tile does not use.
 //
-// Roles inside a CTA (192 threads): warp 0 = TMA producer (one lane) running ahead through the
-// whole share, warp 1 = TMEM allocator and MMA issuer (one lane), warps 2-5 = epilogue (each owns
-// the 32 TMEM lanes of its warp quarter).  The accumulator is double-buffered in TMEM so a segment's
+// Roles inside a CTA (224 threads): warp 0 = TMA producer (one lane) running ahead through the
+// whole share, warp 1 = TMEM allocator and MMA issuer (one lane), warp 6 = second MMA issuer in wide
+// mode, warps 2-5 = epilogue (each owns the 32 TMEM lanes of its warp quarter).  The accumulator is double-buffered in TMEM so a segment's
 // epilogue overlaps the next segment's MMAs.  Stages and accumulators are handed over with
 // mbarriers; every wait is bounded and reports CERB_E_TIMEOUT through a status word.
 #include <stdlib.h>
@@ -150,6 +150,7 @@ struct GemmParams {
   int wide;           // 1: a CTA works on 256 weight rows at a time (two MMA tiles sharing one activation stage)
   int group;          // stages are released to the producer in groups of this many (1 or 2)
   int hint;           // 1: weights evict-first, activations evict-last in L2
+  int issuers;        // MMA-issuing threads: 2 in wide mode (one per weight tile of a unit), else 1
   uint32_t idesc;
   uint32_t acc_cols;  // TMEM columns of one accumulator buffer
 };
@@ -169,7 +170,7 @@ __device__ __forceinline__ bool next_segment(int& u, int u1, int num_kb, Segment
   return true;
 }
 
-__global__ void __launch_bounds__(192, 1) gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmW,
+__global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmW,
                                                            const __grid_constant__ CUtensorMap tmX, const GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
@@ -193,10 +194,10 @@ __global__ void __launch_bounds__(192, 1) gemm_bf16_kernel(const __grid_constant
     aborted_s = 0;
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(smem_u32(&full_bar[s]), 1);
-      mbar_init(smem_u32(&empty_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), (uint32_t)p.issuers);
     }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(smem_u32(&acc_full[i]), 1);
+      mbar_init(smem_u32(&acc_full[i]), (uint32_t)p.issuers);
       mbar_init(smem_u32(&acc_empty[i]), 4);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -258,8 +259,14 @@ __global__ void __launch_bounds__(192, 1) gemm_bf16_kernel(const __grid_constant
         load_x(i);
       }
     }
-  } else if (warp == 1) {
-    if (lane == 0) {
+  } else if (warp == 1 || warp == 6) {
+    // MMA issuers.  Issuing one tcgen05.mma occupies its thread for ~100 cycles whatever the MMA's size, and
+    // a 64-row step needs eight of them per 32 KB of weights, so in wide mode each of the two weight
+    // tiles of a unit has its own issuing thread (warp 1: first tile, warp 6: second tile).  A stage is
+    // free, and an accumulator complete, once both have committed.
+    const int mine = warp == 6 ? 1 : 0;
+    if (lane == 0 && mine < p.issuers) {
+      const int hf0 = mine, hf1 = (p.issuers == 2) ? mine : p.wide;     // weight tiles of a unit this thread issues
       int u = u0;
       Segment sg;
       int i = 0, g = 0;
@@ -275,16 +282,13 @@ __global__ void __launch_bounds__(192, 1) gemm_bf16_kernel(const __grid_constant
           mbar_wait(smem_u32(&full_bar[s]), ph, aborted, p.status);
           tc_fence_after();
           uint32_t a_src = smem_base + (uint32_t)s * stage_bytes;
-          uint64_t adesc = umma_desc_sw128(a_src);
           uint64_t bdesc = umma_desc_sw128(a_src + a_bytes);
+          for (int hf = hf0; hf <= hf1; ++hf) {
+            const uint64_t adesc = umma_desc_sw128(a_src + (uint32_t)hf * A_STAGE_BYTES);
+            const uint32_t d = tmem_d + (uint32_t)(hf * p.n_mma);
 #pragma unroll
-          for (int kk = 0; kk < BK / 16; ++kk) {
-            // advance 16 k elements = 32 bytes inside the swizzled row: +2 in 16-byte units
-            const uint32_t acc = (k > 0 || kk > 0) ? 1u : 0u;
-            umma_bf16(tmem_d, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), p.idesc, acc);
-            if (p.wide)
-              umma_bf16(tmem_d + (uint32_t)p.n_mma, umma_desc_sw128(a_src + A_STAGE_BYTES) + (uint64_t)(kk * 2),
-                        bdesc + (uint64_t)(kk * 2), p.idesc, acc);
+            for (int kk = 0; kk < BK / 16; ++kk)    // advance 16 k elements = 32 bytes inside the swizzled row: +2 in 16-byte units
+              umma_bf16(d, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), p.idesc, (k > 0 || kk > 0) ? 1u : 0u);
           }
           // Release stages once the MMAs have read them.  Releasing two neighbouring k blocks together
           // makes the producer request 256 contiguous bytes of every weight row at once.
@@ -296,7 +300,7 @@ __global__ void __launch_bounds__(192, 1) gemm_bf16_kernel(const __grid_constant
             held = -1;
           }
         }
-        umma_commit(smem_u32(&acc_full[buf]));       // this segment's accumulator is complete
+        umma_commit(smem_u32(&acc_full[buf]));       // this thread's part of the segment's accumulator is complete
         ++g;
       }
     }
@@ -479,6 +483,8 @@ int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, fl
   p.wide = use_wide(M) ? 1 : 0;
   p.group = group == 2 ? 2 : 1;
   p.hint = hint ? 1 : 0;
+  static int issuers = tune("CERB_GEMM_ISSUERS", 2);
+  p.issuers = (p.wide && issuers == 2) ? 2 : 1;
   uint32_t stage_bytes = A_STAGE_BYTES * (1 + p.wide) + (uint32_t)p.n_mma * BK * 2;
   p.stages = (int)((216u * 1024u) / stage_bytes);
   if (p.stages > MAX_STAGES) p.stages = MAX_STAGES;
@@ -493,7 +499,7 @@ int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, fl
     CERB_CUDA_OK(cudaFuncSetAttribute(gemm_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(220 * 1024)));
     configured = true;
   }
-  if (launch_pdl(gemm_bf16_kernel, dim3(g.ctas), dim3(192), smem, st, *tmW, tmX->m[bucket], p) != cudaSuccess) return CERB_E_CUDA;
+  if (launch_pdl(gemm_bf16_kernel, dim3(g.ctas), dim3(224), smem, st, *tmW, tmX->m[bucket], p) != cudaSuccess) return CERB_E_CUDA;
   CERB_LAUNCH_CHECK(c);
   return CERB_OK;
 }
