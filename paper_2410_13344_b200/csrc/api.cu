@@ -131,6 +131,8 @@ size_t carve(cerb_ctx* c, char* base) {
   c->d_argmax = b.take<int32_t>(Mr);
   c->d_treetok = b.take<int32_t>(MB * CERB_MAX_NODES);
   c->d_topk = b.take<int32_t>(MB * CERB_MAX_HEADS * CERB_MAX_TOPK);
+  c->d_topk_cv = b.take<float>((size_t)MB * CERB_MAX_HEADS * kTopkChunks * CERB_MAX_TOPK);
+  c->d_topk_ci = b.take<int32_t>((size_t)MB * CERB_MAX_HEADS * kTopkChunks * CERB_MAX_TOPK);
   c->d_hlast = b.take<char>((size_t)MB * g.d_model * es);
   c->d_x = b.take<char>((size_t)Mr * g.d_model * sizeof(float));     // residual stream, always fp32
   c->d_xn = b.take<char>((size_t)Mr * g.d_model * es);

@@ -115,6 +115,8 @@ struct cerb_ctx {
   float* d_S;
   void *d_hlast, *d_x, *d_xn, *d_q, *d_attn, *d_act, *d_hidden;
   float *d_part, *d_logits, *d_hlogits;
+  float* d_topk_cv;       // per-chunk top-k candidates of the heads' logits: values [B][Hc][kTopkChunks][MAX_TOPK]
+  int32_t* d_topk_ci;     // ... and their token ids
   size_t part_floats;
   float* d_hstate[2];
   float2* d_rope;
@@ -150,6 +152,7 @@ inline int row_bucket(int rows) {
   return b;
 }
 inline int bucket_rows(int b) { return 16 << b; }
+constexpr int kTopkChunks = 16;     // the vocabulary is cut into this many chunks for the heads' top-k
 
 // ---- launch wrappers implemented across the .cu files (all asynchronous on `st`) ----
 

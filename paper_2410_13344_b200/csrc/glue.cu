@@ -192,11 +192,31 @@ __global__ void argmax_rows_kernel(const float* __restrict__ part, int nsplit, s
   const float* r = part + (size_t)blockIdx.x * V;
   float best = -INFINITY;
   int bi = 0x7fffffff;
-  for (int j = threadIdx.x; j < V; j += blockDim.x) {
-    float v = 0.f;
-    for (int s = 0; s < nsplit; ++s) v += r[s * split_stride + j];
-    if (summed) summed[(size_t)blockIdx.x * V + j] = v;
-    if (v > best || (v == best && j < bi)) { best = v; bi = j; }
+  if ((V & 3) == 0 && (split_stride & 3) == 0) {
+    // 16-byte loads, two column groups per thread in flight: the kernel is pure load latency
+    const int V4 = V >> 2;
+#pragma unroll 2
+    for (int j4 = threadIdx.x; j4 < V4; j4 += blockDim.x) {
+      float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+      for (int s = 0; s < nsplit; ++s) {
+        const float4 t = *reinterpret_cast<const float4*>(r + s * split_stride + 4 * j4);
+        a.x += t.x; a.y += t.y; a.z += t.z; a.w += t.w;
+      }
+      if (summed) *reinterpret_cast<float4*>(summed + (size_t)blockIdx.x * V + 4 * j4) = a;
+      const int j = 4 * j4;                       // ascending ids: a later equal value never replaces an earlier one
+      if (a.x > best) { best = a.x; bi = j; }
+      if (a.y > best) { best = a.y; bi = j + 1; }
+      if (a.z > best) { best = a.z; bi = j + 2; }
+      if (a.w > best) { best = a.w; bi = j + 3; }
+    }
+  } else {
+    for (int j = threadIdx.x; j < V; j += blockDim.x) {
+      float v = 0.f;
+      for (int s = 0; s < nsplit; ++s) v += r[s * split_stride + j];
+      if (summed) summed[(size_t)blockIdx.x * V + j] = v;
+      if (v > best || (v == best && j < bi)) { best = v; bi = j; }
+    }
   }
   for (int o = 16; o > 0; o >>= 1) {
     float ov = __shfl_xor_sync(0xffffffffu, best, o);

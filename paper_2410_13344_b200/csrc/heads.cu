@@ -7,7 +7,7 @@
 // each level is a matrix-vector product: the kernel streams W once with 16-byte loads, keeps the
 // (concatenated) input vector in shared memory as fp32 and fuses bias, residual and SiLU.
 // The FC layer reuses the kernel without an epilogue; a per-head top-k (value descending, lower id
-// first among equals) and the tree fill follow.
+// first among equals; per vocabulary chunk, then over the chunks' candidates) and the tree fill follow.
 #include "cerb_internal.cuh"
 
 namespace cerb {
@@ -83,6 +83,7 @@ __global__ void __launch_bounds__(WARPS * 32) head_gemv_kernel(const LevelParams
 #pragma unroll
     for (int nb = 0; nb < NB; ++nb) acc[i][nb] = 0.f;
   const T* Wp = reinterpret_cast<const T*>(J.W);
+#pragma unroll 2
   for (int k = lane * E; k < w; k += 32 * E) {
     float wv[ROWS_PER_WARP][E];
 #pragma unroll
@@ -139,53 +140,103 @@ __global__ void head_init_kernel(const T* __restrict__ h_last, float* __restrict
 
 __device__ __forceinline__ bool better(float va, int ia, float vb, int ib) { return va > vb || (va == vb && ia < ib); }
 
-// k rounds of a block-wide arg-best; round r only considers entries that come strictly after the
-// previous winner in (value descending, id ascending) order, so nothing is modified in place.
-__global__ void __launch_bounds__(1024) topk_kernel(const float* __restrict__ logits, int V, int Hc,
-                                                    const int32_t* __restrict__ kper, int32_t* __restrict__ topk,
-                                                    int32_t* __restrict__ topk_copy) {
+// Block-wide arg-best over (value, id) pairs in (value descending, id ascending) order.
+__device__ __forceinline__ void block_best(float& best, int& bi, float* sv, int* si) {
+  for (int o = 16; o > 0; o >>= 1) {
+    float ov = __shfl_xor_sync(0xffffffffu, best, o);
+    int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (better(ov, oi, best, bi)) { best = ov; bi = oi; }
+  }
+  const int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = blockDim.x >> 5;
+  if (l == 0) { sv[w] = best; si[w] = bi; }
+  __syncthreads();
+  if (w == 0) {
+    best = l < nw ? sv[l] : -INFINITY;
+    bi = l < nw ? si[l] : 0x7fffffff;
+    for (int o = 16; o > 0; o >>= 1) {
+      float ov = __shfl_xor_sync(0xffffffffu, best, o);
+      int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (better(ov, oi, best, bi)) { best = ov; bi = oi; }
+    }
+    if (l == 0) { sv[0] = best; si[0] = bi; }
+  }
+  __syncthreads();
+  best = sv[0];
+  bi = si[0];
+  __syncthreads();
+}
+
+// Per-head top-k in two steps.  Step 1: the vocabulary is cut into kTopkChunks chunks and one CTA per
+// (chunk, head, sequence) finds its chunk's k best in k rounds; round r only considers entries that come
+// strictly after the previous winner in (value descending, id ascending) order, so nothing is modified
+// in place.  The global k best are among these candidates.  Step 2: one CTA per (head, sequence) runs
+// the same k rounds over the kTopkChunks * k candidates.
+__global__ void __launch_bounds__(256) topk_part_kernel(const float* __restrict__ logits, int V, int Hc,
+                                                        const int32_t* __restrict__ kper, float* __restrict__ cand_v,
+                                                        int32_t* __restrict__ cand_i) {
   __shared__ float sv[32];
   __shared__ int si[32];
-  __shared__ float pv_s;
-  __shared__ int pi_s;
+  griddep_wait();
+  griddep_launch();
+  const int ch = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const float* r = logits + ((size_t)b * Hc + h) * V;
+  const int k = kper[h];
+  const int per = (V + kTopkChunks - 1) / kTopkChunks;
+  const int j0 = ch * per, j1 = min(V, j0 + per);
+  float pv = INFINITY;
+  int pi = -1;
+  const size_t o = (((size_t)b * Hc + h) * kTopkChunks + ch) * CERB_MAX_TOPK;
+  for (int round = 0; round < k; ++round) {
+    float best = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int j = j0 + threadIdx.x; j < j1; j += blockDim.x) {
+      const float v = r[j];
+      const bool after = v < pv || (v == pv && j > pi);
+      if (after && better(v, j, best, bi)) { best = v; bi = j; }
+    }
+    block_best(best, bi, sv, si);
+    pv = best;
+    pi = bi;
+    if (threadIdx.x == 0) {
+      cand_v[o + round] = best;
+      cand_i[o + round] = bi == 0x7fffffff ? -1 : bi;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) topk_merge_kernel(const float* __restrict__ cand_v, const int32_t* __restrict__ cand_i,
+                                                         int Hc, const int32_t* __restrict__ kper, int32_t* __restrict__ topk,
+                                                         int32_t* __restrict__ topk_copy) {
+  __shared__ float sv[32];
+  __shared__ int si[32];
   griddep_wait();
   griddep_launch();
   const int h = blockIdx.x, b = blockIdx.y;
-  const float* r = logits + ((size_t)b * Hc + h) * V;
   const int k = kper[h];
+  const size_t base = ((size_t)b * Hc + h) * kTopkChunks * CERB_MAX_TOPK;
+  // candidate of this thread: (chunk, round) = (t / MAX_TOPK, t % MAX_TOPK)
+  float cv = -INFINITY;
+  int ci = 0x7fffffff;
+  const int t = threadIdx.x;
+  if (t < kTopkChunks * CERB_MAX_TOPK && (t % CERB_MAX_TOPK) < k) {
+    const int id = cand_i[base + t];
+    if (id >= 0) { cv = cand_v[base + t]; ci = id; }
+  }
   float pv = INFINITY;
   int pi = -1;
   for (int round = 0; round < CERB_MAX_TOPK; ++round) {
     int32_t res = -1;
     if (round < k) {
-      float best = -INFINITY;
-      int bi = 0x7fffffff;
-      for (int j = threadIdx.x; j < V; j += blockDim.x) {
-        float v = r[j];
-        bool after = v < pv || (v == pv && j > pi);
-        if (after && better(v, j, best, bi)) { best = v; bi = j; }
-      }
-      for (int o = 16; o > 0; o >>= 1) {
-        float ov = __shfl_xor_sync(0xffffffffu, best, o);
-        int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-        if (better(ov, oi, best, bi)) { best = ov; bi = oi; }
-      }
-      int w = threadIdx.x >> 5, l = threadIdx.x & 31;
-      if (l == 0) { sv[w] = best; si[w] = bi; }
-      __syncthreads();
-      if (threadIdx.x == 0) {
-        for (int i = 1; i < (int)(blockDim.x >> 5); ++i)
-          if (better(sv[i], si[i], best, bi)) { best = sv[i]; bi = si[i]; }
-        pv_s = best;
-        pi_s = bi;
-      }
-      __syncthreads();
-      pv = pv_s;
-      pi = pi_s;
+      const bool after = ci != 0x7fffffff && (cv < pv || (cv == pv && ci > pi));
+      float best = after ? cv : -INFINITY;
+      int bi = after ? ci : 0x7fffffff;
+      block_best(best, bi, sv, si);
+      pv = best;
+      pi = bi;
       res = pi == 0x7fffffff ? -1 : pi;
     }
     if (threadIdx.x == 0) {
-      size_t o = ((size_t)b * Hc + h) * CERB_MAX_TOPK + round;
+      const size_t o = ((size_t)b * Hc + h) * CERB_MAX_TOPK + round;
       topk[o] = res;
       if (topk_copy) topk_copy[o] = res;
     }
@@ -277,7 +328,10 @@ int launch_heads(cerb_ctx* c, const cerb_tree* tree, int32_t* tree_tok, const in
     else CERB_TRY(launch_level<float>(c, P, max_rows, max_w, st));
   }
   const float* lg = logits_out ? logits_out : c->d_hlogits;
-  topk_kernel<<<dim3(Hc, B), 1024, 0, st>>>(lg, g.vocab, Hc, c->d_kper, c->d_topk, topk_out);
+  static_assert(kTopkChunks * CERB_MAX_TOPK <= 256, "one candidate per thread in the merge");
+  topk_part_kernel<<<dim3(kTopkChunks, Hc, B), 256, 0, st>>>(lg, g.vocab, Hc, c->d_kper, c->d_topk_cv, c->d_topk_ci);
+  CERB_LAUNCH_CHECK(c);
+  topk_merge_kernel<<<dim3(Hc, B), 256, 0, st>>>(c->d_topk_cv, c->d_topk_ci, Hc, c->d_kper, c->d_topk, topk_out);
   CERB_LAUNCH_CHECK(c);
   if (tree_tok) {
     tree_fill_kernel<<<B, 128, 0, st>>>(c->d_root, c->d_topk, tree->dev.head_of, tree->dev.rank_of, plant, Hc, tree->n,
