@@ -133,6 +133,7 @@ size_t carve(cerb_ctx* c, char* base) {
   c->d_topk = b.take<int32_t>(MB * CERB_MAX_HEADS * CERB_MAX_TOPK);
   c->d_topk_cv = b.take<float>((size_t)MB * CERB_MAX_HEADS * kTopkChunks * CERB_MAX_TOPK);
   c->d_topk_ci = b.take<int32_t>((size_t)MB * CERB_MAX_HEADS * kTopkChunks * CERB_MAX_TOPK);
+  c->d_gemm_tickets = b.take<unsigned int>(kGemmTickets);
   c->d_hlast = b.take<char>((size_t)MB * g.d_model * es);
   c->d_x = b.take<char>((size_t)Mr * g.d_model * sizeof(float));     // residual stream, always fp32
   c->d_xn = b.take<char>((size_t)Mr * g.d_model * es);
@@ -257,9 +258,18 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
     // residual add fused with the MLP norm
     { ProfScope ps(c, K_GLUE, st);
       CERB_TRY(launch_fused_norm(c, c->d_part, ns, (size_t)M * d, nullptr, 0, 0, n, c->mlp_norm[l], c->d_xn, M, st)); }
-    { ProfScope ps(c, K_GEMM, st);
-      CERB_TRY(gemm(c, c->d_xn, &c->tm_xn, c->wgu[l], c->bf16 ? &c->tm_wgu[l] : nullptr, M, 2 * F, d, &ns, st)); }
-    { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_swiglu(c, c->d_part, ns, (size_t)M * 2 * F, c->d_act, M, st)); }
+    if (c->bf16 && gemm_swiglu_fusable(M, F)) {
+      // SwiGLU runs in the GEMM's epilogue: no separate kernel, no second pass over the partial sums
+      ProfScope ps(c, K_GEMM, st);
+      const int nsl = gemm_plan_split(c->sm_count, M, 2 * F, d);
+      if ((size_t)nsl * M * 2 * F > c->part_floats) return CERB_E_NOMEM;
+      const GemmEpilogue epi{1, c->d_act, c->d_gemm_tickets};
+      CERB_TRY(launch_gemm_bf16(c, &c->tm_wgu[l], &c->tm_xn, c->d_part, M, 2 * F, d, nsl, c->d_status, st, &epi));
+    } else {
+      { ProfScope ps(c, K_GEMM, st);
+        CERB_TRY(gemm(c, c->d_xn, &c->tm_xn, c->wgu[l], c->bf16 ? &c->tm_wgu[l] : nullptr, M, 2 * F, d, &ns, st)); }
+      { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_swiglu(c, c->d_part, ns, (size_t)M * 2 * F, c->d_act, M, st)); }
+    }
     { ProfScope ps(c, K_GEMM, st);
       CERB_TRY(gemm(c, c->d_act, &c->tm_act, c->wd[l], c->bf16 ? &c->tm_wd[l] : nullptr, M, d, F, &ns, st)); }
     // residual add fused with the next layer's attention norm, or with the final norm

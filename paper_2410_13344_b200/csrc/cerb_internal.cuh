@@ -117,6 +117,7 @@ struct cerb_ctx {
   float *d_part, *d_logits, *d_hlogits;
   float* d_topk_cv;       // per-chunk top-k candidates of the heads' logits: values [B][Hc][kTopkChunks][MAX_TOPK]
   int32_t* d_topk_ci;     // ... and their token ids
+  unsigned int* d_gemm_tickets;   // kGemmTickets arrival counters of the GEMM's fused epilogue (zero between launches)
   size_t part_floats;
   float* d_hstate[2];
   float2* d_rope;
@@ -152,6 +153,7 @@ inline int row_bucket(int rows) {
   return b;
 }
 inline int bucket_rows(int b) { return 16 << b; }
+constexpr int kGemmTickets = 4096;
 constexpr int kTopkChunks = 16;     // the vocabulary is cut into this many chunks for the heads' top-k
 
 // ---- launch wrappers implemented across the .cu files (all asynchronous on `st`) ----
@@ -171,8 +173,17 @@ int launch_prefill_commit(cerb_ctx* c, int n, cudaStream_t st);
 // gemm_f32.cu / gemm_bf16.cu : out[split][M][N] fp32 partial sums of X[M][K] . W[N][K]^T
 int launch_gemm_f32(cerb_ctx* c, const float* X, const float* W, float* out, int M, int N, int K, cudaStream_t st);
 int gemm_plan_split(int sm_count, int M, int N, int K);
+// Optional fused epilogue of the bf16 GEMM.  kind 1 (SwiGLU): W is [gate rows F][up rows F]; the GEMM
+// pairs gate tile t with up tile t in one unit and the CTA that completes a tile last writes
+// act[row][f] = SiLU(gate) * up (bf16) instead of leaving the partial slots to a separate kernel.
+struct GemmEpilogue {
+  int kind;                 // 0 none, 1 SwiGLU
+  void* act;                // [M][F] bf16
+  unsigned int* tickets;    // kGemmTickets counters, zero on entry and on exit
+};
+bool gemm_swiglu_fusable(int M, int F);
 int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, float* out, int M, int N, int K,
-                     int nsplit, int32_t* status, cudaStream_t st);
+                     int nsplit, int32_t* status, cudaStream_t st, const GemmEpilogue* epi = nullptr);
 int make_weight_map(CUtensorMap* out, const void* W, int N, int K);
 int make_act_maps(ActMaps* out, const void* X, int rows_alloc, int K);
 int init_driver_api();

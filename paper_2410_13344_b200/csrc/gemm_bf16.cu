@@ -153,6 +153,12 @@ struct GemmParams {
   int issuers;        // MMA-issuing threads: 2 in wide mode (one per weight tile of a unit), else 1
   uint32_t idesc;
   uint32_t acc_cols;  // TMEM columns of one accumulator buffer
+  int tile_rows;      // weight rows between the starts of consecutive tiles
+  int half_off;       // weight-row offset of a wide unit's second tile from its first
+  int epi;            // fused epilogue (GemmEpilogue::kind)
+  int F;              // SwiGLU: width of the gate (and of the up) block
+  bf16* act;          // SwiGLU: output [M][F]
+  unsigned int* tickets;
 };
 
 // One run of k blocks inside one (row chunk, weight tile) job.
@@ -179,6 +185,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
   __shared__ __align__(8) uint64_t acc_empty[2];
   __shared__ uint32_t tmem_base_slot;
   __shared__ int aborted_s;
+  __shared__ unsigned int ticket_s;
   volatile int* aborted = &aborted_s;
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -228,11 +235,11 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
         const uint32_t a_dst = smem_base + (uint32_t)s * stage_bytes;
         mbar_expect_tx(fb, stage_bytes);
         if (p.hint) {
-          tma_load_2d_hint(a_dst, &tmW, w_kb * BK, tile * rows_per_tile, fb, pol_w);
-          if (p.wide) tma_load_2d_hint(a_dst + A_STAGE_BYTES, &tmW, w_kb * BK, tile * rows_per_tile + BM, fb, pol_w);
+          tma_load_2d_hint(a_dst, &tmW, w_kb * BK, tile * p.tile_rows, fb, pol_w);
+          if (p.wide) tma_load_2d_hint(a_dst + A_STAGE_BYTES, &tmW, w_kb * BK, tile * p.tile_rows + p.half_off, fb, pol_w);
         } else {
-          tma_load_2d(a_dst, &tmW, w_kb * BK, tile * rows_per_tile, fb);
-          if (p.wide) tma_load_2d(a_dst + A_STAGE_BYTES, &tmW, w_kb * BK, tile * rows_per_tile + BM, fb);
+          tma_load_2d(a_dst, &tmW, w_kb * BK, tile * p.tile_rows, fb);
+          if (p.wide) tma_load_2d(a_dst + A_STAGE_BYTES, &tmW, w_kb * BK, tile * p.tile_rows + p.half_off, fb);
         }
         if (++w_kb == p.num_kb) { w_kb = 0; ++w_job; }
       };
@@ -323,8 +330,31 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
       const int m_base = mchunk * kGemmRowsPerPass;
       const int m_cnt = min(p.n_mma, p.M - m_base);
       const size_t ldo = (size_t)p.N;
+      const int cnt = last_cta - first_cta + 1;        // CTAs that share this job = slots it uses
+      if (p.epi == 1 && cnt == 1) {
+        // SwiGLU, whole tile in this CTA: gate in the first accumulator half, up in the second
+        const int f = tile * p.tile_rows + quarter * 32 + lane;
+        bf16* a = p.act + (size_t)m_base * p.F + f;
+        const uint32_t tg = tmem_base + (uint32_t)buf * p.acc_cols + ((uint32_t)(quarter * 32) << 16);
+        for (int c0 = 0; c0 < m_cnt; c0 += 16) {
+          uint32_t rg[16], ru[16];
+          tmem_ld16(tg + (uint32_t)c0, rg);
+          tmem_ld16(tg + (uint32_t)p.n_mma + (uint32_t)c0, ru);
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            if (c0 + j < m_cnt) {
+              const float gv = __uint_as_float(rg[j]), uv = __uint_as_float(ru[j]);
+              a[(size_t)(c0 + j) * p.F] = __float2bfloat16_rn(gv / (1.0f + expf(-gv)) * uv);
+            }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
+        ++g;
+        continue;
+      }
       for (int hf = 0; hf <= p.wide; ++hf) {
-        const int n_out = tile * rows_per_tile + hf * BM + quarter * 32 + lane;
+        const int n_out = tile * p.tile_rows + hf * p.half_off + quarter * 32 + lane;
         const bool n_ok = n_out < p.N;
         // consecutive lanes hold consecutive output columns: every store instruction writes 128 contiguous bytes
         float* o = p.out + ((size_t)slot * p.M + m_base) * ldo + (n_ok ? n_out : 0);
@@ -347,14 +377,38 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
-      if ((int)blockIdx.x == last_cta) {
+      if (p.epi == 0 && (int)blockIdx.x == last_cta) {
         for (int hf = 0; hf <= p.wide; ++hf) {
-          const int n_out = tile * rows_per_tile + hf * BM + quarter * 32 + lane;
+          const int n_out = tile * p.tile_rows + hf * p.half_off + quarter * 32 + lane;
           if (n_out >= p.N) continue;
           for (int z = last_cta - first_cta + 1; z < p.nslots; ++z) {
             float* zo = p.out + ((size_t)z * p.M + m_base) * ldo + n_out;
             for (int m = 0; m < m_cnt; ++m) { *zo = 0.f; zo += ldo; }
           }
+        }
+      }
+      if (p.epi == 1) {
+        // The CTA that finishes this tile last (by ticket) adds the tile's slots in index order and applies SwiGLU.
+        __threadfence();
+        asm volatile("bar.sync 2, 128;" ::: "memory");
+        if (warp == 2 && lane == 0) ticket_s = atomicAdd(&p.tickets[sg.job], 1u);
+        asm volatile("bar.sync 2, 128;" ::: "memory");
+        if (ticket_s == (unsigned)cnt - 1u) {
+          __threadfence();
+          const int f = tile * p.tile_rows + quarter * 32 + lane;
+          const float* src = p.out + (size_t)m_base * ldo + f;
+          bf16* a = p.act + (size_t)m_base * p.F + f;
+          const size_t sstride = (size_t)p.M * ldo;
+#pragma unroll 4
+          for (int m = 0; m < m_cnt; ++m) {
+            float gv = 0.f, uv = 0.f;
+            for (int z = 0; z < cnt; ++z) {
+              gv += __ldcg(src + z * sstride + (size_t)m * ldo);
+              uv += __ldcg(src + z * sstride + (size_t)m * ldo + p.F);
+            }
+            a[(size_t)m * p.F] = __float2bfloat16_rn(gv / (1.0f + expf(-gv)) * uv);
+          }
+          if (warp == 2 && lane == 0) p.tickets[sg.job] = 0u;      // ready for the next launch
         }
       }
       ++g;
@@ -451,10 +505,18 @@ int make_pool_map(CUtensorMap* out, const void* pool, int n_pool_pages, int H, i
 }
 
 // Number of partial slots the schedule produces for this problem (what consumers must sum).
+// The fused SwiGLU epilogue needs the wide schedule (both halves of a unit in one CTA) and whole tiles.
+// It pays for few rows only (the auto-regressive step): the CTA that completes a tile re-reads the
+// tile's slots with its 128 epilogue threads, which at 64 rows took 55 us per layer against the
+// 6.6 us of the separate kernel that spreads the same bytes over every SM (measured).
+bool gemm_swiglu_fusable(int M, int F) {
+  static int on = tune("CERB_GEMM_SWIGLU", 1);
+  return on && M >= 1 && M <= 16 && use_wide(M) && F % BM == 0;
+}
 int gemm_plan_split(int sm_count, int M, int N, int K) { return make_plan(sm_count, M, N, K).nslots; }
 
 int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, float* out, int M, int N, int K,
-                     int nsplit, int32_t* status, cudaStream_t st) {
+                     int nsplit, int32_t* status, cudaStream_t st, const GemmEpilogue* epi) {
   if (M <= 0 || N <= 0 || K <= 0 || (K % 8) != 0) return CERB_E_SHAPE;
   static int sm_count = 0;
   if (!sm_count) {
@@ -481,6 +543,15 @@ int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, fl
   p.nslots = g.nslots;
   static int group = tune("CERB_GEMM_GROUP", 1), hint = tune("CERB_GEMM_HINT", 1);
   p.wide = use_wide(M) ? 1 : 0;
+  p.tile_rows = BM * (1 + p.wide);
+  p.half_off = BM;
+  p.epi = 0; p.F = 0; p.act = nullptr; p.tickets = nullptr;
+  if (epi && epi->kind == 1) {
+    if (!gemm_swiglu_fusable(M, N / 2) || (N & 1) || g.tiles * g.mchunks > kGemmTickets || !epi->act || !epi->tickets) return CERB_E_SHAPE;
+    p.epi = 1; p.F = N / 2; p.act = (bf16*)epi->act; p.tickets = epi->tickets;
+    p.tile_rows = BM;            // a unit = gate tile t (rows t*128..) and up tile t (rows F + t*128..)
+    p.half_off = p.F;
+  }
   p.group = group == 2 ? 2 : 1;
   p.hint = hint ? 1 : 0;
   static int issuers = tune("CERB_GEMM_ISSUERS", 2);

@@ -86,6 +86,27 @@ def test_7b_width_two_layers_against_oracle(cb):
     assert eng.device_status() == 0
 
 
+def test_7b_width_one_node_step_against_oracle(cb):
+    """The auto-regressive step (one row per sequence) takes its own code paths: the 16-row GEMM bucket
+    with SwiGLU fused into the gate-up GEMM's epilogue, and the one-node attention layout."""
+    ms = synth.shape_7b(n_layers=2)
+    topk = [10, 10, 10, 10]
+    model, layout, heads, eng = _engine(cb, ms, 4, topk, 512)
+    cmodel, sh = cpu(model), oracle_shape(ms)
+    prompt = [int(t) for t in synth.make_prompt(ms.vocab, 150, seq=9)]
+    th1 = eng.tree(synth.single_node_tree())
+    eng.prefill(torch.tensor([prompt], dtype=torch.int32, device="cuda"), [len(prompt)])
+    st = orc.prefill(cmodel, sh, prompt, 512)
+    lens, roots, _ = eng.read_state()
+    tok = torch.tensor([[int(roots[0])]], dtype=torch.int32, device="cuda")
+    node_argmax, logits, hidden = eng.verify(th1, tok, want_logits=True, want_hidden=True)
+    o_hidden, o_logits = orc.verify_tree(cmodel, sh, st, [int(roots[0])], synth.single_node_tree().parent)
+    assert close(hidden[0], o_hidden) < TOL
+    assert_close_large(logits[0], o_logits, TOL, "logits")
+    assert int(node_argmax[0, 0]) == int(torch.argmax(logits[0, 0]))
+    assert eng.device_status() == 0
+
+
 def _depth_tol(n_layers: int) -> float:
     """Two bf16 forwards that differ only in summation order drift apart like a random walk: every
     rounding point re-quantises a tiny difference into one-ulp flips, about 0.2 % of the rms per
