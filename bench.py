@@ -122,13 +122,6 @@ def rank_prompt(vocab: int, prompt_len: int, rank: int) -> torch.Tensor:
     return synth.make_prompt(vocab, prompt_len, seq=rank).to(torch.int32)
 
 
-def percentile_threshold(values, q):
-    """Threshold with a fraction q of the values at or below it (midpoint of neighbouring order statistics)."""
-    s = sorted(values)
-    k = min(max(int(round(q * len(s))), 1), len(s) - 1)
-    return 0.5 * (s[k - 1] + s[k])
-
-
 def algorithmic_bytes(ms: synth.ModelShape, M: int, kv_len: int, n: int, heads_bytes: int):
     """Bytes one step must move at least (weights once, activations in/out at storage precision)."""
     d, F, V, HD = ms.d_model, ms.mlp_dim, ms.vocab, ms.n_heads * ms.head_dim
@@ -150,7 +143,9 @@ def run_cerb(args, rank, world):
     local = int(os.environ.get("LOCAL_RANK", 0))
     torch.cuda.set_device(local)
     ms, prompt_len, wl_name = workload(args.workload)
-    layout = synth.cerberus_layout(4, 4)
+    # comparison modes (Sec. 5): "medusa" = independent heads without the sequential link and no gate,
+    # "no-gate" = Cerberus heads, every step parallel, "ar" = plain auto-regressive decoding
+    layout = synth.medusa_layout(4, 4) if args.mode == "medusa" else synth.cerberus_layout(4, 4)
     topk = TOPK if args.workload == "7b" else [4, 2, 1, 1]
     n_nodes = N_NODES if args.workload == "7b" else 16
     t_setup = time.time()
@@ -181,7 +176,11 @@ def run_cerb(args, rank, world):
         sync()
         cal_S.append(float(eng.h_S[0]))
         truth.extend(int(t) for t in eng.h_tokens[0, :int(eng.h_n_accept[0])])
-    T = percentile_threshold(cal_S, 0.7)          # about 70 % of the steps decode in parallel
+    T = cb.threshold_from_samples(cal_S, 0.7)          # about 70 % of the steps decode in parallel
+    if args.mode in ("medusa", "no-gate"):
+        T = 1e9
+    elif args.mode == "ar":
+        T = -1.0
     setup_s = time.time() - t_setup
 
     def decode(n_steps, plant_lengths=None, e2e=False, h_plant=None, d_plant=None):
@@ -318,7 +317,7 @@ def run_cerb(args, rank, world):
         "metric": METRIC, "value": agg(tok_a) / (ms_a / 1e3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_a / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": wl_name, "parallelism": "replicas" if world > 1 else "single",
+        "config": {"workload": wl_name, "mode": args.mode, "parallelism": "replicas" if world > 1 else "single",
                    "l2": "every step streams > 13 GB of weights, far beyond the 126 MB L2",
                    "threshold": T, "tree_nodes": n_nodes, "topk": topk, "prompt_len": prompt_len,
                    "acceptance": "natural (random-init heads)"},
@@ -511,6 +510,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="cerb", choices=["cerb", "reference"])
     ap.add_argument("--workload", default="7b")
+    ap.add_argument("--mode", default="cerberus", choices=["cerberus", "medusa", "no-gate", "ar"],
+                    help="decoding variant: the method, or one of the comparison modes of Sec. 5")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cal-steps", type=int, default=64, help="auto-regressive calibration steps before the timed runs")
     ap.add_argument("--kernel", default=None, choices=["gemm", "attention"], help="time one kernel alone instead of the step")

@@ -163,6 +163,13 @@ def workspace_bytes(cfg: Config) -> int:
     return out.value
 
 
+def threshold_from_samples(S: Sequence[float], parallel_fraction: float) -> float:
+    """Midpoint of the two order statistics that leave `parallel_fraction` of the gate values at or below it."""
+    s = sorted(S)
+    k = min(max(int(round(parallel_fraction * len(s))), 1), len(s) - 1)
+    return 0.5 * (s[k - 1] + s[k])
+
+
 def tree_ancestors(parent: np.ndarray) -> np.ndarray:
     parent = np.ascontiguousarray(parent, np.int32)
     out = np.zeros((parent.shape[0], 2), np.uint64)
@@ -318,6 +325,19 @@ class Cerberus:
         h = torch.empty(self.B, self.shape.d_model, dtype=self.shape.torch_dtype)
         _check(lib().cerb_read_state(self.ctx, lens.ctypes.data, roots.ctypes.data, h.data_ptr(), _stream()), "cerb_read_state")
         return lens, roots, h
+
+    def calibrate_threshold(self, th: "TreeHandle", n_steps: int, parallel_fraction: float) -> float:
+        """Host-side helper for the gate's threshold T (Sec. 4.2; the paper lists finding T by hand as a
+        limitation): decodes `n_steps` auto-regressive steps from the current state, which changes that
+        state like any decoding does, and returns the value that would have sent `parallel_fraction`
+        of those steps down the parallel path (entropy at or below T).  Batch 1."""
+        assert self.B == 1 and n_steps >= 2
+        S = []
+        for _ in range(n_steps):
+            self.step(th, -1.0)
+            torch.cuda.current_stream().synchronize()
+            S.append(float(self.h_S[0]))
+        return threshold_from_samples(S, parallel_fraction)
 
     def device_status(self) -> int:
         return lib().cerb_device_status(self.ctx, _stream())

@@ -39,3 +39,11 @@ def test_host_only_calls_work_without_a_gpu():
         assert False
     except binding.CerbError as e:
         assert e.code == binding.E_SHAPE
+
+
+def test_threshold_from_samples_splits_the_requested_fraction():
+    from paper_2410_13344_b200 import binding
+    S = [0.3, 7.9, 7.1, 6.5, 7.7, 2.0, 7.3, 6.9, 7.5, 5.0]
+    for frac, below in ((0.5, 5), (0.7, 7), (0.1, 1), (0.0, 1), (1.0, 9)):
+        T = binding.threshold_from_samples(S, frac)
+        assert sum(1 for v in S if v <= T) == below and T not in S

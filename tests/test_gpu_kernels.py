@@ -102,6 +102,7 @@ ATTN_CASES = [
     (5, 32, 3, 128, [511, 512, 513, 2047, 1], 6),
     (2, 64, 3, 128, [4100, 3991], 5),   # 64-node trees with enough keys to take the tcgen05 kernel
     (3, 40, 2, 128, [3000, 2999, 1], 5),
+    (1, 121, 4, 128, [1500], 4),        # 120 candidate paths + root (the paper's middle tree setting, Sec. 5.1)
 ]
 
 

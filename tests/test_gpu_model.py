@@ -27,7 +27,8 @@ class Rig:
                  max_batch=1, max_nodes=64, std=0.02, shuffled=True):
         self.ms = ms
         self.model = synth.make_model(ms, device="cuda", std=std)
-        self.layout = synth.cerberus_layout(n_cheads, n_levels, concat_level)
+        self.layout = (synth.medusa_layout(n_cheads, n_levels) if concat_level == "medusa"
+                       else synth.cerberus_layout(n_cheads, n_levels, concat_level))
         self.heads = synth.make_heads(ms, self.layout, device="cuda", std=std)
         self.topk = list(topk)
         max_pages = (max_tokens + max_nodes + 15) // 16
@@ -130,7 +131,35 @@ def test_config1_planted_candidates_are_accepted(cb, tiny_fp32, thr):
     rig.eng.free_tree(th)
 
 
-@pytest.mark.parametrize("dtype,concat_level", [("fp32", None), ("fp32", 1), ("bf16", None)])
+@pytest.mark.parametrize("mode", ["cerberus", "no_gate", "medusa_heads", "autoregressive"])
+def test_comparison_modes_all_emit_the_greedy_continuation(cb, mode):
+    """The decoding variants the paper compares (Sec. 5: independent heads without the sequential link,
+    the gate switched off, plain auto-regressive decoding) differ in speed, never in output: each emits
+    the base model's greedy continuation, and each step matches the oracle run in the same mode."""
+    ms = synth.tiny_shape("fp32")
+    rig = Rig(cb, ms, concat_level="medusa" if mode == "medusa_heads" else None)
+    prompt = [int(t) for t in synth.make_prompt(ms.vocab, 48, seq=3)]
+    truth, Ss = orc.ar_greedy(rig.cmodel, rig.sh, prompt, 40)
+    T = {"cerberus": orc.calibrate_threshold(Ss[:24]), "no_gate": 1e9, "medusa_heads": 1e9, "autoregressive": -1.0}[mode]
+    tree = synth.best_first_tree(16, rig.topk)
+    th = rig.eng.tree(tree)
+    lengths = [2, 4, 1, 3]
+    toks, recs = _run_gpu(rig, th, T, prompt, 24,
+                          lambda step, emitted: plant_tokens(tree, truth, emitted, lengths[step % len(lengths)]))
+    otoks, orecs, _ = orc.cerberus_greedy(rig.cmodel, rig.sh, rig.cheads, rig.csrc, prompt, tree.parent, tree.head,
+                                          tree.rank, rig.topk, T, 24, plant=oracle_planter(tree, truth, lengths))
+    assert toks == truth[:24] == otoks
+    n, ok = _compare_runs(rig, recs, orecs, 1e-4, False)
+    assert ok and n == len(orecs)
+    modes = {r["mode"] for r in recs}
+    if mode == "autoregressive":
+        assert modes == {1} and all(r["n_accept"] == 1 for r in recs)
+    elif mode != "cerberus":
+        assert modes == {0} and max(r["n_accept"] for r in recs) >= 3
+    rig.eng.free_tree(th)
+
+
+@pytest.mark.parametrize("dtype,concat_level", [("fp32", None), ("fp32", 1), ("bf16", None), ("fp32", "medusa")])
 def test_each_call_matches_oracle(cb, dtype, concat_level):
     """cerb_gate / cerb_draft / cerb_verify / cerb_accept one by one, with values."""
     ms = synth.tiny_shape(dtype)
@@ -279,6 +308,20 @@ def test_batch_16_with_128_node_trees(cb):
         assert outs[b][:k] == truths[b][:k], b
     assert best >= 4
     assert eng.device_status() == 0
+
+
+def test_threshold_calibration_helper(cb, tiny_fp32):
+    """calibrate_threshold decodes auto-regressively and returns the gate value that splits the observed
+    entropies at the requested fraction; replaying the same steps shows that fraction below it."""
+    rig = tiny_fp32
+    prompt = [int(t) for t in synth.make_prompt(rig.ms.vocab, 40, seq=5)]
+    tok = torch.tensor([prompt], dtype=torch.int32, device="cuda")
+    th = rig.eng.tree(synth.best_first_tree(16, rig.topk))
+    rig.eng.prefill(tok, [len(prompt)])
+    T = rig.eng.calibrate_threshold(th, 20, 0.6)
+    _, Ss = orc.ar_greedy(rig.cmodel, rig.sh, prompt, 20)
+    assert sum(1 for v in Ss[:20] if v <= T) == 12
+    rig.eng.free_tree(th)
 
 
 def test_error_codes(cb):
