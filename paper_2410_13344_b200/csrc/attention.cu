@@ -121,6 +121,7 @@ struct AttnParams {
   int n, H, max_pages, nsplit, oob_row;
   int rows_pad;             // rows per split in `partial` (16, 32, 64 or 128)
   uint32_t v_lbo, v_sbo;    // byte offsets of the V operand's descriptor (tensor-core path)
+  int cluster;              // tensor-core path: the splits of a (sequence, head) form one cluster and merge through shared memory
   float scale_log2;
 };
 
@@ -507,6 +508,25 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// Thread-block cluster helpers: barrier over every thread of the cluster, and loads from another CTA's shared memory.
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t a) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ float4 ld_cluster_v4(uint32_t a) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a) : "memory");
+  return v;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -815,7 +835,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     // ---- output: final, or partial + fixed-order merge by the last CTA of this (sequence, head) ----
     const int ct = threadIdx.x - 64, nct = 256, RP = p.rows_pad;
     const float LN2 = 0.6931471805599453f;
-    if (p.nsplit == 1) {
+    if (p.cluster) {
+      // merged after the role branches, where every thread of the cluster meets
+    } else if (p.nsplit == 1) {
       for (int idx = ct; idx < nq * (DH / 4); idx += nct) {
         const int r = idx / (DH / 4), c4 = idx % (DH / 4);
         const float inv = 1.0f / mrg[(size_t)r * ROWF + DH + 1];
@@ -868,6 +890,39 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
         if (ct == 0) p.counters[b * p.H + h] = 0u;          // ready for the next launch
       }
     }
+  }
+  if (p.cluster) {
+    // The splits of this (sequence, head) are the CTAs of one cluster (rank = split).  Each holds its merged
+    // rows (O, m, l) in shared memory; once all have arrived, CTA r finishes rows r, r + nsplit, ...: it reads
+    // those rows from every member in split order, weighs them and writes the final output.  Nobody leaves
+    // before the second barrier, so no shared memory is read after its CTA has gone.
+    cluster_sync_all();
+    if (warp >= 2 && warp < 10) {
+      const int ct = threadIdx.x - 64;
+      const float LN2 = 0.6931471805599453f;
+      const uint32_t mine = smem_u32(smem_gen);
+      const int c4 = ct & 31;
+      for (int r = split + p.nsplit * (ct >> 5); r < nq; r += p.nsplit * 8) {
+        const uint32_t row_off = (uint32_t)r * (ROWF * 4);
+        float M = -INFINITY;
+        for (int s2 = 0; s2 < p.nsplit; ++s2) M = fmaxf(M, ld_cluster_f32(mapa_u32(mine, (uint32_t)s2) + row_off + DH * 4));
+        const float u = M == -INFINITY ? 0.f : M;
+        float Lsum = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s2 = 0; s2 < p.nsplit; ++s2) {
+          const uint32_t base = mapa_u32(mine, (uint32_t)s2) + row_off;
+          const float w = ex2(ld_cluster_f32(base + DH * 4) - u);
+          Lsum += ld_cluster_f32(base + DH * 4 + 4) * w;
+          const float4 v = ld_cluster_v4(base + (uint32_t)c4 * 16u);
+          acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+        }
+        const float inv = 1.0f / Lsum;
+        *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.n + r) * p.H + h) * DH + c4 * 4) =
+            make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+        if (c4 == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
+      }
+    }
+    cluster_sync_all();
   }
   tc_fence_before();
   __syncthreads();
@@ -1018,6 +1073,7 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
   p.oob_row = a->n_pool_pages * a->n_heads * CERB_PAGE;
   p.scale_log2 = a->scale * 1.4426950408889634f;
   p.rows_pad = nq_pad(a->n);
+  p.cluster = 0;
   // V tile in shared memory: [half of head_dim][64 keys][128 bytes]; 8-key groups are 1024 bytes apart
   p.v_lbo = 8192u;
   p.v_sbo = 1024u;
@@ -1029,8 +1085,14 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
       CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM));
       configured = true;
     }
-    rc = launch_pdl(tree_attn_tc_kernel, dim3(p.nsplit, p.H, a->B), dim3(TC_THREADS), TC_SMEM, st, *tmK, *tmV, p) == cudaSuccess
-             ? CERB_OK : CERB_E_CUDA;
+    static const int use_cluster = getenv("CERB_ATTN_CLUSTER") ? atoi(getenv("CERB_ATTN_CLUSTER")) : 1;
+    p.cluster = (use_cluster && p.nsplit >= 2 && p.nsplit <= 8) ? 1 : 0;
+    if (p.cluster)
+      rc = launch_pdl_cluster(tree_attn_tc_kernel, dim3(p.nsplit, p.H, a->B), dim3(TC_THREADS), TC_SMEM, st, (unsigned)p.nsplit,
+                              *tmK, *tmV, p) == cudaSuccess ? CERB_OK : CERB_E_CUDA;
+    else
+      rc = launch_pdl(tree_attn_tc_kernel, dim3(p.nsplit, p.H, a->B), dim3(TC_THREADS), TC_SMEM, st, *tmK, *tmV, p) == cudaSuccess
+               ? CERB_OK : CERB_E_CUDA;
   } else if (a->head_dim == 128) {
     if (np == 16) rc = launch_cfg<128, 1, 4, 3>(p, tmK, tmV, a->B, st);
     else if (np == 32) rc = launch_cfg<128, 2, 4, 3>(p, tmK, tmV, a->B, st);

@@ -103,6 +103,9 @@ ATTN_CASES = [
     (2, 64, 3, 128, [4100, 3991], 5),   # 64-node trees with enough keys to take the tcgen05 kernel
     (3, 40, 2, 128, [3000, 2999, 1], 5),
     (1, 121, 4, 128, [1500], 4),        # 120 candidate paths + root (the paper's middle tree setting, Sec. 5.1)
+    (1, 64, 32, 128, [8200], 5),        # tcgen05 kernel, four key splits merged inside a thread-block cluster
+    (1, 128, 8, 128, [3000], 6),        # ... three splits
+    (2, 100, 16, 128, [2500, 77], 5),   # ... ragged: the short sequence leaves most splits without keys
 ]
 
 
