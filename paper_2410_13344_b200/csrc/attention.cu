@@ -544,8 +544,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
   __shared__ unsigned int ticket_s;
   volatile int* aborted = &aborted_s;
 
-  griddep_wait();
-  griddep_launch();
+  // Everything up to the first use of Q or of this step's tree keys runs before griddep_wait(): lengths,
+  // live node counts and the page table were written at least two kernels ago, and so were the prefix
+  // keys.  Set-up, the page list and the first prefix tiles thus overlap the previous kernel's tail.
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   const uint32_t q_base = smem_base + STAGES * TC_STAGE_BYTES;
@@ -600,7 +601,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     }
     __syncwarp();
     if (lane == 0) {
+      // tiles of the first ring that lie wholly inside the prefix may be fetched before the wait
+      int early = 0;
+      while (early < T && early < STAGES && (t0 + early + 1) * TILE <= L) ++early;
       for (int i = 0; i < T; ++i) {
+        if (i == early) { griddep_wait(); griddep_launch(); }
         const int s = i % STAGES;
         mbar_wait_polite(smem_u32(&empty_bar[s]), ((uint32_t)(i / STAGES) & 1u) ^ 1u, aborted, p.status);
         const uint32_t fb = smem_u32(&full_bar[s]);
@@ -618,7 +623,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
         }
       }
     }
+    griddep_wait();      // (a lane that has waited already returns at once)
+    griddep_launch();
   } else if (warp == 1) {
+    griddep_wait();
+    griddep_launch();
     // ---------------- QK^T issuer ----------------
     // (issuing one tcgen05.mma costs this thread ~95 cycles whatever its size, measured, so the two
     // products are issued by two different warps)
@@ -642,6 +651,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       }
     }
   } else if (warp == 10) {
+    griddep_wait();
+    griddep_launch();
     // ---------------- PV issuer ----------------
     if (lane == 0) {
       // B operand (V) is MN-major, N = 128 (two 64-wide swizzle atoms, p.v_lbo bytes apart)
@@ -672,6 +683,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     const int row = (warp & 3) * 32 + lane;                    // = TMEM lane
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const bool valid = row < nq;
+    griddep_wait();
+    griddep_launch();
     if (g == 0) {
       // stage this row of Q (zeros past the last node) in the swizzled K-major layout
       const uint4* src = reinterpret_cast<const uint4*>(p.q + (((size_t)b * p.n + (valid ? row : 0)) * p.H + h) * DH);
@@ -813,7 +826,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     }
     tc_fence_before();
     compute_bar(256);
-    if (g == 0) {
+    if (g == 0 && !p.cluster) {
       // merge the two groups' streams, row by row, into group 0's rows
       float* ra = mrg + (size_t)row * ROWF;
       const float* rb = mrg + ((size_t)128 + row) * ROWF;
@@ -904,17 +917,25 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       const int c4 = ct & 31;
       for (int r = split + p.nsplit * (ct >> 5); r < nq; r += p.nsplit * 8) {
         const uint32_t row_off = (uint32_t)r * (ROWF * 4);
+        // 2 * nsplit partial rows: the two softmax groups of every split, in (split, group) order
+        constexpr uint32_t GROUP_OFF = 128u * ROWF * 4u;
         float M = -INFINITY;
-        for (int s2 = 0; s2 < p.nsplit; ++s2) M = fmaxf(M, ld_cluster_f32(mapa_u32(mine, (uint32_t)s2) + row_off + DH * 4));
+        for (int s2 = 0; s2 < p.nsplit; ++s2) {
+          const uint32_t base = mapa_u32(mine, (uint32_t)s2) + row_off + DH * 4;
+          M = fmaxf(M, fmaxf(ld_cluster_f32(base), ld_cluster_f32(base + GROUP_OFF)));
+        }
         const float u = M == -INFINITY ? 0.f : M;
         float Lsum = 0.f;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int s2 = 0; s2 < p.nsplit; ++s2) {
-          const uint32_t base = mapa_u32(mine, (uint32_t)s2) + row_off;
-          const float w = ex2(ld_cluster_f32(base + DH * 4) - u);
-          Lsum += ld_cluster_f32(base + DH * 4 + 4) * w;
-          const float4 v = ld_cluster_v4(base + (uint32_t)c4 * 16u);
-          acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+#pragma unroll
+          for (int gg = 0; gg < 2; ++gg) {
+            const uint32_t base = mapa_u32(mine, (uint32_t)s2) + row_off + (uint32_t)gg * GROUP_OFF;
+            const float w = ex2(ld_cluster_f32(base + DH * 4) - u);
+            Lsum += ld_cluster_f32(base + DH * 4 + 4) * w;
+            const float4 v = ld_cluster_v4(base + (uint32_t)c4 * 16u);
+            acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+          }
         }
         const float inv = 1.0f / Lsum;
         *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.n + r) * p.H + h) * DH + c4 * 4) =
