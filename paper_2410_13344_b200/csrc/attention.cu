@@ -150,8 +150,9 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  griddep_wait();
-  griddep_launch();
+  // Lengths, live node counts, the page table and the prefix keys were written at least two kernels ago:
+  // set-up, the page list and the first prefix tiles run before griddep_wait() and overlap the previous
+  // kernel's tail; Q and this step's tree keys are only touched after it.
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int L = p.len[b];
@@ -187,7 +188,10 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
     }
     __syncwarp();
     if (lane == 0) {
+      int early = 0;
+      while (t0 + early < t_end && early < STAGES && (t0 + early + 1) * TILE <= L) ++early;
       for (int t = t0, i = 0; t < t_end; ++t, ++i) {
+        if (i == early) { griddep_wait(); griddep_launch(); }
         int s = i % STAGES;
         uint32_t ph = (uint32_t)(i / STAGES) & 1u;
         mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, aborted, p.status);
@@ -206,8 +210,12 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
         }
       }
     }
+    griddep_wait();      // (a lane that has waited already returns at once)
+    griddep_launch();
   } else {
     // ---------------- compute warps ----------------
+    griddep_wait();
+    griddep_launch();
     const int qi = warp % WQ, ki = warp / WQ;
     const int g = lane >> 2, tq = lane & 3;
     const int r0 = qi * 16 + g, r1 = r0 + 8;                // this thread's two query rows
