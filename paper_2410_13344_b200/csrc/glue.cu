@@ -70,10 +70,22 @@ __global__ void __launch_bounds__(NORM_THREADS) fused_norm_kernel(float* __restr
                                                                    const int32_t* __restrict__ n_active, int n, int V,
                                                                    const T* __restrict__ gain, T* __restrict__ out, int d, float eps) {
   __shared__ float red[32];
-  griddep_wait();
-  griddep_launch();
   const int row = blockIdx.x;
   float* xr = x + (size_t)row * d;
+  // The residual stream was last written by the previous norm (at least two kernels ago) and the gains
+  // never change: both are fetched before waiting for the kernel in front (a GEMM, or whatever produced
+  // the token ids), so that after the wait only that kernel's output remains to be read.
+  float keep[NORM_MAX_ITER][4], gv[NORM_MAX_ITER][4];
+#pragma unroll
+  for (int it = 0; it < NORM_MAX_ITER; ++it) {
+    const int j = (it * NORM_THREADS + threadIdx.x) * 4;
+    if (j < d) {
+      if (!embed) ld4(xr + j, keep[it]);
+      if (out) ld4(gain + j, gv[it]);
+    }
+  }
+  griddep_wait();
+  griddep_launch();
   const T* src = nullptr;
   if (embed) {
     int b = row / n, v = row % n, t = 0;
@@ -81,7 +93,6 @@ __global__ void __launch_bounds__(NORM_THREADS) fused_norm_kernel(float* __restr
     if (t < 0 || t >= V) t = 0;
     src = embed + (size_t)t * d;
   }
-  float keep[NORM_MAX_ITER][4];
   float ss = 0.f;
 #pragma unroll
   for (int it = 0; it < NORM_MAX_ITER; ++it) {
@@ -89,7 +100,10 @@ __global__ void __launch_bounds__(NORM_THREADS) fused_norm_kernel(float* __restr
     if (j < d) {
       float v[4];
       if (src) ld4(src + j, v);
-      else ld4(xr + j, v);
+      else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) v[e] = keep[it][e];
+      }
       if (nsplit > 0) {
         float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
         const float* pr = part + (size_t)row * d + j;
@@ -113,10 +127,9 @@ __global__ void __launch_bounds__(NORM_THREADS) fused_norm_kernel(float* __restr
   for (int it = 0; it < NORM_MAX_ITER; ++it) {
     const int j = (it * NORM_THREADS + threadIdx.x) * 4;
     if (j < d) {
-      float gv[4], ov[4];
-      ld4(gain + j, gv);
+      float ov[4];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) ov[e] = keep[it][e] * r * gv[e];
+      for (int e = 0; e < 4; ++e) ov[e] = keep[it][e] * r * gv[it][e];
       st4(o + j, ov);
     }
   }
@@ -130,19 +143,23 @@ __global__ void rope_append_kernel(const float* __restrict__ part, int nsplit, s
                                    const int32_t* __restrict__ depth, const int32_t* __restrict__ page_table,
                                    int max_pages, const float2* __restrict__ rope, int max_pos, int n, int H, int Dh,
                                    T* __restrict__ q, T* __restrict__ kpool, T* __restrict__ vpool) {
-  griddep_wait();
-  griddep_launch();
+  // Lengths, live node counts, the tree, the page table and the rotation table are at least two kernels
+  // old: the chain of dependent index loads runs before the wait for the QKV GEMM in front.
   const int row = blockIdx.x, h = blockIdx.y, b = row / n, v = row % n;
-  if (v >= n_active[b]) return;
   const int HD = H * Dh, half = Dh >> 1;
+  const bool active = v < n_active[b];
   const int L = len[b];
   const int pos = L + depth[v], slot = L + v;
-  if (pos >= max_pos || slot >= max_pos) return;
-  const int page = page_table[(size_t)b * max_pages + slot / CERB_PAGE];
+  const bool ok = active && pos < max_pos && slot < max_pos;
+  const int page = ok ? page_table[(size_t)b * max_pages + slot / CERB_PAGE] : 0;
+  const float2 cs0 = (ok && (int)threadIdx.x < half) ? rope[(size_t)pos * half + threadIdx.x] : make_float2(1.f, 0.f);
+  griddep_wait();
+  griddep_launch();
+  if (!ok) return;
   const size_t kv = (((size_t)page * H + h) * CERB_PAGE + (size_t)(slot % CERB_PAGE)) * Dh;
   const float* pr = part + (size_t)row * 3 * HD + h * Dh;
   for (int i = threadIdx.x; i < half; i += blockDim.x) {
-    float2 cs = rope[(size_t)pos * half + i];
+    float2 cs = i == (int)threadIdx.x ? cs0 : rope[(size_t)pos * half + i];
     float q1 = 0.f, q2 = 0.f, k1 = 0.f, k2 = 0.f, v1 = 0.f, v2 = 0.f;
     for (int s = 0; s < nsplit; ++s) {
       const float* p = pr + s * split_stride + i;
