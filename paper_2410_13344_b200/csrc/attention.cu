@@ -1089,12 +1089,16 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
   p.n = a->n;
   p.H = a->n_heads;
   p.max_pages = a->max_pages;
-  // The tcgen05 kernel's MMAs are 128 rows tall: it takes the 65..128-node trees, and the 33..64-node trees
-  // once there is enough work to amortise its longer set-up (measured cross-over: about 8K keys per head over
-  // the batch).  Narrow trees and one-node steps stay on the warp-MMA kernel.  CERB_ATTN_TC=0 / 1 forces one.
+  // The tcgen05 kernel's MMAs are 128 rows tall: it takes the 65..128-node trees.  For 33..64-node trees the
+  // measured cross-overs decide (7B shape, inside the decoding step): with few sequences it wins between
+  // about 1K and 3K keys (4.23 against 4.29 ms per step at 1K, 4.28 against 4.32 at 2K, but 5.50 against
+  // 5.04 at 4K, where the warp-MMA kernel's two CTAs per SM pay off), with four or more sequences from
+  // about 8K keys over the batch (110 against 137 us at 4 x 4K).  Narrow trees and one-node steps stay on
+  // the warp-MMA kernel.  CERB_ATTN_TC=0 / 1 forces one.
   static const int force_tc = getenv("CERB_ATTN_TC") ? atoi(getenv("CERB_ATTN_TC")) : -1;
   const int np_ = nq_pad(a->n);
-  const bool auto_tc = np_ == 128 || (np_ == 64 && (long long)a->B * a->max_len >= 8192);
+  const bool mid = a->B >= 4 ? (long long)a->B * a->max_len >= 8192 : (a->max_len >= 1024 && a->max_len < 3072);
+  const bool auto_tc = np_ == 128 || (np_ == 64 && mid);
   const bool tensor_path = a->head_dim == 128 && (force_tc < 0 ? auto_tc : force_tc != 0);
   // the tensor-core kernel runs one CTA per SM, the warp-MMA kernel two
   p.nsplit = plan_nsplit(a->B, a->n_heads, nq_pad(a->n), a->max_len, tensor_path ? 148 : kTargetCtas);

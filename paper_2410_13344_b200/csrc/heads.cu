@@ -273,13 +273,13 @@ int launch_level(cerb_ctx* c, const LevelParams& P, int max_rows, int max_w, cud
   LevelParams Q = P;
   if (P.B == 1) {
     Q.b0 = 0;
-    head_gemv_kernel<T, 1><<<grid, WARPS * 32, smem1, st>>>(Q);
+    launch_pdl(head_gemv_kernel<T, 1>, grid, dim3(WARPS * 32), smem1, st, Q);
     CERB_LAUNCH_CHECK(c);
   } else {
     if (smem1 * 4 > 200 * 1024) return CERB_E_SHAPE;
     for (int b0 = 0; b0 < P.B; b0 += 4) {
       Q.b0 = b0;
-      head_gemv_kernel<T, 4><<<grid, WARPS * 32, smem1 * 4, st>>>(Q);
+      launch_pdl(head_gemv_kernel<T, 4>, grid, dim3(WARPS * 32), smem1 * 4, st, Q);
       CERB_LAUNCH_CHECK(c);
     }
   }
@@ -293,8 +293,8 @@ int launch_heads(cerb_ctx* c, const cerb_tree* tree, int32_t* tree_tok, const in
   const cerb_config& g = c->cfg;
   const int Hc = g.n_cheads, L = g.n_levels, d = g.d_model, B = c->B;
   if (Hc <= 0) return CERB_E_STATE;
-  if (c->bf16) head_init_kernel<bf16><<<dim3(B, Hc), 256, 0, st>>>((const bf16*)c->d_hlast, c->d_hstate[0], Hc, c->head_wmax, d);
-  else head_init_kernel<float><<<dim3(B, Hc), 256, 0, st>>>((const float*)c->d_hlast, c->d_hstate[0], Hc, c->head_wmax, d);
+  if (c->bf16) launch_pdl(head_init_kernel<bf16>, dim3(B, Hc), dim3(256), 0, st, (const bf16*)c->d_hlast, c->d_hstate[0], Hc, c->head_wmax, d);
+  else launch_pdl(head_init_kernel<float>, dim3(B, Hc), dim3(256), 0, st, (const float*)c->d_hlast, c->d_hstate[0], Hc, c->head_wmax, d);
   CERB_LAUNCH_CHECK(c);
   for (int j = 0; j <= L; ++j) {
     LevelParams P;
@@ -329,13 +329,13 @@ int launch_heads(cerb_ctx* c, const cerb_tree* tree, int32_t* tree_tok, const in
   }
   const float* lg = logits_out ? logits_out : c->d_hlogits;
   static_assert(kTopkChunks * CERB_MAX_TOPK <= 256, "one candidate per thread in the merge");
-  topk_part_kernel<<<dim3(kTopkChunks, Hc, B), 256, 0, st>>>(lg, g.vocab, Hc, c->d_kper, c->d_topk_cv, c->d_topk_ci);
+  launch_pdl(topk_part_kernel, dim3(kTopkChunks, Hc, B), dim3(256), 0, st, lg, g.vocab, Hc, (const int32_t*)c->d_kper, c->d_topk_cv, c->d_topk_ci);
   CERB_LAUNCH_CHECK(c);
-  topk_merge_kernel<<<dim3(Hc, B), 256, 0, st>>>(c->d_topk_cv, c->d_topk_ci, Hc, c->d_kper, c->d_topk, topk_out);
+  launch_pdl(topk_merge_kernel, dim3(Hc, B), dim3(256), 0, st, (const float*)c->d_topk_cv, (const int32_t*)c->d_topk_ci, Hc, (const int32_t*)c->d_kper, c->d_topk, topk_out);
   CERB_LAUNCH_CHECK(c);
   if (tree_tok) {
-    tree_fill_kernel<<<B, 128, 0, st>>>(c->d_root, c->d_topk, tree->dev.head_of, tree->dev.rank_of, plant, Hc, tree->n,
-                                        tree_tok);
+    launch_pdl(tree_fill_kernel, dim3(B), dim3(128), 0, st, (const int32_t*)c->d_root, (const int32_t*)c->d_topk,
+               (const int32_t*)tree->dev.head_of, (const int32_t*)tree->dev.rank_of, plant, Hc, tree->n, tree_tok);
     CERB_LAUNCH_CHECK(c);
   }
   return CERB_OK;
