@@ -468,11 +468,13 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
 // normalisation).
 namespace {
 
-constexpr int TC_STAGES = 3;
 constexpr uint32_t TC_KV_BYTES = 16384;               // K (or V) of one 64-key tile, two 64-wide halves
 constexpr uint32_t TC_STAGE_BYTES = 2 * TC_KV_BYTES;
-constexpr uint32_t TC_Q_BYTES = 32768, TC_P_BYTES = 16384;   // P: one term (hi or lo) of one softmax group
-constexpr size_t TC_SMEM = (size_t)TC_STAGES * TC_STAGE_BYTES + TC_Q_BYTES + 4 * TC_P_BYTES + 1024;
+constexpr uint32_t TC_P_BYTES = 16384;                 // P: one term (hi or lo) of one softmax group
+// Trees of up to 64 nodes need only 64 rows of Q in shared memory (the MMA still reads 128 rows; what it
+// finds past the 64th produces score rows nobody uses), which makes room for a fourth K/V stage.
+__host__ __device__ constexpr uint32_t tc_q_half_bytes(int stages) { return stages == 4 ? 8192u : 16384u; }   // one 64-wide half of head_dim
+constexpr size_t tc_smem(int stages) { return (size_t)stages * TC_STAGE_BYTES + 2 * tc_q_half_bytes(stages) + 4 * TC_P_BYTES + 1024; }
 constexpr int TC_DH = 128, TC_ROWF = TC_DH + 4;
 constexpr int TC_THREADS = 352;                       // producer, QK^T issuer, two softmax groups of four warps, PV issuer
 constexpr float TC_RESCALE = 8.0f;                    // log2 of the growth of a row maximum that forces a rescale
@@ -541,9 +543,12 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+template <int STAGES>
 __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                      const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
-  constexpr int DH = TC_DH, ROWF = TC_ROWF, STAGES = TC_STAGES;
+  constexpr int DH = TC_DH, ROWF = TC_ROWF;
+  constexpr uint32_t QHALF = tc_q_half_bytes(STAGES), TC_Q_BYTES = 2 * QHALF;
+  constexpr int QROWS = (int)(QHALF / 128);
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], s_full[2], s_free[2], p_ready[2], pv_done[2], q_ready;
   __shared__ int page_list[kMaxPagesPerCta];
@@ -641,7 +646,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     // products are issued by two different warps)
     if (lane == 0 && T > 0) {
       const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
-      const uint64_t q_desc0 = desc_k_sw128(q_base), q_desc1 = desc_k_sw128(q_base + 16384u);
+      const uint64_t q_desc0 = desc_k_sw128(q_base), q_desc1 = desc_k_sw128(q_base + QHALF);
       mbar_wait(smem_u32(&q_ready), 0, aborted, p.status);
       for (int i = 0; i < T; ++i) {
         const int g = i & 1, k = i >> 1;
@@ -699,8 +704,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
 #pragma unroll
       for (int c = 0; c < 16; ++c) {
         uint4 v = valid ? src[c] : make_uint4(0, 0, 0, 0);
-        *reinterpret_cast<uint4*>(smem_gen + (q_base - smem_base) + (uint32_t)(c >> 3) * 16384u + (uint32_t)row * 128u +
-                                  (uint32_t)(((c & 7) ^ (row & 7)) << 4)) = v;
+        if (row < QROWS)
+          *reinterpret_cast<uint4*>(smem_gen + (q_base - smem_base) + (uint32_t)(c >> 3) * QHALF + (uint32_t)row * 128u +
+                                    (uint32_t)(((c & 7) ^ (row & 7)) << 4)) = v;
       }
       proxy_fence();
       __syncwarp();
@@ -1115,16 +1121,20 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
   if (tensor_path) {
     static bool configured = false;
     if (!configured) {
-      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM));
+      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_tc_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem(3)));
+      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem(4)));
       configured = true;
     }
+    static const int four = getenv("CERB_ATTN_STAGES4") ? atoi(getenv("CERB_ATTN_STAGES4")) : 1;
+    auto kern = (four && a->n <= 64) ? tree_attn_tc_kernel<4> : tree_attn_tc_kernel<3>;
+    const size_t TC_SMEM = (four && a->n <= 64) ? tc_smem(4) : tc_smem(3);
     static const int use_cluster = getenv("CERB_ATTN_CLUSTER") ? atoi(getenv("CERB_ATTN_CLUSTER")) : 1;
     p.cluster = (use_cluster && p.nsplit >= 2 && p.nsplit <= 8) ? 1 : 0;
     if (p.cluster)
-      rc = launch_pdl_cluster(tree_attn_tc_kernel, dim3(p.nsplit, p.H, a->B), dim3(TC_THREADS), TC_SMEM, st, (unsigned)p.nsplit,
+      rc = launch_pdl_cluster(kern, dim3(p.nsplit, p.H, a->B), dim3(TC_THREADS), TC_SMEM, st, (unsigned)p.nsplit,
                               *tmK, *tmV, p) == cudaSuccess ? CERB_OK : CERB_E_CUDA;
     else
-      rc = launch_pdl(tree_attn_tc_kernel, dim3(p.nsplit, p.H, a->B), dim3(TC_THREADS), TC_SMEM, st, *tmK, *tmV, p) == cudaSuccess
+      rc = launch_pdl(kern, dim3(p.nsplit, p.H, a->B), dim3(TC_THREADS), TC_SMEM, st, *tmK, *tmV, p) == cudaSuccess
                ? CERB_OK : CERB_E_CUDA;
   } else if (a->head_dim == 128) {
     if (np == 16) rc = launch_cfg<128, 1, 4, 3>(p, tmK, tmV, a->B, st);

@@ -100,10 +100,12 @@ ATTN_CASES = [
     (16, 16, 32, 128, [40] * 16, 3),    # more (sequence, head) pairs than CTAs wanted: no split
     (16, 128, 2, 128, [8192 - 17 * i for i in range(16)], 6),   # sweep corner: batch 16, 128 nodes, 8K keys
     (5, 32, 3, 128, [511, 512, 513, 2047, 1], 6),
-    (2, 64, 3, 128, [4100, 3991], 5),   # 64-node trees with enough keys to take the tcgen05 kernel
+    (2, 64, 3, 128, [4100, 3991], 5),   # 64-node trees, long caches, few sequences: warp-MMA kernel with eight splits
     (3, 40, 2, 128, [3000, 2999, 1], 5),
     (1, 121, 4, 128, [1500], 4),        # 120 candidate paths + root (the paper's middle tree setting, Sec. 5.1)
-    (1, 64, 32, 128, [8200], 5),        # tcgen05 kernel, four key splits merged inside a thread-block cluster
+    (1, 64, 32, 128, [8200], 5),
+    (1, 64, 8, 128, [2500], 5),         # tcgen05 kernel, five key splits merged inside a thread-block cluster
+    (4, 64, 2, 128, [2100, 2000, 1900, 2047], 5),   # ... batch of four, ragged
     (1, 128, 8, 128, [3000], 6),        # ... three splits
     (2, 100, 16, 128, [2500, 77], 5),   # ... ragged: the short sequence leaves most splits without keys
 ]
