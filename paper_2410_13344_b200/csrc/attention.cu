@@ -469,12 +469,20 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
 namespace {
 
 constexpr uint32_t TC_KV_BYTES = 16384;               // K (or V) of one 64-key tile, two 64-wide halves
-constexpr uint32_t TC_STAGE_BYTES = 2 * TC_KV_BYTES;
-constexpr uint32_t TC_P_BYTES = 16384;                 // P: one term (hi or lo) of one softmax group
-// Trees of up to 64 nodes need only 64 rows of Q in shared memory (the MMA still reads 128 rows; what it
-// finds past the 64th produces score rows nobody uses), which makes room for a fourth K/V stage.
-__host__ __device__ constexpr uint32_t tc_q_half_bytes(int stages) { return stages == 4 ? 8192u : 16384u; }   // one 64-wide half of head_dim
-constexpr size_t tc_smem(int stages) { return (size_t)stages * TC_STAGE_BYTES + 2 * tc_q_half_bytes(stages) + 4 * TC_P_BYTES + 1024; }
+// K and V tiles travel through rings of 16 KB stages.  The depth of the rings, not HBM, sets the tile rate
+// up to the point where the tensor pipe is busy (a freed stage is back after a TMA round trip of ~2 us;
+// measured at 64 nodes: three K+V stages 1.36 us per 64-key tile, four or five 1.0 us).
+//  * Trees of up to 64 nodes keep only 64 rows of Q and of every P buffer in shared memory (the MMAs still
+//    read 128 rows; what they find past the 64th only reaches score and output rows nobody uses), which
+//    leaves room for five K and five V stages; K and V of a tile then share one pair of barriers (UNI).
+//  * Wider trees need all 128 rows: two K and five V stages with barriers of their own -- a K tile is
+//    free again as soon as its QK^T MMAs have retired, a V tile only after the PV MMAs one softmax later.
+// (One QK^T MMA set of N = 128 over two neighbouring key tiles, filling both groups' score buffers at
+// once, was tried: 24 instead of 32 MMAs per 128 keys, but the groups then run in lockstep and lose
+// their overlap -- 692 against 529 us at batch 16 x 64 nodes x 8K keys.)
+__host__ __device__ constexpr size_t tc_smem(int sk, int sv, int qrows) {
+  return (size_t)(sk + sv) * TC_KV_BYTES + 2 * (size_t)qrows * 128 + 4 * (size_t)qrows * 128 + 1024;   // rings, Q, P (2 groups x hi, lo)
+}
 constexpr int TC_DH = 128, TC_ROWF = TC_DH + 4;
 constexpr int TC_THREADS = 352;                       // producer, QK^T issuer, two softmax groups of four warps, PV issuer
 constexpr float TC_RESCALE = 8.0f;                    // log2 of the growth of a row maximum that forces a rescale
@@ -543,14 +551,14 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-template <int STAGES>
+template <int SK, int SV, int QROWS, bool UNI>
 __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                      const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
   constexpr int DH = TC_DH, ROWF = TC_ROWF;
-  constexpr uint32_t QHALF = tc_q_half_bytes(STAGES), TC_Q_BYTES = 2 * QHALF;
-  constexpr int QROWS = (int)(QHALF / 128);
+  constexpr uint32_t QHALF = (uint32_t)QROWS * 128u, TC_Q_BYTES = 2 * QHALF;
+  constexpr uint32_t TC_P_BYTES = (uint32_t)QROWS * 128u;      // P: one term (hi or lo) of one softmax group
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_bar[STAGES], empty_bar[STAGES], s_full[2], s_free[2], p_ready[2], pv_done[2], q_ready;
+  __shared__ __align__(8) uint64_t full_k[SK], empty_k[SK], full_v[SV], empty_v[SV], s_full[2], s_free[2], p_ready[2], pv_done[2], q_ready;
   __shared__ int page_list[kMaxPagesPerCta];
   __shared__ uint32_t tmem_slot;
   __shared__ int aborted_s;
@@ -562,8 +570,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
   // keys.  Set-up, the page list and the first prefix tiles thus overlap the previous kernel's tail.
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t q_base = smem_base + STAGES * TC_STAGE_BYTES;
-  const uint32_t p_base = q_base + TC_Q_BYTES;          // [group][hi, lo] x 16 KB
+  // Order matters: with 64-row buffers the 128-row MMAs read 8 KB past the end of a P buffer and of Q's
+  // second half; P comes first, then Q, then the rings, so that every such read stays inside this CTA's
+  // shared memory (the last P buffer runs into Q, Q into the K ring).
+  const uint32_t p_base = smem_base;                    // [group][hi, lo] x TC_P_BYTES
+  const uint32_t q_base = p_base + 4 * TC_P_BYTES;
+  const uint32_t k_ring = q_base + TC_Q_BYTES;
+  const uint32_t v_ring = k_ring + SK * TC_KV_BYTES;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int L = p.len[b];
@@ -578,9 +591,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
 
   if (threadIdx.x == 0) {
     aborted_s = (*p.status != 0);
-    for (int s = 0; s < STAGES; ++s) {
-      mbar_init(smem_u32(&full_bar[s]), 1);
-      mbar_init(smem_u32(&empty_bar[s]), 1);
+    for (int s = 0; s < SK; ++s) {
+      mbar_init(smem_u32(&full_k[s]), 1);
+      mbar_init(smem_u32(&empty_k[s]), 1);
+    }
+    for (int s = 0; s < SV; ++s) {
+      mbar_init(smem_u32(&full_v[s]), 1);
+      mbar_init(smem_u32(&empty_v[s]), 1);
     }
     for (int g = 0; g < 2; ++g) {
       mbar_init(smem_u32(&s_full[g]), 1);
@@ -616,23 +633,35 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     if (lane == 0) {
       // tiles of the first ring that lie wholly inside the prefix may be fetched before the wait
       int early = 0;
-      while (early < T && early < STAGES && (t0 + early + 1) * TILE <= L) ++early;
+      while (early < T && early < SK && (t0 + early + 1) * TILE <= L) ++early;
       for (int i = 0; i < T; ++i) {
         if (i == early) { griddep_wait(); griddep_launch(); }
-        const int s = i % STAGES;
-        mbar_wait_polite(smem_u32(&empty_bar[s]), ((uint32_t)(i / STAGES) & 1u) ^ 1u, aborted, p.status);
-        const uint32_t fb = smem_u32(&full_bar[s]);
-        mbar_expect_tx(fb, TC_STAGE_BYTES);
-        const uint32_t kdst = smem_base + (uint32_t)s * TC_STAGE_BYTES, vdst = kdst + TC_KV_BYTES;
+        const int sk = i % SK, sv = i % SV;
+        // UNI: K and V of a tile share the V ring's barriers (SK == SV): one wait and one arrival per tile
+        if (!UNI) mbar_wait_polite(smem_u32(&empty_k[sk]), ((uint32_t)(i / SK) & 1u) ^ 1u, aborted, p.status);
+        else mbar_wait_polite(smem_u32(&empty_v[sv]), ((uint32_t)(i / SV) & 1u) ^ 1u, aborted, p.status);
+        const uint32_t fk = UNI ? smem_u32(&full_v[sv]) : smem_u32(&full_k[sk]);
+        mbar_expect_tx(fk, UNI ? 2 * TC_KV_BYTES : TC_KV_BYTES);
+        const uint32_t kdst = k_ring + (uint32_t)sk * TC_KV_BYTES;
 #pragma unroll
         for (int pg = 0; pg < PAGES_PER_TILE; ++pg) {
           const int row = page_list[i * PAGES_PER_TILE + pg];       // out-of-range rows are zero-filled by TMA
 #pragma unroll
-          for (int hf = 0; hf < 2; ++hf) {
-            const uint32_t off = (uint32_t)hf * 8192u + (uint32_t)pg * (CERB_PAGE * 128);
-            tma_load_2d(kdst + off, &tmK, hf * 64, row, fb);
-            tma_load_2d(vdst + off, &tmV, hf * 64, row, fb);
-          }
+          for (int hf = 0; hf < 2; ++hf)
+            tma_load_2d(kdst + (uint32_t)hf * 8192u + (uint32_t)pg * (CERB_PAGE * 128), &tmK, hf * 64, row, fk);
+        }
+        const uint32_t fv = smem_u32(&full_v[sv]);
+        if (!UNI) {
+          mbar_wait_polite(smem_u32(&empty_v[sv]), ((uint32_t)(i / SV) & 1u) ^ 1u, aborted, p.status);
+          mbar_expect_tx(fv, TC_KV_BYTES);
+        }
+        const uint32_t vdst = v_ring + (uint32_t)sv * TC_KV_BYTES;
+#pragma unroll
+        for (int pg = 0; pg < PAGES_PER_TILE; ++pg) {
+          const int row = page_list[i * PAGES_PER_TILE + pg];
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf)
+            tma_load_2d(vdst + (uint32_t)hf * 8192u + (uint32_t)pg * (CERB_PAGE * 128), &tmV, hf * 64, row, fv);
         }
       }
     }
@@ -650,16 +679,18 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       mbar_wait(smem_u32(&q_ready), 0, aborted, p.status);
       for (int i = 0; i < T; ++i) {
         const int g = i & 1, k = i >> 1;
-        mbar_wait(smem_u32(&full_bar[i % STAGES]), (uint32_t)(i / STAGES) & 1u, aborted, p.status);
+        if (!UNI) mbar_wait(smem_u32(&full_k[i % SK]), (uint32_t)(i / SK) & 1u, aborted, p.status);
+        else mbar_wait(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, aborted, p.status);
         mbar_wait(smem_u32(&s_free[g]), ((uint32_t)k & 1u) ^ 1u, aborted, p.status);
         tc_fence_after();
-        const uint32_t kb = smem_base + (uint32_t)(i % STAGES) * TC_STAGE_BYTES;
+        const uint32_t kb = k_ring + (uint32_t)(i % SK) * TC_KV_BYTES;
         const uint64_t k_desc0 = desc_k_sw128(kb), k_desc1 = desc_k_sw128(kb + 8192u);
         const uint32_t d = tmem + (uint32_t)g * 64u;
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) umma(d, q_desc0 + (uint64_t)(kk * 2), k_desc0 + (uint64_t)(kk * 2), idesc_s, kk ? 1u : 0u);
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) umma(d, q_desc1 + (uint64_t)(kk * 2), k_desc1 + (uint64_t)(kk * 2), idesc_s, 1u);
+        if (!UNI) umma_commit(smem_u32(&empty_k[i % SK]));     // the K tile is free once these MMAs have retired
         umma_commit(smem_u32(&s_full[g]));
       }
     }
@@ -673,8 +704,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       for (int j = 0; j < T; ++j) {
         const int g = j & 1, k = j >> 1;
         mbar_wait(smem_u32(&p_ready[g]), (uint32_t)k & 1u, aborted, p.status);
+        mbar_wait(smem_u32(&full_v[j % SV]), (uint32_t)(j / SV) & 1u, aborted, p.status);
         tc_fence_after();
-        const uint32_t vb = smem_base + (uint32_t)(j % STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
+        const uint32_t vb = v_ring + (uint32_t)(j % SV) * TC_KV_BYTES;
         const uint32_t d = tmem + 128u + (uint32_t)g * 128u;
         const uint64_t ph = desc_k_sw128(p_base + (uint32_t)g * 2u * TC_P_BYTES), pl = desc_k_sw128(p_base + (uint32_t)g * 2u * TC_P_BYTES + TC_P_BYTES);
 #pragma unroll
@@ -683,9 +715,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
           umma(d, ph + (uint64_t)(ks * 2), vd, idesc_pv, (k == 0 && ks == 0) ? 0u : 1u);
           umma(d, pl + (uint64_t)(ks * 2), vd, idesc_pv, 1u);
         }
-        // The scores of this tile were complete before its probabilities could be formed, so once
-        // these MMAs retire both K and V of the stage are free.
-        umma_commit(smem_u32(&empty_bar[j % STAGES]));
+        umma_commit(smem_u32(&empty_v[j % SV]));
         umma_commit(smem_u32(&pv_done[g]));
       }
     }
@@ -781,10 +811,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       }
       if (key0 + TILE > kv_total) {
         // last, partial tile: rows past the end may hold anything (stale pool memory); zero V there so
-        // that a zero probability times a non-finite value cannot poison the sum.  The tile has
-        // landed: its scores were computed from it.
+        // that a zero probability times a non-finite value cannot poison the sum.  V travels apart
+        // from K, so wait until it has landed.
+        mbar_wait(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, aborted, p.status);
         const int first_bad = kv_total - key0;
-        uint8_t* vgen = smem_gen + (size_t)(i % STAGES) * TC_STAGE_BYTES + TC_KV_BYTES;
+        uint8_t* vgen = smem_gen + (v_ring - smem_base) + (size_t)(i % SV) * TC_KV_BYTES;
         for (int idx = gt; idx < (TILE - first_bad) * 16; idx += 128) {
           const int r = first_bad + (idx >> 4), c = idx & 15;
           *reinterpret_cast<uint4*>(vgen + (size_t)(c >> 3) * 8192 + r * 128 + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
@@ -803,8 +834,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
           lo[e] = pack_bf16(p0 - hf.x, p1 - hf.y);
         }
         const uint32_t off = (uint32_t)((c ^ (row & 7)) << 4);
-        *reinterpret_cast<uint4*>(ph + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        *reinterpret_cast<uint4*>(pl + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        if (row < QROWS) {
+          *reinterpret_cast<uint4*>(ph + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *reinterpret_cast<uint4*>(pl + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
       }
       proxy_fence();
       tc_fence_before();
@@ -1024,10 +1057,11 @@ __global__ void __launch_bounds__(128) tree_attn_f32_kernel(const float* __restr
 
 // A split reads `per` tiles of 64 keys and writes an n-row fp32 partial, so wide trees get fewer,
 // longer splits: at least n/8 tiles each keeps the partial traffic near one eighth of the K/V read.
-int plan_nsplit(int B, int H, int n, int max_len, int target_ctas) {
+int plan_nsplit(int B, int H, int n, int max_len, int target_ctas, bool one_wave = false) {
   int tiles = (max_len + TILE - 1) / TILE;
   if (tiles < 1) tiles = 1;
-  int want = (target_ctas + B * H - 1) / (B * H);
+  // the tensor-core kernel holds an SM by itself: its CTAs must fit in one wave, so round down for it
+  int want = one_wave ? target_ctas / (B * H) : (target_ctas + B * H - 1) / (B * H);
   int min_tiles = n / 8 > 1 ? n / 8 : 1;
   if (want > tiles / min_tiles) want = tiles / min_tiles;
   if (want > kMaxSplit) want = kMaxSplit;
@@ -1095,19 +1129,17 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
   p.n = a->n;
   p.H = a->n_heads;
   p.max_pages = a->max_pages;
-  // The tcgen05 kernel's MMAs are 128 rows tall: it takes the 65..128-node trees.  For 33..64-node trees the
-  // measured cross-overs decide (7B shape, inside the decoding step): with few sequences it wins between
-  // about 1K and 3K keys (4.23 against 4.29 ms per step at 1K, 4.28 against 4.32 at 2K, but 5.50 against
-  // 5.04 at 4K, where the warp-MMA kernel's two CTAs per SM pay off), with four or more sequences from
-  // about 8K keys over the batch (110 against 137 us at 4 x 4K).  Narrow trees and one-node steps stay on
-  // the warp-MMA kernel.  CERB_ATTN_TC=0 / 1 forces one.
+  // The tcgen05 kernel's MMAs are 128 rows tall: it takes the 65..128-node trees, and the 33..64-node trees
+  // from about 1K keys per sequence (measured inside the 7B decoding step, batch 1, ms per 64-node forward,
+  // tcgen05 against warp-MMA: 4.18 / 4.18 at 512 keys, 4.20 / 4.29 at 1K, 4.21 / 4.31 at 2K, 4.50 / 4.99 at
+  // 4K, 5.02 / 6.20 at 8K; kernel alone at 2 x 2K keys 29 / 45 us).  Narrow trees and one-node steps stay on
+  // the warp-MMA kernel, whose 16- and 32-row layouts waste no tensor work.  CERB_ATTN_TC=0 / 1 forces one.
   static const int force_tc = getenv("CERB_ATTN_TC") ? atoi(getenv("CERB_ATTN_TC")) : -1;
   const int np_ = nq_pad(a->n);
-  const bool mid = a->B >= 4 ? (long long)a->B * a->max_len >= 8192 : (a->max_len >= 1024 && a->max_len < 3072);
-  const bool auto_tc = np_ == 128 || (np_ == 64 && mid);
+  const bool auto_tc = np_ == 128 || (np_ == 64 && a->max_len >= 1024);
   const bool tensor_path = a->head_dim == 128 && (force_tc < 0 ? auto_tc : force_tc != 0);
   // the tensor-core kernel runs one CTA per SM, the warp-MMA kernel two
-  p.nsplit = plan_nsplit(a->B, a->n_heads, nq_pad(a->n), a->max_len, tensor_path ? 148 : kTargetCtas);
+  p.nsplit = plan_nsplit(a->B, a->n_heads, nq_pad(a->n), a->max_len, tensor_path ? 148 : kTargetCtas, tensor_path);
   if (p.nsplit < 1) return CERB_E_SHAPE;
   p.oob_row = a->n_pool_pages * a->n_heads * CERB_PAGE;
   p.scale_log2 = a->scale * 1.4426950408889634f;
@@ -1121,13 +1153,12 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
   if (tensor_path) {
     static bool configured = false;
     if (!configured) {
-      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_tc_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem(3)));
-      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem(4)));
+      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_tc_kernel<2, 5, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem(2, 5, 128)));
+      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_tc_kernel<5, 5, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem(5, 5, 64)));
       configured = true;
     }
-    static const int four = getenv("CERB_ATTN_STAGES4") ? atoi(getenv("CERB_ATTN_STAGES4")) : 1;
-    auto kern = (four && a->n <= 64) ? tree_attn_tc_kernel<4> : tree_attn_tc_kernel<3>;
-    const size_t TC_SMEM = (four && a->n <= 64) ? tc_smem(4) : tc_smem(3);
+    auto kern = a->n <= 64 ? tree_attn_tc_kernel<5, 5, 64, true> : tree_attn_tc_kernel<2, 5, 128, false>;
+    const size_t TC_SMEM = a->n <= 64 ? tc_smem(5, 5, 64) : tc_smem(2, 5, 128);
     static const int use_cluster = getenv("CERB_ATTN_CLUSTER") ? atoi(getenv("CERB_ATTN_CLUSTER")) : 1;
     p.cluster = (use_cluster && p.nsplit >= 2 && p.nsplit <= 8) ? 1 : 0;
     if (p.cluster)

@@ -100,7 +100,7 @@ ATTN_CASES = [
     (16, 16, 32, 128, [40] * 16, 3),    # more (sequence, head) pairs than CTAs wanted: no split
     (16, 128, 2, 128, [8192 - 17 * i for i in range(16)], 6),   # sweep corner: batch 16, 128 nodes, 8K keys
     (5, 32, 3, 128, [511, 512, 513, 2047, 1], 6),
-    (2, 64, 3, 128, [4100, 3991], 5),   # 64-node trees, long caches, few sequences: warp-MMA kernel with eight splits
+    (2, 64, 3, 128, [4100, 3991], 5),   # 64-node trees over long caches: tcgen05 kernel, eight splits in one cluster
     (3, 40, 2, 128, [3000, 2999, 1], 5),
     (1, 121, 4, 128, [1500], 4),        # 120 candidate paths + root (the paper's middle tree setting, Sec. 5.1)
     (1, 64, 32, 128, [8200], 5),
