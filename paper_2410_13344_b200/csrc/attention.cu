@@ -1132,11 +1132,13 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
   // The tcgen05 kernel's MMAs are 128 rows tall: it takes the 65..128-node trees, and the 33..64-node trees
   // from about 1K keys per sequence (measured inside the 7B decoding step, batch 1, ms per 64-node forward,
   // tcgen05 against warp-MMA: 4.18 / 4.18 at 512 keys, 4.20 / 4.29 at 1K, 4.21 / 4.31 at 2K, 4.50 / 4.99 at
-  // 4K, 5.02 / 6.20 at 8K; kernel alone at 2 x 2K keys 29 / 45 us).  Narrow trees and one-node steps stay on
-  // the warp-MMA kernel, whose 16- and 32-row layouts waste no tensor work.  CERB_ATTN_TC=0 / 1 forces one.
+  // 4K, 5.02 / 6.20 at 8K; kernel alone at 2 x 2K keys 29 / 45 us), and so do the 17..32-node trees (kernel
+  // alone 20 / 30 us at 2K keys, 43 / 68 us at 8K, 523 / 552 us at 16 x 8K).  Trees of up to 16 nodes and
+  // one-node steps stay on the warp-MMA kernel, whose 16-row layout wastes no tensor work and which streams
+  // at 7.0 TB/s at batch 16 x 8K keys (the tcgen05 kernel: 4.2).  CERB_ATTN_TC=0 / 1 forces one.
   static const int force_tc = getenv("CERB_ATTN_TC") ? atoi(getenv("CERB_ATTN_TC")) : -1;
   const int np_ = nq_pad(a->n);
-  const bool auto_tc = np_ == 128 || (np_ == 64 && a->max_len >= 1024);
+  const bool auto_tc = np_ == 128 || ((np_ == 64 || np_ == 32) && a->max_len >= 1024);
   const bool tensor_path = a->head_dim == 128 && (force_tc < 0 ? auto_tc : force_tc != 0);
   // the tensor-core kernel runs one CTA per SM, the warp-MMA kernel two
   p.nsplit = plan_nsplit(a->B, a->n_heads, nq_pad(a->n), a->max_len, tensor_path ? 148 : kTargetCtas, tensor_path);
