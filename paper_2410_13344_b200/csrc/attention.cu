@@ -105,6 +105,25 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
+// Thread-block cluster helpers: barrier over every thread of the cluster, and loads from another CTA's shared memory.
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t a) {
+  float v;
+  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
+  return v;
+}
+__device__ __forceinline__ float4 ld_cluster_v4(uint32_t a) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a) : "memory");
+  return v;
+}
 __device__ __forceinline__ void compute_bar(int nthreads) { asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory"); }
 
 struct AttnParams {
@@ -393,7 +412,9 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
     // ---- output: final, or partial + fixed-order merge by the last CTA of this (sequence, head) ----
     const int ct = warp * 32 + lane, nct = NW * 32;
     const float LN2 = 0.6931471805599453f;
-    if (p.nsplit == 1) {
+    if (p.cluster) {
+      // merged after the role branches, where every thread of the cluster meets
+    } else if (p.nsplit == 1) {
       for (int idx = ct; idx < nq * DH; idx += nct) {
         int r = idx / DH, c = idx % DH;
         float l = mrg[(size_t)r * ROWF + DH + 1];
@@ -446,6 +467,39 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
         if (ct == 0) p.counters[b * p.H + h] = 0u;       // ready for the next launch
       }
     }
+  }
+  if (p.cluster) {
+    // The splits of this (sequence, head) are the CTAs of one cluster (rank = split): each holds its rows
+    // (O, m, l) in shared memory; after the first barrier CTA r merges rows r, r + nsplit, ... from all members
+    // in split order and writes the output.  Nobody leaves before the second barrier.
+    cluster_sync_all();
+    if (warp < NW) {
+      constexpr int C4 = DH / 4;
+      const int ct = warp * 32 + lane, rows_per_pass = (NW * 32) / C4;
+      const float LN2 = 0.6931471805599453f;
+      const uint32_t mine = smem_u32(smem_gen);
+      const int c4 = ct % C4;
+      for (int r = split + p.nsplit * (ct / C4); r < nq; r += p.nsplit * rows_per_pass) {
+        const uint32_t row_off = (uint32_t)r * (ROWF * 4);
+        float M = -INFINITY;
+        for (int s2 = 0; s2 < p.nsplit; ++s2) M = fmaxf(M, ld_cluster_f32(mapa_u32(mine, (uint32_t)s2) + row_off + DH * 4));
+        const float u = M == -INFINITY ? 0.f : M;
+        float Lsum = 0.f;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s2 = 0; s2 < p.nsplit; ++s2) {
+          const uint32_t base = mapa_u32(mine, (uint32_t)s2) + row_off;
+          const float w = exp2f(ld_cluster_f32(base + DH * 4) - u);
+          Lsum += ld_cluster_f32(base + DH * 4 + 4) * w;
+          const float4 v = ld_cluster_v4(base + (uint32_t)c4 * 16u);
+          acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+        }
+        const float inv = 1.0f / Lsum;
+        *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.n + r) * p.H + h) * DH + c4 * 4) =
+            make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
+        if (c4 == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
+      }
+    }
+    cluster_sync_all();
   }
 }
 
@@ -526,25 +580,6 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-// Thread-block cluster helpers: barrier over every thread of the cluster, and loads from another CTA's shared memory.
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
-}
-__device__ __forceinline__ uint32_t mapa_u32(uint32_t saddr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ float ld_cluster_f32(uint32_t a) {
-  float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
-  return v;
-}
-__device__ __forceinline__ float4 ld_cluster_v4(uint32_t a) {
-  float4 v;
-  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a) : "memory");
-  return v;
-}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -1057,14 +1092,14 @@ __global__ void __launch_bounds__(128) tree_attn_f32_kernel(const float* __restr
 
 // A split reads `per` tiles of 64 keys and writes an n-row fp32 partial, so wide trees get fewer,
 // longer splits: at least n/8 tiles each keeps the partial traffic near one eighth of the K/V read.
-int plan_nsplit(int B, int H, int n, int max_len, int target_ctas, bool one_wave = false) {
+int plan_nsplit(int B, int H, int n, int max_len, int target_ctas, bool one_wave = false, int max_split = kMaxSplit) {
   int tiles = (max_len + TILE - 1) / TILE;
   if (tiles < 1) tiles = 1;
   // the tensor-core kernel holds an SM by itself: its CTAs must fit in one wave, so round down for it
   int want = one_wave ? target_ctas / (B * H) : (target_ctas + B * H - 1) / (B * H);
   int min_tiles = n / 8 > 1 ? n / 8 : 1;
   if (want > tiles / min_tiles) want = tiles / min_tiles;
-  if (want > kMaxSplit) want = kMaxSplit;
+  if (want > max_split) want = max_split;
   if (want > tiles) want = tiles;
   if (want < 1) want = 1;
   int per = (tiles + want - 1) / want;
@@ -1084,6 +1119,9 @@ int launch_cfg(const AttnParams& p, const CUtensorMap* tmK, const CUtensorMap* t
     configured = true;
   }
   dim3 grid(p.nsplit, p.H, B);
+  if (p.cluster)
+    return launch_pdl_cluster(tree_attn_bf16_kernel<DH, WQ, WK, STAGES>, grid, dim3((WQ * WK + 1) * 32), smem, st, (unsigned)p.nsplit,
+                              *tmK, *tmV, p) == cudaSuccess ? CERB_OK : CERB_E_CUDA;
   if (launch_pdl(tree_attn_bf16_kernel<DH, WQ, WK, STAGES>, grid, dim3((WQ * WK + 1) * 32), smem, st, *tmK, *tmV, p) != cudaSuccess)
     return CERB_E_CUDA;
   return CERB_OK;
@@ -1141,12 +1179,16 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
   const bool auto_tc = np_ == 128 || ((np_ == 64 || np_ == 32) && a->max_len >= 1024);
   const bool tensor_path = a->head_dim == 128 && (force_tc < 0 ? auto_tc : force_tc != 0);
   // the tensor-core kernel runs one CTA per SM, the warp-MMA kernel two
-  p.nsplit = plan_nsplit(a->B, a->n_heads, nq_pad(a->n), a->max_len, tensor_path ? 148 : kTargetCtas, tensor_path);
+  // With clusters the splits of a (sequence, head) merge through distributed shared memory: at most 8 of them
+  // (the portable cluster size).  CERB_ATTN_CLUSTER=0 keeps the merge through global partials (up to 32 splits).
+  static const int use_cluster = getenv("CERB_ATTN_CLUSTER") ? atoi(getenv("CERB_ATTN_CLUSTER")) : 1;
+  p.nsplit = plan_nsplit(a->B, a->n_heads, nq_pad(a->n), a->max_len, tensor_path ? 148 : kTargetCtas, tensor_path,
+                         use_cluster ? 8 : kMaxSplit);
   if (p.nsplit < 1) return CERB_E_SHAPE;
   p.oob_row = a->n_pool_pages * a->n_heads * CERB_PAGE;
   p.scale_log2 = a->scale * 1.4426950408889634f;
   p.rows_pad = nq_pad(a->n);
-  p.cluster = 0;
+  p.cluster = (use_cluster && p.nsplit >= 2 && p.nsplit <= 8) ? 1 : 0;
   // V tile in shared memory: [half of head_dim][64 keys][128 bytes]; 8-key groups are 1024 bytes apart
   p.v_lbo = 8192u;
   p.v_sbo = 1024u;
@@ -1161,8 +1203,6 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
     }
     auto kern = a->n <= 64 ? tree_attn_tc_kernel<5, 5, 64, true> : tree_attn_tc_kernel<2, 5, 128, false>;
     const size_t TC_SMEM = a->n <= 64 ? tc_smem(5, 5, 64) : tc_smem(2, 5, 128);
-    static const int use_cluster = getenv("CERB_ATTN_CLUSTER") ? atoi(getenv("CERB_ATTN_CLUSTER")) : 1;
-    p.cluster = (use_cluster && p.nsplit >= 2 && p.nsplit <= 8) ? 1 : 0;
     if (p.cluster)
       rc = launch_pdl_cluster(kern, dim3(p.nsplit, p.H, a->B), dim3(TC_THREADS), TC_SMEM, st, (unsigned)p.nsplit,
                               *tmK, *tmV, p) == cudaSuccess ? CERB_OK : CERB_E_CUDA;
