@@ -120,6 +120,20 @@ def test_tree_attention_bf16(cb, case):
         assert close(got_l, l, 0) < 2e-3
 
 
+def test_global_partial_merge_path_in_a_child_process():
+    """By default the key splits merge inside a thread-block cluster.  The older route (partials in the
+    scratch buffer, merged by the CTA that arrives last) stays selectable by an environment switch that is
+    read once per process: run the bf16 attention cases again in a child process with it set."""
+    import os
+    import subprocess
+    import sys
+    env = dict(os.environ, CERB_ATTN_CLUSTER="0")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-m", "pytest", "tests/test_gpu_kernels.py", "-q", "-x", "-m", "gpu", "-k",
+                        "test_tree_attention_bf16"], cwd=root, env=env, capture_output=True, text=True, timeout=1200)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+
+
 def test_tree_attention_bf16_partial_activity(cb):
     res = _attention_case(cb, "bf16", 3, 32, 4, 128, [90, 10, 200], 4, seed_id=40, n_active=[32, 0, 5])
     assert len(res) == 2
