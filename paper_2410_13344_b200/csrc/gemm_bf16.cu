@@ -256,6 +256,8 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
       // while that kernel is still finishing, then wait for it and fetch the activations.
       const int pre = n_units < p.stages ? n_units : p.stages;
       for (int i = 0; i < pre; ++i) load_w(i);
+      // the activation map's descriptor is fetched now, not by the first load after the wait
+      asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tmX) : "memory");
       griddep_wait();
       for (int i = 0; i < pre; ++i) load_x(i);
       for (int i = pre; i < n_units; ++i) {
