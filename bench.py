@@ -377,7 +377,7 @@ def _oracle_sample(ms, model, heads, layout, tree, prompt_len, n_sample_layers):
 
 def cpu_baseline(ms, model, heads, layout, tree, prompt_len, tokens_per_step, par_fraction, budget_s):
     t0 = time.time()
-    ns = 1 if ms.n_layers >= 8 else ms.n_layers
+    ns = 4 if ms.n_layers >= 8 else ms.n_layers        # 4 layers in float64 = 6.5 GB of host memory at the 7B shape
     orc, sub, sh, st, tok = _oracle_sample(ms, model, heads, layout, tree, prompt_len, ns)
     t1 = time.time()
     orc.verify_tree(sub, sh, st, tok, tree.parent)
