@@ -1178,12 +1178,13 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
   const int np_ = nq_pad(a->n);
   const bool auto_tc = np_ == 128 || ((np_ == 64 || np_ == 32) && a->max_len >= 1024);
   const bool tensor_path = a->head_dim == 128 && (force_tc < 0 ? auto_tc : force_tc != 0);
-  // the tensor-core kernel runs one CTA per SM, the warp-MMA kernel two
   // With clusters the splits of a (sequence, head) merge through distributed shared memory: at most 8 of them
   // (the portable cluster size).  CERB_ATTN_CLUSTER=0 keeps the merge through global partials (up to 32 splits).
   static const int use_cluster = getenv("CERB_ATTN_CLUSTER") ? atoi(getenv("CERB_ATTN_CLUSTER")) : 1;
-  p.nsplit = plan_nsplit(a->B, a->n_heads, nq_pad(a->n), a->max_len, tensor_path ? 148 : kTargetCtas, tensor_path,
-                         use_cluster ? 8 : kMaxSplit);
+  // CTAs that fit at once: one per SM for the tensor-core kernel and for the warp-MMA layouts of 32 rows and more
+  // (288 threads x 168 registers), two per SM for the 16-row layout (160 threads); the grid is planned to fit one wave
+  const int resident = (tensor_path || np_ > 16) ? 148 : kTargetCtas;
+  p.nsplit = plan_nsplit(a->B, a->n_heads, nq_pad(a->n), a->max_len, resident, true, use_cluster ? 8 : kMaxSplit);
   if (p.nsplit < 1) return CERB_E_SHAPE;
   p.oob_row = a->n_pool_pages * a->n_heads * CERB_PAGE;
   p.scale_log2 = a->scale * 1.4426950408889634f;
