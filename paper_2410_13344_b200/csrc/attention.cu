@@ -106,8 +106,45 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 // Thread-block cluster helpers: barrier over every thread of the cluster, and loads from another CTA's shared memory.
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+// Rendezvous of the CTAs of a cluster with bounded waits.  Every CTA owns two mbarriers that expect one
+// arrival per member; to meet, one thread of every CTA arrives on that barrier of every member (remote
+// arrive, release at cluster scope) and whoever goes on to read the others' shared memory first waits on its
+// own copy (acquire at cluster scope) with the same cycle budget as every other wait of these kernels.  The
+// hardware cluster barrier is used once only, split in two: every thread arrives right after the barriers
+// are initialised and waits just before the first remote arrive, so that no arrival can reach a barrier that
+// is not initialised yet; that wait depends on nothing but the members having started.
+__device__ __forceinline__ void cluster_start_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
+__device__ __forceinline__ void cluster_start_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// `idx` numbers the calling threads of the CTA from 0: thread s signals member s (the arrivals leave in parallel).
+__device__ __forceinline__ void cluster_meet(uint64_t* bar, int members, int idx, volatile int* aborted, int32_t* status) {
+  const uint32_t local = (uint32_t)__cvta_generic_to_shared(bar);
+  if (idx < members) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"((uint32_t)idx));
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+  }
+  for (int i = 0; i < 1024; ++i)
+    if (mbar_try_wait_cluster(local, 0)) return;
+  const long long t0 = clock64();
+  const long long budget = *aborted ? 40000ll : kWaitCycles;
+  for (;;) {
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait_cluster(local, 0)) return;
+    if (clock64() - t0 > budget) break;
+  }
+  *aborted = 1;
+  atomicExch(status, CERB_E_TIMEOUT);
 }
 __device__ __forceinline__ uint32_t mapa_u32(uint32_t saddr, uint32_t rank) {
   uint32_t r;
@@ -165,6 +202,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
   __shared__ int page_list[kMaxPagesPerCta];
   __shared__ int aborted_s;
   __shared__ unsigned int ticket_s;
+  __shared__ __align__(8) uint64_t cl_bar[2];
   volatile int* aborted = &aborted_s;
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -189,10 +227,13 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
       mbar_init(smem_u32(&full_bar[s]), 1);
       mbar_init(smem_u32(&empty_bar[s]), NW);
     }
+    mbar_init(smem_u32(&cl_bar[0]), (uint32_t)p.nsplit);
+    mbar_init(smem_u32(&cl_bar[1]), (uint32_t)p.nsplit);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     if (too_long) atomicExch(p.status, CERB_E_SHAPE);
   }
   __syncthreads();
+  if (p.cluster) cluster_start_arrive();
   const int t_end = too_long ? t0 : t1;
 
   float* mrg = reinterpret_cast<float*>(smem_gen);   // [NQ][ROWF], used after the key loop
@@ -471,9 +512,10 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
   if (p.cluster) {
     // The splits of this (sequence, head) are the CTAs of one cluster (rank = split): each holds its rows
     // (O, m, l) in shared memory; after the first barrier CTA r merges rows r, r + nsplit, ... from all members
-    // in split order and writes the output.  Nobody leaves before the second barrier.
-    cluster_sync_all();
+    // in split order and writes the output.  Nobody leaves before the second meeting.
+    cluster_start_wait();
     if (warp < NW) {
+      cluster_meet(&cl_bar[0], p.nsplit, (int)threadIdx.x, aborted, p.status);     // every member's rows are in place
       constexpr int C4 = DH / 4;
       const int ct = warp * 32 + lane, rows_per_pass = (NW * 32) / C4;
       const float LN2 = 0.6931471805599453f;
@@ -498,8 +540,10 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
             make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
         if (c4 == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
       }
+      compute_bar(NW * 32);                                                          // this CTA has read all it needs
+      if (warp == 0) cluster_meet(&cl_bar[1], p.nsplit, lane, aborted, p.status);
     }
-    cluster_sync_all();
+    __syncthreads();                           // nobody exits before warp 0 has seen every member done
   }
 }
 
@@ -598,6 +642,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
   __shared__ uint32_t tmem_slot;
   __shared__ int aborted_s;
   __shared__ unsigned int ticket_s;
+  __shared__ __align__(8) uint64_t cl_bar[2];
   volatile int* aborted = &aborted_s;
 
   // Everything up to the first use of Q or of this step's tree keys runs before griddep_wait(): lengths,
@@ -641,6 +686,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       mbar_init(smem_u32(&pv_done[g]), 1);
     }
     mbar_init(smem_u32(&q_ready), 4);
+    mbar_init(smem_u32(&cl_bar[0]), (uint32_t)p.nsplit);
+    mbar_init(smem_u32(&cl_bar[1]), (uint32_t)p.nsplit);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     if (too_long) atomicExch(p.status, CERB_E_SHAPE);
   }
@@ -652,6 +699,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (p.cluster) cluster_start_arrive();
   // tensor memory: columns 0-63 / 64-127 = S of group 0 / 1, 128-255 / 256-383 = O of group 0 / 1
   const uint32_t tmem = tmem_slot;
   float* mrg = reinterpret_cast<float*>(smem_gen);   // [2][128][ROWF] over the whole buffer, once the key loop is over
@@ -990,9 +1038,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     // The splits of this (sequence, head) are the CTAs of one cluster (rank = split).  Each holds its merged
     // rows (O, m, l) in shared memory; once all have arrived, CTA r finishes rows r, r + nsplit, ...: it reads
     // those rows from every member in split order, weighs them and writes the final output.  Nobody leaves
-    // before the second barrier, so no shared memory is read after its CTA has gone.
-    cluster_sync_all();
+    // before the second meeting, so no shared memory is read after its CTA has gone.
+    cluster_start_wait();
     if (warp >= 2 && warp < 10) {
+      cluster_meet(&cl_bar[0], p.nsplit, (int)threadIdx.x - 64, aborted, p.status);  // every member's rows are in place
       const int ct = threadIdx.x - 64;
       const float LN2 = 0.6931471805599453f;
       const uint32_t mine = smem_u32(smem_gen);
@@ -1024,11 +1073,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
             make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
         if (c4 == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
       }
+      compute_bar(256);                                                              // this CTA has read all it needs
+      if (warp == 2) cluster_meet(&cl_bar[1], p.nsplit, lane, aborted, p.status);
     }
-    cluster_sync_all();
   }
   tc_fence_before();
-  __syncthreads();
+  __syncthreads();                             // nobody exits before warp 2 has seen every member done
   if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
 }
 
