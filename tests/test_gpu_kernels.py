@@ -141,6 +141,15 @@ def test_tree_attention_bf16_partial_activity(cb):
         assert close(got_o, O, 0) < TOL_BF16 and close(got_l, l, 0) < 2e-3
 
 
+def test_tree_attention_bf16_partial_activity_on_the_tensor_core_path(cb):
+    """Long caches take the tcgen05 kernel, whose key splits form clusters: a sequence without live nodes makes
+    whole clusters leave at once, one with five live nodes leaves most query rows empty."""
+    res = _attention_case(cb, "bf16", 3, 64, 8, 128, [1500, 1200, 2100], 5, seed_id=42, n_active=[64, 0, 5])
+    assert len(res) == 2
+    for got_o, got_l, O, l in res:
+        assert close(got_o, O, 0) < TOL_BF16 and close(got_l, l, 0) < 2e-3
+
+
 def test_tree_attention_bf16_is_deterministic(cb):
     a = _attention_case(cb, "bf16", 1, 64, 8, 128, [3000], 5, seed_id=41)[0]
     b = _attention_case(cb, "bf16", 1, 64, 8, 128, [3000], 5, seed_id=41)[0]
