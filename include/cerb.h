@@ -280,7 +280,12 @@ int cerb_device_status(cerb_ctx* ctx, void* stream);
  * attention, 2 decoding heads + top-k + tree fill, 3 element-wise glue (embedding, norms, RoPE
  * and KV append, residual, SwiGLU, argmax), 4 gate, 5 acceptance + KV compaction.
  * ms_out and groups_out are host arrays of CERB_PROF_KINDS entries.  Event recording costs a few
- * microseconds per bracket, so time whole steps with profiling off. */
+ * microseconds per bracket and keeps neighbouring kernels from overlapping, so time whole steps with
+ * profiling off.  cerb_profile_enable(ctx, 2) selects a second mode that leaves the launch sequence
+ * untouched: every bf16 GEMM launch records, in the device's nanosecond timer, when its first CTA got past
+ * the wait for the previous kernel and when its last CTA finished; cerb_profile_read then returns the sum of
+ * those spans in ms_out[0] and their number in groups_out[0] (other families 0; at most 4096 launches
+ * between reads).  on = 0 switches profiling off, 1 selects the event brackets. */
 #define CERB_PROF_KINDS 6
 int cerb_profile_enable(cerb_ctx* ctx, int32_t on);
 int cerb_profile_read(cerb_ctx* ctx, double* ms_out, int64_t* groups_out, void* stream);

@@ -344,8 +344,10 @@ class Cerberus:
 
     PROF_KINDS = ("gemm", "attention", "heads", "glue", "gate", "accept")
 
-    def profile(self, on: bool):
-        _check(lib().cerb_profile_enable(self.ctx, 1 if on else 0), "cerb_profile_enable")
+    def profile(self, on):
+        """False / 0: off; True / 1: CUDA-event brackets per kernel family; 2: the GEMM kernels stamp their own
+        spans with the device timer (the launch sequence stays as it is)."""
+        _check(lib().cerb_profile_enable(self.ctx, int(on)), "cerb_profile_enable")
 
     def profile_read(self):
         """{family: (milliseconds, launch groups)} since the last read."""

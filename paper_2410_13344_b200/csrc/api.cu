@@ -46,7 +46,7 @@ struct ProfScope {
   cudaStream_t st;
   long idx;
   ProfScope(cerb_ctx* c_, int kind, cudaStream_t st_) : c(c_), st(st_), idx(-1) {
-    if (!c->prof_on || c->prof_used >= kProfMaxPairs) return;
+    if (!c->prof_on || c->prof_mode != 1 || c->prof_used >= kProfMaxPairs) return;
     if (c->prof_used * 2 >= c->prof_ev.size()) {
       cudaEvent_t a, b;
       if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) return;
@@ -134,6 +134,7 @@ size_t carve(cerb_ctx* c, char* base) {
   c->d_topk_cv = b.take<float>((size_t)MB * CERB_MAX_HEADS * kTopkChunks * CERB_MAX_TOPK);
   c->d_topk_ci = b.take<int32_t>((size_t)MB * CERB_MAX_HEADS * kTopkChunks * CERB_MAX_TOPK);
   c->d_gemm_tickets = b.take<unsigned int>(kGemmTickets);
+  c->d_gemm_clock = b.take<unsigned long long>(2 * kGemmClockSlots);
   c->d_hlast = b.take<char>((size_t)MB * g.d_model * es);
   c->d_x = b.take<char>((size_t)Mr * g.d_model * sizeof(float));     // residual stream, always fp32
   c->d_xn = b.take<char>((size_t)Mr * g.d_model * es);
@@ -209,6 +210,12 @@ int tree_build(cerb_ctx* c, const int32_t* parent, const int32_t* head_of, const
   return CERB_OK;
 }
 
+// Device-clock profiling (mode 2): the next GEMM launch stamps its span into the next free slot.
+unsigned long long* gemm_clock_slot(cerb_ctx* c) {
+  if (!c->prof_on || c->prof_mode != 2 || c->gemm_clock_used >= kGemmClockSlots) return nullptr;
+  return c->d_gemm_clock + c->gemm_clock_used++;
+}
+
 // out = X . W^T as fp32 split partials in d_part; returns the split count.
 int gemm(cerb_ctx* c, const void* X, const ActMaps* xm, const void* W, const CUtensorMap* wm, int M, int N, int K,
          int* nsplit, cudaStream_t st) {
@@ -216,7 +223,7 @@ int gemm(cerb_ctx* c, const void* X, const ActMaps* xm, const void* W, const CUt
     int ns = gemm_plan_split(c->sm_count, M, N, K);
     if ((size_t)ns * M * N > c->part_floats) return CERB_E_NOMEM;
     *nsplit = ns;
-    return launch_gemm_bf16(c, wm, xm, c->d_part, M, N, K, ns, c->d_status, st);
+    return launch_gemm_bf16(c, wm, xm, c->d_part, M, N, K, ns, c->d_status, st, nullptr, gemm_clock_slot(c));
   }
   if ((size_t)M * N > c->part_floats) return CERB_E_NOMEM;
   *nsplit = 1;
@@ -264,7 +271,7 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
       const int nsl = gemm_plan_split(c->sm_count, M, 2 * F, d);
       if ((size_t)nsl * M * 2 * F > c->part_floats) return CERB_E_NOMEM;
       const GemmEpilogue epi{1, c->d_act, c->d_gemm_tickets};
-      CERB_TRY(launch_gemm_bf16(c, &c->tm_wgu[l], &c->tm_xn, c->d_part, M, 2 * F, d, nsl, c->d_status, st, &epi));
+      CERB_TRY(launch_gemm_bf16(c, &c->tm_wgu[l], &c->tm_xn, c->d_part, M, 2 * F, d, nsl, c->d_status, st, &epi, gemm_clock_slot(c)));
     } else {
       { ProfScope ps(c, K_GEMM, st);
         CERB_TRY(gemm(c, c->d_xn, &c->tm_xn, c->wgu[l], c->bf16 ? &c->tm_wgu[l] : nullptr, M, 2 * F, d, &ns, st)); }
@@ -384,6 +391,8 @@ int cerb_load(const cerb_config* cfg, const cerb_weights* w, void* workspace_dev
   c->verified_tree = nullptr;
   c->launches = 0;
   c->prof_on = false;
+  c->prof_mode = 0;
+  c->gemm_clock_used = 0;
   c->prof_used = 0;
   memset(c->tree_used, 0, sizeof(c->tree_used));
   memset(c->h_len, 0, sizeof(c->h_len));
@@ -675,8 +684,15 @@ int cerb_device_status(cerb_ctx* c, void* stream) {
 }
 
 int cerb_profile_enable(cerb_ctx* c, int32_t on) {
-  if (!c) return CERB_E_ARG;
+  if (!c || on < 0 || on > 2) return CERB_E_ARG;
   c->prof_on = on != 0;
+  c->prof_mode = on;
+  if (on == 2) {
+    // starts collect a minimum, ends a maximum
+    CERB_CUDA_OK(cudaMemset(c->d_gemm_clock, 0xFF, kGemmClockSlots * sizeof(unsigned long long)));
+    CERB_CUDA_OK(cudaMemset(c->d_gemm_clock + kGemmClockSlots, 0, kGemmClockSlots * sizeof(unsigned long long)));
+    c->gemm_clock_used = 0;
+  }
   return CERB_OK;
 }
 
@@ -684,6 +700,19 @@ int cerb_profile_read(cerb_ctx* c, double* ms_out, int64_t* groups_out, void* st
   if (!c || !ms_out || !groups_out) return CERB_E_ARG;
   CERB_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
   for (int k = 0; k < CERB_PROF_KINDS; ++k) { ms_out[k] = 0.0; groups_out[k] = 0; }
+  if (c->prof_mode == 2) {
+    const int n = c->gemm_clock_used;
+    std::vector<unsigned long long> h(2 * (size_t)kGemmClockSlots);
+    CERB_CUDA_OK(cudaMemcpy(h.data(), c->d_gemm_clock, h.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+    for (int i = 0; i < n; ++i) {
+      const unsigned long long t0 = h[i], t1 = h[kGemmClockSlots + i];
+      if (t1 > t0) { ms_out[0] += (double)(t1 - t0) * 1e-6; groups_out[0] += 1; }
+    }
+    CERB_CUDA_OK(cudaMemset(c->d_gemm_clock, 0xFF, kGemmClockSlots * sizeof(unsigned long long)));
+    CERB_CUDA_OK(cudaMemset(c->d_gemm_clock + kGemmClockSlots, 0, kGemmClockSlots * sizeof(unsigned long long)));
+    c->gemm_clock_used = 0;
+    return CERB_OK;
+  }
   for (size_t i = 0; i < c->prof_used; ++i) {
     float ms = 0.f;
     if (cudaEventElapsedTime(&ms, c->prof_ev[2 * i], c->prof_ev[2 * i + 1]) != cudaSuccess) continue;

@@ -161,6 +161,9 @@ struct cerb_ctx {
 
   // optional per-family timing (cerb_profile_*)
   bool prof_on;
+  int prof_mode;                      // 1: CUDA-event brackets per family; 2: the GEMM kernels stamp their own span
+  unsigned long long* d_gemm_clock;   // [2][kGemmClockSlots]: first CTA past its dependency wait, last CTA done (ns)
+  int gemm_clock_used;
   std::vector<cudaEvent_t> prof_ev;   // begin/end pairs
   std::vector<int> prof_kind;         // family of each pair
   size_t prof_used;                   // pairs recorded since the last read
@@ -175,6 +178,7 @@ inline int row_bucket(int rows) {
 }
 inline int bucket_rows(int b) { return 16 << b; }
 constexpr int kGemmTickets = 4096;
+constexpr int kGemmClockSlots = 4096;
 constexpr int kTopkChunks = 16;     // the vocabulary is cut into this many chunks for the heads' top-k
 
 // ---- launch wrappers implemented across the .cu files (all asynchronous on `st`) ----
@@ -204,7 +208,8 @@ struct GemmEpilogue {
 };
 bool gemm_swiglu_fusable(int M, int F);
 int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, float* out, int M, int N, int K,
-                     int nsplit, int32_t* status, cudaStream_t st, const GemmEpilogue* epi = nullptr);
+                     int nsplit, int32_t* status, cudaStream_t st, const GemmEpilogue* epi = nullptr,
+                     unsigned long long* clock_slot = nullptr);
 int make_weight_map(CUtensorMap* out, const void* W, int N, int K);
 int make_act_maps(ActMaps* out, const void* X, int rows_alloc, int K);
 int init_driver_api();

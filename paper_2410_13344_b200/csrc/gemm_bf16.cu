@@ -126,6 +126,11 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
@@ -159,6 +164,8 @@ struct GemmParams {
   int F;              // SwiGLU: width of the gate (and of the up) block
   bf16* act;          // SwiGLU: output [M][F]
   unsigned int* tickets;
+  unsigned long long* clk;   // measurement only: clk[0] <- min over CTAs of the time the dependency wait returned,
+                             // clk[kGemmClockSlots] <- max over CTAs of the time the CTA finished (globaltimer, ns); or null
 };
 
 // One run of k blocks inside one (row chunk, weight tile) job.
@@ -259,6 +266,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
       // the activation map's descriptor is fetched now, not by the first load after the wait
       asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tmX) : "memory");
       griddep_wait();
+      if (p.clk) atomicMin(p.clk, globaltimer_ns());
       for (int i = 0; i < pre; ++i) load_x(i);
       for (int i = pre; i < n_units; ++i) {
         const int s = i % p.stages;
@@ -418,6 +426,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
   }
   tc_fence_before();
   __syncthreads();
+  if (p.clk && threadIdx.x == 0) atomicMax(p.clk + kGemmClockSlots, globaltimer_ns());
   if (warp == 1) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2u * p.acc_cols) : "memory");
   }
@@ -518,7 +527,7 @@ bool gemm_swiglu_fusable(int M, int F) {
 int gemm_plan_split(int sm_count, int M, int N, int K) { return make_plan(sm_count, M, N, K).nslots; }
 
 int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, float* out, int M, int N, int K,
-                     int nsplit, int32_t* status, cudaStream_t st, const GemmEpilogue* epi) {
+                     int nsplit, int32_t* status, cudaStream_t st, const GemmEpilogue* epi, unsigned long long* clock_slot) {
   if (M <= 0 || N <= 0 || K <= 0 || (K % 8) != 0) return CERB_E_SHAPE;
   static int sm_count = 0;
   if (!sm_count) {
@@ -548,6 +557,7 @@ int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, fl
   p.tile_rows = BM * (1 + p.wide);
   p.half_off = BM;
   p.epi = 0; p.F = 0; p.act = nullptr; p.tickets = nullptr;
+  p.clk = clock_slot;
   if (epi && epi->kind == 1) {
     if (!gemm_swiglu_fusable(M, N / 2) || (N & 1) || g.tiles * g.mchunks > kGemmTickets || !epi->act || !epi->tickets) return CERB_E_SHAPE;
     p.epi = 1; p.F = N / 2; p.act = (bf16*)epi->act; p.tickets = epi->tickets;
