@@ -324,6 +324,32 @@ def test_threshold_calibration_helper(cb, tiny_fp32):
     rig.eng.free_tree(th)
 
 
+def test_profiling_modes(cb):
+    """Mode 1 brackets every kernel family with events; mode 2 lets each bf16 GEMM launch stamp its own span
+    with the device timer.  Both count the GEMMs of one verification forward: four per layer and the LM head."""
+    ms = synth.tiny_shape("bf16")
+    rig = Rig(cb, ms)
+    eng = rig.eng
+    prompt = [int(t) for t in synth.make_prompt(ms.vocab, 30, seq=6)]
+    eng.prefill(torch.tensor([prompt], dtype=torch.int32, device="cuda"), [len(prompt)])
+    th = eng.tree(synth.best_first_tree(16, rig.topk))
+    tok = torch.zeros(1, 16, dtype=torch.int32, device="cuda")
+    n_gemm = 4 * ms.n_layers + 1
+    for mode in (1, 2):
+        eng.profile(mode)
+        eng.profile_read()
+        eng.verify(th, tok)
+        prof = eng.profile_read()
+        assert prof["gemm"][1] == n_gemm and 0.0 < prof["gemm"][0] < 1e3, (mode, prof)
+        if mode == 1:
+            assert prof["attention"][1] == ms.n_layers and prof["glue"][1] > 0
+        else:
+            assert prof["attention"][1] == 0
+    eng.profile(False)
+    assert cb.lib().cerb_profile_enable(eng.ctx, 3) == cb.E_ARG
+    assert eng.device_status() == 0
+
+
 def test_error_codes(cb):
     ms = synth.tiny_shape("fp32")
     rig = Rig(cb, ms, max_tokens=128)
