@@ -39,7 +39,10 @@ template <typename T> struct Vec16;
 template <> struct Vec16<bf16> {
   static constexpr int N = 8;
   static __device__ __forceinline__ void load(const bf16* p, float* f) {
-    uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
+    uint4 v;
+    // streamed once: no L1 allocation, and the memory side is asked for 256-byte pieces
+    asm volatile("ld.global.nc.L1::no_allocate.L2::256B.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
 #pragma unroll
     for (int i = 0; i < 4; ++i) { float2 t = __bfloat1622float2(h[i]); f[2 * i] = t.x; f[2 * i + 1] = t.y; }
