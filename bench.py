@@ -2,6 +2,7 @@
 """Benchmark of the Cerberus decoding step on a 7B-shaped, random-init bf16 model.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl cerb|reference] [--workload 7b|tiny]
+    python bench.py --sweep            # verify step alone over batch x KV length x tree nodes
 
 A "step" is one whole decoding step (gate, draft when the gate allows it, tree verification
 through all layers, acceptance and KV compaction) of one sequence.  Prints ONE JSON line.
@@ -517,6 +518,81 @@ def run_kernel(args):
     print(json.dumps(out))
 
 
+def run_sweep(args):
+    """The verify step alone (row a5 + a6: embedding .. LM head + argmax over every tree node) at the 7B shape over
+    batch x committed KV length x tree nodes, random-parent trees of depth <= 6, KV produced by a real prefill of
+    random token ids.  One JSON line per point: step latency (undisturbed launch sequence, CUDA events), attention
+    GB/s over its algorithmic bytes (event brackets around the attention launches), GEMM TFLOP/s from the kernels'
+    own device-clock spans and its fraction of the binding roofline min(tensor peak, rows x HBM)."""
+    from paper_2410_13344_b200 import binding as cb
+    import __graft_entry__
+    __graft_entry__.build()
+    torch.cuda.set_device(0)
+    hbm_peak, tf_peak, kind = peaks()
+    ms = synth.shape_7b()
+    model = synth.make_model(ms, device="cuda")
+    HD = ms.n_heads * ms.head_dim
+    params = ms.n_layers * (3 * HD * ms.d_model + ms.d_model * HD + 3 * ms.mlp_dim * ms.d_model) + ms.vocab * ms.d_model
+    batches = [int(x) for x in args.sweep_B.split(",")]
+    lens = [int(x) for x in args.sweep_len.split(",")]
+    nodes = [int(x) for x in args.sweep_n.split(",")]
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    points = []
+    for B in batches:
+        for L in lens:
+            eng = cb.Cerberus(ms, model, None, None, (), max_tokens=L + 16, max_batch=B, max_nodes=128)
+            prompts = torch.stack([synth.make_prompt(ms.vocab, L, seq=b).to(torch.int32) for b in range(B)]).cuda().contiguous()
+            eng.prefill(prompts, [L] * B)
+            torch.cuda.synchronize()
+            for n in nodes:
+                th = eng.tree(synth.random_parent_tree(n, 6, tree_id=n))
+                tok = torch.stack([synth.make_prompt(ms.vocab, n, seq=1000 + b).to(torch.int32) for b in range(B)]).cuda().contiguous()
+                run = lambda: eng.verify(th, tok)          # verify without accept leaves the committed state as it is
+                for _ in range(3):
+                    run()
+                torch.cuda.synchronize()
+                e0, e1 = ev(), ev()
+                e0.record()
+                for _ in range(args.iters):
+                    run()
+                e1.record()
+                torch.cuda.synchronize()
+                step_ms = e0.elapsed_time(e1) / args.iters
+                k = max(2, args.iters // 2)
+                eng.profile(1); eng.profile_read()
+                for _ in range(k):
+                    run()
+                prof = eng.profile_read()
+                eng.profile(2)
+                for _ in range(k):
+                    run()
+                clk = eng.profile_read()
+                eng.profile(False)
+                M = B * n
+                gemm_b, attn_b, _ = algorithmic_bytes(ms, M, L, n, 0)
+                attn_b *= B
+                attn_ms = prof["attention"][0] / k
+                gemm_ev_ms, gemm_ck_ms = prof["gemm"][0] / k, clk["gemm"][0] / k
+                flops = 2.0 * M * params
+                bound_ms = max(flops / (tf_peak * 1e9), gemm_b / (hbm_peak * 1e6))
+                pt = {"B": B, "len": L, "n": n, "rows": M, "step_us": step_ms * 1e3,
+                      "attn_us_per_layer": attn_ms / ms.n_layers * 1e3, "attn_GBs": attn_b / attn_ms / 1e6,
+                      "attn_frac_of_measured": attn_b / attn_ms / 1e6 / hbm_peak, "attn_frac_of_8TBs": attn_b / attn_ms / 1e6 / HBM_NOMINAL_GBS,
+                      "gemm_ms_events": gemm_ev_ms, "gemm_ms_device_clock": gemm_ck_ms,
+                      "gemm_TFs": flops / gemm_ck_ms / 1e9, "gemm_frac_of_tensor_peak": flops / gemm_ck_ms / 1e9 / tf_peak,
+                      "gemm_weight_GBs": gemm_b / gemm_ck_ms / 1e6, "gemm_bound": "tensor" if flops / (tf_peak * 1e9) > gemm_b / (hbm_peak * 1e6) else "hbm",
+                      "gemm_frac_of_binding_roofline": bound_ms / gemm_ck_ms, "glue_ms_events": prof["glue"][0] / k}
+                assert eng.device_status() == 0
+                print(json.dumps(pt), flush=True)
+                points.append(pt)
+                eng.free_tree(th)
+            eng.close()
+            del eng, prompts
+            torch.cuda.empty_cache()
+    print(json.dumps({"sweep": "verify step, 7B shape, bf16", "points": len(points), "peaks": kind, "hbm_GBs": hbm_peak,
+                      "tensor_TFs": tf_peak, "iters": args.iters}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -536,6 +612,10 @@ def main():
     ap.add_argument("--n", type=int, default=64)
     ap.add_argument("--len", type=int, default=2048)
     ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--sweep", action="store_true", help="verify step alone over batch x KV length x tree nodes (7B shape)")
+    ap.add_argument("--sweep-B", default="1,2,4,8,16")
+    ap.add_argument("--sweep-len", default="512,2048,8192")
+    ap.add_argument("--sweep-n", default="16,32,64,128")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     rank = int(os.environ.get("RANK", 0))
@@ -545,6 +625,9 @@ def main():
         return
     if args.kernel:
         run_kernel(args)
+        return
+    if args.sweep:
+        run_sweep(args)
         return
     if world > 1:
         init_dist()
