@@ -59,7 +59,8 @@ extern "C" {
 #define CERB_MODE_AR  1        /* auto-regressive step: one-node tree          */
 
 #define CERB_PAGE        16    /* tokens per KV page                                  */
-#define CERB_MAX_NODES   128   /* tree nodes per sequence (2 x 64-bit ancestor words) */
+#define CERB_MAX_NODES   192   /* tree nodes per sequence; Sec. 5.1 uses up to 150 candidates + the root */
+#define CERB_ANC_WORDS   3     /* 64-bit words of one node's ancestor mask (CERB_MAX_NODES / 64)       */
 #define CERB_MAX_DEPTH   8     /* deepest node; an accepted path has <= 9 nodes       */
 #define CERB_MAX_HEADS   8     /* decoding heads                                      */
 #define CERB_MAX_LEVELS  8     /* Resblocks per decoding head                         */
@@ -84,7 +85,7 @@ typedef struct cerb_config {
   int32_t max_pages;             /* page-table columns per sequence: capacity = 16 * max_pages tokens */
   int32_t n_pool_pages;          /* physical pages per layer in each pool */
   int32_t max_batch;             /* <= CERB_MAX_BATCH */
-  int32_t max_nodes;             /* <= CERB_MAX_NODES; also the prefill chunk */
+  int32_t max_nodes;             /* <= CERB_MAX_NODES; prefill runs in chunks of min(max_nodes, 128) tokens */
   int32_t n_cheads;              /* Cerberus heads CH_0 .. CH_{n_cheads-1} */
   int32_t n_levels;              /* Resblocks per head */
   /* Section 4.1 wiring: concat_src[h][j] = -1 for the plain Resblock
@@ -223,7 +224,7 @@ typedef struct cerb_attn_args {
   const int32_t* page_table;    /* dev [B][max_pages] */
   const int32_t* len;           /* dev [B] prefix lengths; tree keys sit at slots len .. len+n-1 */
   const int32_t* n_active;      /* dev [B] or NULL (= n) */
-  const uint64_t* anc;          /* dev [n][2]: bit j (word j/64) set iff j is an ancestor of i or i itself */
+  const uint64_t* anc;          /* dev [n][CERB_ANC_WORDS]: bit j (word j/64) set iff j is an ancestor of i or i itself */
   void* out;                    /* dev [B][n][H][Dh] */
   float* lse;                   /* dev [B][H][n] or NULL */
   float scale;
@@ -253,7 +254,7 @@ int cerb_tree_attention(const cerb_attn_args* args, void* stream);
 #define CERB_STATIC_ATTN_SCRATCH_BYTES (16u << 20)
 int cerb_tree_attention_noalloc(const cerb_attn_args* args, void* stream);
 
-/* Ancestor bitmasks of a tree, the form cerb_tree_attention takes: anc_out host [n][2]. */
+/* Ancestor bitmasks of a tree, the form cerb_tree_attention takes: anc_out host [n][CERB_ANC_WORDS]. */
 int cerb_tree_ancestors(const int32_t* parent, int32_t n, uint64_t* anc_out);
 
 /* Stand-alone dense GEMM as the verification forward runs it (Algorithm 1, TL_i / LH):

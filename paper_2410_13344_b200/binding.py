@@ -22,7 +22,8 @@ OK = 0
 E_ARG, E_SHAPE, E_NOMEM, E_STATE, E_NONFINITE, E_TIMEOUT, E_CUDA = -1, -2, -3, -4, -5, -6, -7
 F32, BF16 = 0, 1
 MODE_PAR, MODE_AR = 0, 1
-PAGE, MAX_NODES, MAX_DEPTH, MAX_HEADS, MAX_LEVELS, MAX_TOPK, MAX_BATCH, MAX_TREES = 16, 128, 8, 8, 8, 16, 16, 8
+PAGE, MAX_NODES, MAX_DEPTH, MAX_HEADS, MAX_LEVELS, MAX_TOPK, MAX_BATCH, MAX_TREES = 16, 192, 8, 8, 8, 16, 16, 8
+ANC_WORDS = 3
 PATH_MAX = MAX_DEPTH + 1
 
 EXPORTS = [
@@ -172,7 +173,7 @@ def threshold_from_samples(S: Sequence[float], parallel_fraction: float) -> floa
 
 def tree_ancestors(parent: np.ndarray) -> np.ndarray:
     parent = np.ascontiguousarray(parent, np.int32)
-    out = np.zeros((parent.shape[0], 2), np.uint64)
+    out = np.zeros((parent.shape[0], ANC_WORDS), np.uint64)
     _check(lib().cerb_tree_ancestors(parent.ctypes.data, parent.shape[0], out.ctypes.data), "cerb_tree_ancestors")
     return out
 
@@ -371,7 +372,7 @@ def tree_attention(q: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.Tensor, 
                    lens: torch.Tensor, anc: torch.Tensor, scale: float, max_len: int,
                    n_active: Optional[torch.Tensor] = None, want_lse: bool = True, scratch: Optional[torch.Tensor] = None):
     """q [B][n][H][Dh]; pools [pages][H][16][Dh]; page_table [B][max_pages] int32; lens [B] int32;
-    anc [n][2] int64 bit patterns.  Returns (out, lse)."""
+    anc [n][ANC_WORDS] int64 bit patterns.  Returns (out, lse)."""
     B, n, H, Dh = q.shape
     dt = BF16 if q.dtype == torch.bfloat16 else F32
     out = torch.empty_like(q)

@@ -175,7 +175,7 @@ int tree_build(cerb_ctx* c, const int32_t* parent, const int32_t* head_of, const
   t->parent.assign(parent, parent + n);
   t->depth.assign(n, 0);
   std::vector<int32_t> hv(CERB_MAX_NODES, 0), rv(CERB_MAX_NODES, 0), pv(CERB_MAX_NODES, 0), dv(CERB_MAX_NODES, 0);
-  std::vector<uint64_t> anc(CERB_MAX_NODES * 2, 0);
+  std::vector<uint64_t> anc(CERB_MAX_NODES * CERB_ANC_WORDS, 0);
   int rc = cerb_tree_ancestors(parent, n, anc.data());
   if (rc != CERB_OK) { delete t; return rc; }
   t->max_depth = 0;
@@ -204,7 +204,7 @@ int tree_build(cerb_ctx* c, const int32_t* parent, const int32_t* head_of, const
             cudaMemcpy(t->dev.depth, dv.data(), ib, cudaMemcpyHostToDevice) == cudaSuccess &&
             cudaMemcpy(t->dev.head_of, hv.data(), ib, cudaMemcpyHostToDevice) == cudaSuccess &&
             cudaMemcpy(t->dev.rank_of, rv.data(), ib, cudaMemcpyHostToDevice) == cudaSuccess &&
-            cudaMemcpy(t->dev.anc, anc.data(), CERB_MAX_NODES * 2 * sizeof(uint64_t), cudaMemcpyHostToDevice) == cudaSuccess;
+            cudaMemcpy(t->dev.anc, anc.data(), CERB_MAX_NODES * CERB_ANC_WORDS * sizeof(uint64_t), cudaMemcpyHostToDevice) == cudaSuccess;
   if (!ok) { delete t; return CERB_E_CUDA; }
   *out = t;
   return CERB_OK;
@@ -328,16 +328,14 @@ int cerb_tree_ancestors(const int32_t* parent, int32_t n, uint64_t* anc_out) {
   if (!parent || !anc_out || n < 1 || n > CERB_MAX_NODES) return CERB_E_ARG;
   if (parent[0] != -1) return CERB_E_ARG;
   for (int v = 0; v < n; ++v) {
-    uint64_t a0 = 0, a1 = 0;
+    uint64_t* mine = anc_out + (size_t)v * CERB_ANC_WORDS;
+    for (int w = 0; w < CERB_ANC_WORDS; ++w) mine[w] = 0;
     if (v > 0) {
       int p = parent[v];
       if (p < 0 || p >= v) return CERB_E_ARG;
-      a0 = anc_out[p * 2];
-      a1 = anc_out[p * 2 + 1];
+      for (int w = 0; w < CERB_ANC_WORDS; ++w) mine[w] = anc_out[(size_t)p * CERB_ANC_WORDS + w];
     }
-    if (v < 64) a0 |= 1ull << v; else a1 |= 1ull << (v - 64);
-    anc_out[v * 2] = a0;
-    anc_out[v * 2 + 1] = a1;
+    mine[v >> 6] |= 1ull << (v & 63);
   }
   return CERB_OK;
 }
@@ -425,10 +423,11 @@ int cerb_load(const cerb_config* cfg, const cerb_weights* w, void* workspace_dev
       if ((rc = make_act_maps(&c->tm_hlast, c->d_hlast, CERB_MAX_BATCH, g.d_model)) != CERB_OK) break;
     }
     if ((rc = launch_rope_table(c, 0)) != CERB_OK) break;
-    std::vector<int32_t> par(g.max_nodes);
-    for (int v = 0; v < g.max_nodes; ++v) par[v] = v - 1;
+    const int chunk = g.max_nodes < kPrefillChunkMax ? g.max_nodes : kPrefillChunkMax;
+    std::vector<int32_t> par(chunk);
+    for (int v = 0; v < chunk; ++v) par[v] = v - 1;
     // the prefill chain is deeper than an acceptable path may be: no depth limit for it
-    if ((rc = tree_build(c, par.data(), nullptr, nullptr, g.max_nodes, CERB_MAX_TREES, false, false, &c->chain)) != CERB_OK) break;
+    if ((rc = tree_build(c, par.data(), nullptr, nullptr, chunk, CERB_MAX_TREES, false, false, &c->chain)) != CERB_OK) break;
     int32_t one = -1;
     if ((rc = tree_build(c, &one, nullptr, nullptr, 1, CERB_MAX_TREES + 1, false, true, &c->single)) != CERB_OK) break;
     if (cudaDeviceSynchronize() != cudaSuccess) { rc = CERB_E_CUDA; break; }
@@ -494,7 +493,7 @@ int cerb_prefill(cerb_ctx* c, const int32_t* tokens_dev, const int32_t* lens_hos
   CERB_CUDA_OK(cudaStreamSynchronize(st));
   for (int b = 0; b < B; ++b) c->h_stage[b] = lens_host[b];
   CERB_CUDA_OK(cudaMemcpyAsync(c->d_lens_in, c->h_stage, B * sizeof(int32_t), cudaMemcpyHostToDevice, st));
-  const int C = c->cfg.max_nodes;
+  const int C = c->chain->n;          // min(max_nodes, 128) tokens per chunk
   for (int off = 0; off < longest; off += C) {
     for (int b = 0; b < B; ++b) c->h_len[b] = lens_host[b] < off ? lens_host[b] : off;
     CERB_TRY(launch_set_nactive(c, 1, off, C, st));

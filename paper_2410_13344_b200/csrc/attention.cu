@@ -179,6 +179,9 @@ struct AttnParams {
   unsigned int* counters;   // [B*H]
   int32_t* status;
   int n, H, max_pages, nsplit, oob_row;
+  int row0, rows;           // query rows row0 .. row0 + rows - 1 of the tree are this launch's (q, out, lse and anc already point
+                            // at row0); a tree of more than 128 nodes takes two launches.  n stays the tree's node count
+                            // (the row stride between sequences); only keys below row0 + rows can be ancestors of these rows.
   int rows_pad;             // rows per split in `partial` (16, 32, 64 or 128)
   uint32_t v_lbo, v_sbo;    // byte offsets of the V operand's descriptor (tensor-core path)
   int cluster;              // tensor-core path: the splits of a (sequence, head) form one cluster and merge through shared memory
@@ -217,9 +220,10 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int L = p.len[b];
-  const int nq = p.n_active ? min(p.n_active[b], p.n) : p.n;
+  const int nq_all = p.n_active ? min(p.n_active[b], p.n) : p.n;      // live nodes of this sequence
+  const int nq = min(nq_all - p.row0, p.rows);                        // live query rows of this launch
   if (nq <= 0) return;
-  const int kv_total = L + nq;
+  const int kv_total = L + min(nq_all, p.row0 + p.rows);
   const int tiles = (kv_total + TILE - 1) / TILE;
   const int per = (tiles + p.nsplit - 1) / p.nsplit;
   const int t0 = min(tiles, split * per), t1 = min(tiles, t0 + per);
@@ -297,9 +301,12 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
         qa[kk][3] = r1 < nq ? *reinterpret_cast<const uint32_t*>(q1 + c + 8) : 0u;
       }
     }
-    uint64_t anc0[2] = {0, 0}, anc1[2] = {0, 0};
-    if (r0 < nq) { anc0[0] = p.anc[r0 * 2]; anc0[1] = p.anc[r0 * 2 + 1]; }
-    if (r1 < nq) { anc1[0] = p.anc[r1 * 2]; anc1[1] = p.anc[r1 * 2 + 1]; }
+    uint64_t anc0[CERB_ANC_WORDS], anc1[CERB_ANC_WORDS];
+#pragma unroll
+    for (int w = 0; w < CERB_ANC_WORDS; ++w) {
+      anc0[w] = r0 < nq ? p.anc[r0 * CERB_ANC_WORDS + w] : 0ull;
+      anc1[w] = r1 < nq ? p.anc[r1 * CERB_ANC_WORDS + w] : 0ull;
+    }
 
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
     float o[DH / 8][4];
@@ -357,7 +364,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
             if (!vis && kpos < kv_total) {
               int j = kpos - L;
               const uint64_t* a = (e < 2) ? anc0 : anc1;
-              vis = (a[j >> 6] >> (j & 63)) & 1ull;
+              vis = ((j < 64 ? a[0] : j < 128 ? a[1] : a[2]) >> (j & 63)) & 1ull;     // selects, not an indexed local array
             }
             if (!vis) v = -INFINITY;
           }
@@ -664,9 +671,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int L = p.len[b];
-  const int nq = p.n_active ? min(p.n_active[b], p.n) : p.n;
+  const int nq_all = p.n_active ? min(p.n_active[b], p.n) : p.n;      // live nodes of this sequence
+  const int nq = min(nq_all - p.row0, p.rows);                        // live query rows of this launch
   if (nq <= 0) return;
-  const int kv_total = L + nq;
+  const int kv_total = L + min(nq_all, p.row0 + p.rows);
   const int tiles = (kv_total + TILE - 1) / TILE;
   const int per = (tiles + p.nsplit - 1) / p.nsplit;
   const int t0 = min(tiles, split * per), t1 = min(tiles, t0 + per);
@@ -846,8 +854,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&q_ready));
     }
-    uint64_t anc0 = 0, anc1 = 0;
-    if (valid) { anc0 = p.anc[row * 2]; anc1 = p.anc[row * 2 + 1]; }
+    uint64_t anc0 = 0, anc1 = 0, anc2 = 0;
+    if (valid) { anc0 = p.anc[row * CERB_ANC_WORDS]; anc1 = p.anc[row * CERB_ANC_WORDS + 1]; anc2 = p.anc[row * CERB_ANC_WORDS + 2]; }
     const uint32_t s_addr = tmem + lane_base + (uint32_t)g * 64u;
     const uint32_t o_addr = tmem + lane_base + 128u + (uint32_t)g * 128u;
     uint8_t* ph = smem_gen + (p_base - smem_base) + (uint32_t)g * 2u * TC_P_BYTES + (uint32_t)row * 128u;
@@ -873,7 +881,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
           bool vis = kpos < L;
           if (!vis && kpos < kv_total) {
             const int t = kpos - L;
-            vis = ((t < 64 ? anc0 : anc1) >> (t & 63)) & 1ull;
+            vis = ((t < 64 ? anc0 : t < 128 ? anc1 : anc2) >> (t & 63)) & 1ull;
           }
           sc[j] = vis ? sc[j] * p.scale_log2 : -INFINITY;
           mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
@@ -1126,7 +1134,7 @@ __global__ void __launch_bounds__(128) tree_attn_f32_kernel(const float* __restr
   const int nq = n_active ? min(n_active[b], n) : n;
   if (i >= nq) return;
   const int L = len[b], warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint64_t a0 = anc[i * 2], a1 = anc[i * 2 + 1];
+  const uint64_t a0 = anc[i * CERB_ANC_WORDS], a1 = anc[i * CERB_ANC_WORDS + 1], a2 = anc[i * CERB_ANC_WORDS + 2];
   float qv[E], acc[E];
   const float* qp = q + (((size_t)b * n + i) * H + h) * DH;
   for (int e = 0; e < E; ++e) { qv[e] = qp[lane + 32 * e]; acc[e] = 0.f; }
@@ -1134,7 +1142,7 @@ __global__ void __launch_bounds__(128) tree_attn_f32_kernel(const float* __restr
   for (int kpos = warp; kpos < L + nq; kpos += 4) {
     if (kpos >= L) {
       int j = kpos - L;
-      if (!(((j < 64 ? a0 : a1) >> (j & 63)) & 1ull)) continue;
+      if (!(((j < 64 ? a0 : j < 128 ? a1 : a2) >> (j & 63)) & 1ull)) continue;
     }
     int page = page_table[(size_t)b * max_pages + kpos / CERB_PAGE];
     size_t off = (((size_t)page * H + h) * CERB_PAGE + kpos % CERB_PAGE) * DH;
@@ -1205,6 +1213,84 @@ size_t attn_scratch_bytes(int B, int n, int H, int Dh) {
   return kCounterBytes + rows * (size_t)nq_pad(n) * (size_t)(Dh + 4) * sizeof(float);
 }
 
+constexpr int kAttnRowsPerLaunch = 128;
+
+// One launch of the bf16 kernels over query rows row0 .. row0 + rows - 1 (rows <= 128) of every sequence's tree.
+static int launch_attn_window(const cerb_attn_args* a, int row0, int rows, const CUtensorMap* tmK, const CUtensorMap* tmV,
+                              int32_t* status, cudaStream_t st) {
+  AttnParams p;
+  const size_t row_elems = (size_t)a->n_heads * a->head_dim;
+  p.q = (const bf16*)a->q + (size_t)row0 * row_elems;
+  p.page_table = a->page_table;
+  p.len = a->len;
+  p.n_active = a->n_active;
+  p.anc = a->anc + (size_t)row0 * CERB_ANC_WORDS;
+  p.out = (bf16*)a->out + (size_t)row0 * row_elems;
+  p.lse = a->lse ? a->lse + row0 : nullptr;
+  p.row0 = row0;
+  p.rows = rows;
+  p.counters = (unsigned int*)a->scratch;
+  p.partial = (float*)((char*)a->scratch + kCounterBytes);
+  p.status = status;
+  p.n = a->n;
+  p.H = a->n_heads;
+  p.max_pages = a->max_pages;
+  // The tcgen05 kernel's MMAs are 128 rows tall: it takes the 65..128-node trees, and the 33..64-node trees
+  // from about 1K keys per sequence (measured inside the 7B decoding step, batch 1, ms per 64-node forward,
+  // tcgen05 against warp-MMA: 4.18 / 4.18 at 512 keys, 4.20 / 4.29 at 1K, 4.21 / 4.31 at 2K, 4.50 / 4.99 at
+  // 4K, 5.02 / 6.20 at 8K; kernel alone at 2 x 2K keys 29 / 45 us), and so do the 17..32-node trees (kernel
+  // alone 20 / 30 us at 2K keys, 43 / 68 us at 8K, 523 / 552 us at 16 x 8K).  Trees of up to 16 nodes and
+  // one-node steps stay on the warp-MMA kernel, whose 16-row layout wastes no tensor work and which streams
+  // at 7.0 TB/s at batch 16 x 8K keys (the tcgen05 kernel: 4.2).  CERB_ATTN_TC=0 / 1 forces one.
+  static const int force_tc = getenv("CERB_ATTN_TC") ? atoi(getenv("CERB_ATTN_TC")) : -1;
+  const int np_ = nq_pad(rows);
+  const bool auto_tc = np_ == 128 || ((np_ == 64 || np_ == 32) && a->max_len >= 1024);
+  const bool tensor_path = a->head_dim == 128 && (force_tc < 0 ? auto_tc : force_tc != 0);
+  // With clusters the splits of a (sequence, head) merge through distributed shared memory: at most 8 of them
+  // (the portable cluster size).  CERB_ATTN_CLUSTER=0 keeps the merge through global partials (up to 32 splits).
+  static const int use_cluster = getenv("CERB_ATTN_CLUSTER") ? atoi(getenv("CERB_ATTN_CLUSTER")) : 1;
+  // CTAs that fit at once: one per SM for the tensor-core kernel and for the warp-MMA layouts of 32 rows and more
+  // (288 threads x 168 registers), two per SM for the 16-row layout (160 threads); the grid is planned to fit one wave
+  const int resident = (tensor_path || np_ > 16) ? 148 : kTargetCtas;
+  p.nsplit = plan_nsplit(a->B, a->n_heads, nq_pad(rows), a->max_len, resident, true, use_cluster ? 8 : kMaxSplit);
+  if (p.nsplit < 1) return CERB_E_SHAPE;
+  p.oob_row = a->n_pool_pages * a->n_heads * CERB_PAGE;
+  p.scale_log2 = a->scale * 1.4426950408889634f;
+  p.rows_pad = nq_pad(rows);
+  p.cluster = (use_cluster && p.nsplit >= 2 && p.nsplit <= 8) ? 1 : 0;
+  // V tile in shared memory: [half of head_dim][64 keys][128 bytes]; 8-key groups are 1024 bytes apart
+  p.v_lbo = 8192u;
+  p.v_sbo = 1024u;
+  int np = nq_pad(rows), rc = CERB_E_SHAPE;
+  if (tensor_path) {
+    static bool configured = false;
+    if (!configured) {
+      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_tc_kernel<2, 5, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem(2, 5, 128)));
+      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_tc_kernel<5, 5, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem(5, 5, 64)));
+      configured = true;
+    }
+    auto kern = rows <= 64 ? tree_attn_tc_kernel<5, 5, 64, true> : tree_attn_tc_kernel<2, 5, 128, false>;
+    const size_t TC_SMEM = rows <= 64 ? tc_smem(5, 5, 64) : tc_smem(2, 5, 128);
+    if (p.cluster)
+      rc = launch_pdl_cluster(kern, dim3(p.nsplit, p.H, a->B), dim3(TC_THREADS), TC_SMEM, st, (unsigned)p.nsplit,
+                              *tmK, *tmV, p) == cudaSuccess ? CERB_OK : CERB_E_CUDA;
+    else
+      rc = launch_pdl(kern, dim3(p.nsplit, p.H, a->B), dim3(TC_THREADS), TC_SMEM, st, *tmK, *tmV, p) == cudaSuccess
+               ? CERB_OK : CERB_E_CUDA;
+  } else if (a->head_dim == 128) {
+    if (np == 16) rc = launch_cfg<128, 1, 4, 3>(p, tmK, tmV, a->B, st);
+    else if (np == 32) rc = launch_cfg<128, 2, 4, 3>(p, tmK, tmV, a->B, st);
+    else if (np == 64) rc = launch_cfg<128, 4, 2, 3>(p, tmK, tmV, a->B, st);
+    else rc = launch_cfg<128, 8, 1, 3>(p, tmK, tmV, a->B, st);
+  } else if (a->head_dim == 64) {
+    if (np == 16) rc = launch_cfg<64, 1, 4, 4>(p, tmK, tmV, a->B, st);
+    else if (np == 32) rc = launch_cfg<64, 2, 4, 4>(p, tmK, tmV, a->B, st);
+    else if (np == 64) rc = launch_cfg<64, 4, 2, 4>(p, tmK, tmV, a->B, st);
+    else rc = launch_cfg<64, 8, 1, 4>(p, tmK, tmV, a->B, st);
+  }
+  return rc;
+}
+
 int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMap* tmK, const CUtensorMap* tmV,
                           int sm_count, int32_t* status, cudaStream_t st) {
   (void)sm_count;
@@ -1224,76 +1310,16 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
     return CERB_OK;
   }
   if (a->B * a->n_heads > (int)(kCounterBytes / sizeof(unsigned int)) - 4) return CERB_E_SHAPE;   // last 16 bytes: status word
-  AttnParams p;
-  p.q = (const bf16*)a->q;
-  p.page_table = a->page_table;
-  p.len = a->len;
-  p.n_active = a->n_active;
-  p.anc = a->anc;
-  p.out = (bf16*)a->out;
-  p.lse = a->lse;
-  p.counters = (unsigned int*)a->scratch;
-  p.partial = (float*)((char*)a->scratch + kCounterBytes);
-  p.status = status;
-  p.n = a->n;
-  p.H = a->n_heads;
-  p.max_pages = a->max_pages;
-  // The tcgen05 kernel's MMAs are 128 rows tall: it takes the 65..128-node trees, and the 33..64-node trees
-  // from about 1K keys per sequence (measured inside the 7B decoding step, batch 1, ms per 64-node forward,
-  // tcgen05 against warp-MMA: 4.18 / 4.18 at 512 keys, 4.20 / 4.29 at 1K, 4.21 / 4.31 at 2K, 4.50 / 4.99 at
-  // 4K, 5.02 / 6.20 at 8K; kernel alone at 2 x 2K keys 29 / 45 us), and so do the 17..32-node trees (kernel
-  // alone 20 / 30 us at 2K keys, 43 / 68 us at 8K, 523 / 552 us at 16 x 8K).  Trees of up to 16 nodes and
-  // one-node steps stay on the warp-MMA kernel, whose 16-row layout wastes no tensor work and which streams
-  // at 7.0 TB/s at batch 16 x 8K keys (the tcgen05 kernel: 4.2).  CERB_ATTN_TC=0 / 1 forces one.
-  static const int force_tc = getenv("CERB_ATTN_TC") ? atoi(getenv("CERB_ATTN_TC")) : -1;
-  const int np_ = nq_pad(a->n);
-  const bool auto_tc = np_ == 128 || ((np_ == 64 || np_ == 32) && a->max_len >= 1024);
-  const bool tensor_path = a->head_dim == 128 && (force_tc < 0 ? auto_tc : force_tc != 0);
-  // With clusters the splits of a (sequence, head) merge through distributed shared memory: at most 8 of them
-  // (the portable cluster size).  CERB_ATTN_CLUSTER=0 keeps the merge through global partials (up to 32 splits).
-  static const int use_cluster = getenv("CERB_ATTN_CLUSTER") ? atoi(getenv("CERB_ATTN_CLUSTER")) : 1;
-  // CTAs that fit at once: one per SM for the tensor-core kernel and for the warp-MMA layouts of 32 rows and more
-  // (288 threads x 168 registers), two per SM for the 16-row layout (160 threads); the grid is planned to fit one wave
-  const int resident = (tensor_path || np_ > 16) ? 148 : kTargetCtas;
-  p.nsplit = plan_nsplit(a->B, a->n_heads, nq_pad(a->n), a->max_len, resident, true, use_cluster ? 8 : kMaxSplit);
-  if (p.nsplit < 1) return CERB_E_SHAPE;
-  p.oob_row = a->n_pool_pages * a->n_heads * CERB_PAGE;
-  p.scale_log2 = a->scale * 1.4426950408889634f;
-  p.rows_pad = nq_pad(a->n);
-  p.cluster = (use_cluster && p.nsplit >= 2 && p.nsplit <= 8) ? 1 : 0;
-  // V tile in shared memory: [half of head_dim][64 keys][128 bytes]; 8-key groups are 1024 bytes apart
-  p.v_lbo = 8192u;
-  p.v_sbo = 1024u;
   if (a->scratch_bytes < attn_scratch_bytes(a->B, a->n, a->n_heads, a->head_dim)) return CERB_E_NOMEM;
-  int np = nq_pad(a->n), rc = CERB_E_SHAPE;
-  if (tensor_path) {
-    static bool configured = false;
-    if (!configured) {
-      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_tc_kernel<2, 5, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem(2, 5, 128)));
-      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_tc_kernel<5, 5, 64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem(5, 5, 64)));
-      configured = true;
-    }
-    auto kern = a->n <= 64 ? tree_attn_tc_kernel<5, 5, 64, true> : tree_attn_tc_kernel<2, 5, 128, false>;
-    const size_t TC_SMEM = a->n <= 64 ? tc_smem(5, 5, 64) : tc_smem(2, 5, 128);
-    if (p.cluster)
-      rc = launch_pdl_cluster(kern, dim3(p.nsplit, p.H, a->B), dim3(TC_THREADS), TC_SMEM, st, (unsigned)p.nsplit,
-                              *tmK, *tmV, p) == cudaSuccess ? CERB_OK : CERB_E_CUDA;
-    else
-      rc = launch_pdl(kern, dim3(p.nsplit, p.H, a->B), dim3(TC_THREADS), TC_SMEM, st, *tmK, *tmV, p) == cudaSuccess
-               ? CERB_OK : CERB_E_CUDA;
-  } else if (a->head_dim == 128) {
-    if (np == 16) rc = launch_cfg<128, 1, 4, 3>(p, tmK, tmV, a->B, st);
-    else if (np == 32) rc = launch_cfg<128, 2, 4, 3>(p, tmK, tmV, a->B, st);
-    else if (np == 64) rc = launch_cfg<128, 4, 2, 3>(p, tmK, tmV, a->B, st);
-    else rc = launch_cfg<128, 8, 1, 3>(p, tmK, tmV, a->B, st);
-  } else if (a->head_dim == 64) {
-    if (np == 16) rc = launch_cfg<64, 1, 4, 4>(p, tmK, tmV, a->B, st);
-    else if (np == 32) rc = launch_cfg<64, 2, 4, 4>(p, tmK, tmV, a->B, st);
-    else if (np == 64) rc = launch_cfg<64, 4, 2, 4>(p, tmK, tmV, a->B, st);
-    else rc = launch_cfg<64, 8, 1, 4>(p, tmK, tmV, a->B, st);
+  // A CTA holds at most 128 query rows (the tensor-core MMA's height, eight 16-row warps in the warp-MMA kernel).
+  // A wider tree (Sec. 5.1 goes up to 150 candidates + the root) takes one launch per window of 128 rows; the
+  // launches are stream-ordered and share the scratch.  Keys are not windowed: rows of the second window see the
+  // whole tree, rows of the first only nodes below 128 (an ancestor has a lower index than its descendant).
+  for (int row0 = 0; row0 < a->n; row0 += kAttnRowsPerLaunch) {
+    const int rows = a->n - row0 < kAttnRowsPerLaunch ? a->n - row0 : kAttnRowsPerLaunch;
+    CERB_TRY(launch_attn_window(a, row0, rows, tmK, tmV, status, st));
+    CERB_LAUNCH_CHECK(c);
   }
-  if (rc != CERB_OK) return rc;
-  CERB_LAUNCH_CHECK(c);
   return CERB_OK;
 }
 

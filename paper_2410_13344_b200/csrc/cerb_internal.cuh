@@ -79,6 +79,7 @@ inline cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 
 }
 
 constexpr int kPathMax = CERB_MAX_DEPTH + 1;
+constexpr int kPrefillChunkMax = 128;   // prompt tokens per prefill chunk (a chain-shaped tree), whatever max_nodes is
 constexpr int kGemmRowsPerPass = 256;   // activation rows one tcgen05 pass covers (the MMA's N extent)
 constexpr int kGemmMaxSplit = 16;
 
@@ -88,9 +89,9 @@ struct TreeDev {
   int32_t* depth;
   int32_t* head_of;
   int32_t* rank_of;
-  uint64_t* anc;     // [CERB_MAX_NODES][2]
+  uint64_t* anc;     // [CERB_MAX_NODES][CERB_ANC_WORDS]
 };
-constexpr size_t kTreeSlotBytes = 4 * CERB_MAX_NODES * sizeof(int32_t) + CERB_MAX_NODES * 2 * sizeof(uint64_t);
+constexpr size_t kTreeSlotBytes = 4 * CERB_MAX_NODES * sizeof(int32_t) + CERB_MAX_NODES * CERB_ANC_WORDS * sizeof(uint64_t);
 
 // Tensor maps for one activation buffer used as the MMA's B operand, one per row bucket.
 constexpr int kRowBuckets = 5;          // 16, 32, 64, 128, 256 rows

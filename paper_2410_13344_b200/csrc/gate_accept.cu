@@ -53,12 +53,12 @@ __global__ void __launch_bounds__(256) gate_kernel(const T* __restrict__ h_last,
   }
 }
 
-// One CTA of 128 threads per sequence, thread v <-> node v.
+// One CTA of 192 threads (CERB_MAX_NODES) per sequence, thread v <-> node v.
 //   match[v] = token of v equals the model's argmax at v's parent   (root: always)
 //   v is accepted-reachable iff every node on its root path matches: (anc[v] & ~match) == 0
 //   winner = deepest reachable node, lowest index among equals; its ancestors, ascending, are the path.
 template <typename T>
-__global__ void __launch_bounds__(128) accept_kernel(const int32_t* __restrict__ tok, const int32_t* __restrict__ argmax,
+__global__ void __launch_bounds__(CERB_MAX_NODES) accept_kernel(const int32_t* __restrict__ tok, const int32_t* __restrict__ argmax,
                                                      const int32_t* __restrict__ n_active,
                                                      const int32_t* __restrict__ parent, const int32_t* __restrict__ depth,
                                                      const uint64_t* __restrict__ anc, int n, int32_t* __restrict__ len,
@@ -66,8 +66,9 @@ __global__ void __launch_bounds__(128) accept_kernel(const int32_t* __restrict__
                                                      const T* __restrict__ hidden, T* __restrict__ h_last, int d,
                                                      int32_t* __restrict__ n_accept, int32_t* __restrict__ path,
                                                      int32_t* __restrict__ out_tok) {
-  __shared__ uint32_t mword[4];
-  __shared__ int skey[4];
+  constexpr int NWARP = CERB_MAX_NODES / 32;
+  __shared__ uint32_t mword[NWARP];
+  __shared__ int skey[NWARP];
   __shared__ int best_s;
   griddep_wait();
   griddep_launch();
@@ -79,23 +80,28 @@ __global__ void __launch_bounds__(128) accept_kernel(const int32_t* __restrict__
   uint32_t bal = __ballot_sync(0xffffffffu, match);
   if ((v & 31) == 0) mword[v >> 5] = bal;
   __syncthreads();
-  uint64_t mm0 = (uint64_t)mword[0] | ((uint64_t)mword[1] << 32), mm1 = (uint64_t)mword[2] | ((uint64_t)mword[3] << 32);
+  uint64_t mm[CERB_ANC_WORDS];
+#pragma unroll
+  for (int w = 0; w < CERB_ANC_WORDS; ++w) mm[w] = (uint64_t)mword[2 * w] | ((uint64_t)mword[2 * w + 1] << 32);
   int key = -1;
   if (v < na) {
-    uint64_t a0 = anc[v * 2], a1 = anc[v * 2 + 1];
-    if ((a0 & ~mm0) == 0 && (a1 & ~mm1) == 0) key = depth[v] * 256 + (255 - v);
+    bool reach = true;
+#pragma unroll
+    for (int w = 0; w < CERB_ANC_WORDS; ++w) reach = reach && (anc[v * CERB_ANC_WORDS + w] & ~mm[w]) == 0;
+    if (reach) key = depth[v] * 256 + (255 - v);
   }
   for (int o = 16; o > 0; o >>= 1) key = max(key, __shfl_xor_sync(0xffffffffu, key, o));
   if ((v & 31) == 0) skey[v >> 5] = key;
   __syncthreads();
   if (v == 0) {
-    int k = max(max(skey[0], skey[1]), max(skey[2], skey[3]));
+    int k = skey[0];
+#pragma unroll
+    for (int w = 1; w < NWARP; ++w) k = max(k, skey[w]);
     int best = k < 0 ? 0 : 255 - (k & 255);
     best_s = best;
-    uint64_t a[2] = {anc[best * 2], anc[best * 2 + 1]};
     int cnt = 0;
-    for (int w = 0; w < 2; ++w) {
-      uint64_t bits = a[w];
+    for (int w = 0; w < CERB_ANC_WORDS; ++w) {
+      uint64_t bits = anc[best * CERB_ANC_WORDS + w];
       while (bits && cnt < kPathMax) {
         int j = __ffsll((long long)bits) - 1;
         bits &= bits - 1;
@@ -173,11 +179,11 @@ int launch_accept(cerb_ctx* c, const cerb_tree* tree, const int32_t* tree_tok, c
   const cerb_config& g = c->cfg;
   const TreeDev& t = tree->dev;
   if (c->bf16)
-    accept_kernel<bf16><<<c->B, 128, 0, st>>>(tree_tok, node_argmax, n_active, t.parent, t.depth, t.anc, tree->n, c->d_len,
+    accept_kernel<bf16><<<c->B, CERB_MAX_NODES, 0, st>>>(tree_tok, node_argmax, n_active, t.parent, t.depth, t.anc, tree->n, c->d_len,
                                               c->d_len_old, c->d_root, (const bf16*)c->d_hidden, (bf16*)c->d_hlast,
                                               g.d_model, n_accept, path, out_tok);
   else
-    accept_kernel<float><<<c->B, 128, 0, st>>>(tree_tok, node_argmax, n_active, t.parent, t.depth, t.anc, tree->n, c->d_len,
+    accept_kernel<float><<<c->B, CERB_MAX_NODES, 0, st>>>(tree_tok, node_argmax, n_active, t.parent, t.depth, t.anc, tree->n, c->d_len,
                                                c->d_len_old, c->d_root, (const float*)c->d_hidden, (float*)c->d_hlast,
                                                g.d_model, n_accept, path, out_tok);
   CERB_LAUNCH_CHECK(c);

@@ -29,7 +29,13 @@ def test_host_only_calls_work_without_a_gpu():
     import numpy as np
     assert binding.strerror(binding.E_TIMEOUT) == "a bounded device-side wait ran out"
     anc = binding.tree_ancestors(synth.chain_tree(70).parent)
-    assert int(anc[69, 0]) == (1 << 64) - 1 and int(anc[69, 1]) == (1 << 6) - 1
+    assert anc.shape == (70, binding.ANC_WORDS)
+    assert int(anc[69, 0]) == (1 << 64) - 1 and int(anc[69, 1]) == (1 << 6) - 1 and int(anc[69, 2]) == 0
+    wide = binding.tree_ancestors(synth.chain_tree(151).parent)       # 150 candidates + root (Sec. 5.1)
+    assert [int(x) for x in wide[150]] == [(1 << 64) - 1, (1 << 64) - 1, (1 << 23) - 1]
+    star = np.array([-1] + [0] * 191, np.int32)                       # the largest tree: every node a child of the root
+    s = binding.tree_ancestors(star)
+    assert [int(x) for x in s[191]] == [1, 0, 1 << 63] and [int(x) for x in s[64]] == [1, 1, 0]
     cfg = binding.make_config(synth.shape_7b(), synth.cerberus_layout(4), [10] * 4, 200, 200, 1, 64)
     nbytes = binding.workspace_bytes(cfg)
     assert 10 << 20 < nbytes < 2 << 30

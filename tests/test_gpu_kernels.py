@@ -108,6 +108,11 @@ ATTN_CASES = [
     (4, 64, 2, 128, [2100, 2000, 1900, 2047], 5),   # ... batch of four, ragged
     (1, 128, 8, 128, [3000], 6),        # ... three splits
     (2, 100, 16, 128, [2500, 77], 5),   # ... ragged: the short sequence leaves most splits without keys
+    (1, 151, 4, 128, [1500], 4),        # 150 candidate paths + root (the paper's widest tree, Sec. 5.1): three ancestor
+                                        # words, two launches of query rows (128 + 23), both on the tcgen05 kernel
+    (2, 192, 2, 128, [300, 77], 6),     # the largest tree the library takes; short caches: second window on the warp-MMA kernel
+    (2, 151, 2, 64, [500, 100], 5),     # head_dim 64: warp-MMA kernel for both windows
+    (3, 140, 3, 128, [2000, 1, 640], 6),
 ]
 
 
@@ -150,13 +155,23 @@ def test_tree_attention_bf16_partial_activity_on_the_tensor_core_path(cb):
         assert close(got_o, O, 0) < TOL_BF16 and close(got_l, l, 0) < 2e-3
 
 
+def test_tree_attention_bf16_partial_activity_beyond_128_nodes(cb):
+    """151-node tree, live node counts on either side of the 128-row boundary between the two launches:
+    the second launch has 23, 2 and no live rows."""
+    res = _attention_case(cb, "bf16", 3, 151, 4, 128, [1400, 90, 1100], 5, seed_id=43, n_active=[151, 130, 5])
+    assert len(res) == 3
+    for got_o, got_l, O, l in res:
+        assert close(got_o, O, 0) < TOL_BF16 and close(got_l, l, 0) < 2e-3
+
+
 def test_tree_attention_bf16_is_deterministic(cb):
     a = _attention_case(cb, "bf16", 1, 64, 8, 128, [3000], 5, seed_id=41)[0]
     b = _attention_case(cb, "bf16", 1, 64, 8, 128, [3000], 5, seed_id=41)[0]
     assert torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
 
 
-@pytest.mark.parametrize("case", [(1, 16, 4, 64, [64], 4), (2, 40, 2, 128, [33, 5], 5), (1, 128, 2, 64, [10], 6)])
+@pytest.mark.parametrize("case", [(1, 16, 4, 64, [64], 4), (2, 40, 2, 128, [33, 5], 5), (1, 128, 2, 64, [10], 6),
+                                  (2, 151, 2, 64, [40, 3], 6)])
 def test_tree_attention_f32(cb, case):
     B, n, H, Dh, lens, md = case
     for got_o, got_l, O, l in _attention_case(cb, "fp32", B, n, H, Dh, lens, md, seed_id=50 + n):
@@ -166,7 +181,7 @@ def test_tree_attention_f32(cb, case):
 def test_abi_rejects_bad_arguments(cb):
     L = cb.lib()
     assert L.cerb_tree_attention(None, None) == cb.E_ARG
-    out = np.zeros((4, 2), np.uint64)
+    out = np.zeros((4, cb.ANC_WORDS), np.uint64)
     bad = np.array([-1, 0, 3, 1], np.int32)       # parent after child
     assert L.cerb_tree_ancestors(bad.ctypes.data, 4, out.ctypes.data) == cb.E_ARG
     good = np.array([-1, 0, 0, 1], np.int32)

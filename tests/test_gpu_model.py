@@ -350,6 +350,55 @@ def test_profiling_modes(cb):
     assert eng.device_status() == 0
 
 
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_151_node_trees(cb, dtype):
+    """The paper's widest setting (Sec. 5.1: top-10 per head, 150 candidate paths + the root): three ancestor
+    words, attention in two launches of query rows.  Planted candidates; the run must emit the auto-regressive
+    greedy continuation, and one verification forward must agree with the oracle node by node."""
+    ms = synth.tiny_shape(dtype)
+    rig = Rig(cb, ms, max_batch=2, max_tokens=400, max_nodes=160, topk=(10, 10, 10, 10))
+    eng = rig.eng
+    tree = synth.best_first_tree(151, rig.topk)
+    th = eng.tree(tree)
+    lens = [150, 37]
+    prompts = [[int(t) for t in synth.make_prompt(ms.vocab, L, seq=60 + b)] for b, L in enumerate(lens)]
+    tok = torch.zeros(2, max(lens), dtype=torch.int32, device="cuda")
+    for b, p in enumerate(prompts):
+        tok[b, :len(p)] = torch.tensor(p, dtype=torch.int32)
+    eng.prefill(tok, lens)
+    # one verification forward against the oracle's per-node definition (explicit root-to-node sequences)
+    tt = torch.stack([synth.make_prompt(ms.vocab, 151, seq=70 + b).to(torch.int32) for b in range(2)]).cuda().contiguous()
+    am, logits, _ = eng.verify(th, tt, want_logits=True)
+    torch.cuda.synchronize()
+    tol = 1e-4 if dtype == "fp32" else 2e-2
+    for b in range(2):
+        st = orc.prefill(rig.cmodel, rig.sh, prompts[b], 600)
+        _, want = orc.verify_tree(rig.cmodel, rig.sh, st, [int(t) for t in tt[b]], tree.parent)
+        assert close(logits[b], want, 0) < tol, b
+        for v in (0, 63, 64, 127, 128, 150):
+            assert int(am[b, v]) == int(orc.argmax_f32(logits[b, v].cpu().reshape(1, -1))[0]), (b, v)
+    if dtype == "fp32":
+        n_new = 8
+        truths = [orc.ar_greedy(rig.cmodel, rig.sh, p, n_new + 6)[0] for p in prompts]
+        eng.prefill(tok, lens)
+        outs = [[], []]
+        best = 0
+        for step in range(n_new):
+            plant = torch.tensor([plant_tokens(tree, truths[b], len(outs[b]), 1 + (step + b) % 5) for b in range(2)],
+                                 dtype=torch.int32, device="cuda")
+            eng.step(th, 1e9, plant)
+            torch.cuda.synchronize()
+            for b in range(2):
+                na = int(eng.h_n_accept[b])
+                best = max(best, na)
+                outs[b].extend(int(t) for t in eng.h_tokens[b, :na])
+        for b in range(2):
+            k = min(len(outs[b]), n_new + 6)
+            assert outs[b][:k] == truths[b][:k], b
+        assert best >= 4
+    assert eng.device_status() == 0
+
+
 def test_error_codes(cb):
     ms = synth.tiny_shape("fp32")
     rig = Rig(cb, ms, max_tokens=128)
