@@ -24,7 +24,10 @@ def cb():
 
 @pytest.mark.parametrize("M,N,K", [(64, 256, 512), (1, 128, 64), (16, 688, 256), (64, 256, 688), (100, 1000, 1024),
                                    (300, 384, 320), (64, 4096, 4096), (7, 130, 72),
-                                   (2048, 640, 512), (1000, 11008, 256), (129, 256, 11008)])
+                                   (2048, 640, 512), (1000, 11008, 256), (129, 256, 11008),
+                                   # row chunks of 256 walked side by side: 3 chunks (49 groups), 6 ragged chunks,
+                                   # and more chunks than half the SMs (back to the plain unit list)
+                                   (513, 1536, 384), (1281, 300, 1024), (19201, 128, 64)])
 def test_gemm_bf16_matches_definition(cb, M, N, K):
     X = synth.normal(11, 1, (M, K), 1.0, dtype=torch.bfloat16, device="cuda")
     W = synth.normal(11, 2, (N, K), 0.05, dtype=torch.bfloat16, device="cuda")
