@@ -493,7 +493,10 @@ def run_kernel(args):
         us = timeit(lambda i: cb.gemm(X, Ws[i % nrot], scratch))
         byts = (N * K + M * K) * 2 + M * N * 4
         out = {"kernel": "gemm", "M": M, "N": N, "K": K, "us": us, "GBs": byts / us / 1e3, "frac_hbm": byts / us / 1e3 / hbm_peak,
-               "TFs": 2.0 * M * N * K / us / 1e6, "frac_tensor": 2.0 * M * N * K / us / 1e6 / tf_peak, "peaks": kind, "rotating_buffers": nrot}
+               "TFs": 2.0 * M * N * K / us / 1e6, "frac_tensor": 2.0 * M * N * K / us / 1e6 / tf_peak, "peaks": kind, "rotating_buffers": nrot,
+               "note": "per-call time of cerb_gemm = the GEMM kernel plus the kernel that sums its fp32 partial slots into one "
+                       "matrix; from a few hundred rows on the second one is a large part (the step's own consumers read the "
+                       "slots directly) -- for the GEMM kernel alone see --sweep (device-clock spans) or the ncu summaries"}
     else:
         B, n, L, H, Dh = args.B, args.n, args.len, 32, 128
         max_len = L + n
