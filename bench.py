@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the Cerberus decoding step on a 7B-shaped, random-init bf16 model.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl cerb|reference] [--workload 7b|tiny]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl cerb|reference] [--workload 7b|13b|tiny]
     python bench.py --sweep            # verify step alone over batch x KV length x tree nodes
 
 A "step" is one whole decoding step (gate, draft when the gate allows it, tree verification
@@ -41,9 +41,20 @@ GEMM_TRAFFIC = 186.4e6
 GEMM_TRAFFIC_NOTE = {"launch": "M=64 N=22016 K=4096", "algorithmic_bytes_per_launch": 183.7e6}
 
 
+def draft_setup(name: str):
+    """(decoding heads, top-k per head, tree nodes) of a workload."""
+    if name == "7b":
+        return 4, TOPK, N_NODES
+    if name == "13b":
+        return 5, [10] * 5, N_NODES
+    return 4, [4, 2, 1, 1], 16
+
+
 def workload(name: str):
     if name == "7b":
         return synth.shape_7b(), PROMPT_LEN, "7B-shaped bf16 model, 4 Cerberus heads, 64-node tree, 2048-token prompt, batch 1"
+    if name == "13b":
+        return synth.shape_13b(), 4096, "13B-shaped bf16 model, 5 Cerberus heads, 64-node tree, 4096-token prompt, batch 1"
     if name == "tiny":
         ms = synth.tiny_shape("bf16")
         return ms, 64, "tiny bf16 model (debug)"
@@ -147,9 +158,8 @@ def run_cerb(args, rank, world):
     ms, prompt_len, wl_name = workload(args.workload)
     # comparison modes (Sec. 5): "medusa" = independent heads without the sequential link and no gate,
     # "no-gate" = Cerberus heads, every step parallel, "ar" = plain auto-regressive decoding
-    layout = synth.medusa_layout(4, 4) if args.mode == "medusa" else synth.cerberus_layout(4, 4)
-    topk = TOPK if args.workload == "7b" else [4, 2, 1, 1]
-    n_nodes = N_NODES if args.workload == "7b" else 16
+    n_ch, topk, n_nodes = draft_setup(args.workload)
+    layout = synth.medusa_layout(n_ch, 4) if args.mode == "medusa" else synth.cerberus_layout(n_ch, 4)
     t_setup = time.time()
     model = synth.make_model(ms, device="cuda")
     heads = synth.make_heads(ms, layout, device="cuda")
@@ -324,11 +334,11 @@ def run_cerb(args, rank, world):
     gemm_flops = sum(2 * M * gemm_params for M in n_b)
     par_steps = [i for i, m in enumerate(modes_a) if m == 0]
     line = {
-        "metric": METRIC, "value": agg(tok_a) / (ms_a / 1e3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC.replace("7B", "13B") if args.workload == "13b" else METRIC, "value": agg(tok_a) / (ms_a / 1e3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_a / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": wl_name, "mode": args.mode, "parallelism": "replicas" if world > 1 else "single",
-                   "l2": "every step streams > 13 GB of weights, far beyond the 126 MB L2",
+                   "l2": "every step streams the model's weights (13 GB at the 7B shape), far beyond the 126 MB L2",
                    "threshold": T, "tree_nodes": n_nodes, "topk": topk, "prompt_len": prompt_len,
                    "acceptance": "natural (random-init heads)"},
         "verify_step_latency_us": ms_a / args.steps * 1e3,
@@ -418,9 +428,8 @@ def run_reference(args, rank, world):
     if rank != 0:
         return
     ms, prompt_len, wl_name = workload(args.workload)
-    layout = synth.cerberus_layout(4, 4)
-    topk = TOPK if args.workload == "7b" else [4, 2, 1, 1]
-    n_nodes = N_NODES if args.workload == "7b" else 16
+    n_ch, topk, n_nodes = draft_setup(args.workload)
+    layout = synth.cerberus_layout(n_ch, 4)
     tree = synth.best_first_tree(n_nodes, topk)
     # one layer of the model (the sample) plus embedding / LM head, generated on the host
     # (values do not matter for timing; a seeded torch generator is much faster on the host than the
@@ -532,7 +541,7 @@ def run_sweep(args):
     __graft_entry__.build()
     torch.cuda.set_device(0)
     hbm_peak, tf_peak, kind = peaks()
-    ms = synth.shape_7b()
+    ms = synth.shape_13b() if args.workload == "13b" else synth.shape_7b()
     model = synth.make_model(ms, device="cuda")
     HD = ms.n_heads * ms.head_dim
     params = ms.n_layers * (3 * HD * ms.d_model + ms.d_model * HD + 3 * ms.mlp_dim * ms.d_model) + ms.vocab * ms.d_model
@@ -592,7 +601,7 @@ def run_sweep(args):
             eng.close()
             del eng, prompts
             torch.cuda.empty_cache()
-    print(json.dumps({"sweep": "verify step, 7B shape, bf16", "points": len(points), "peaks": kind, "hbm_GBs": hbm_peak,
+    print(json.dumps({"sweep": "verify step, %s shape, bf16" % ("13B" if args.workload == "13b" else "7B"), "points": len(points), "peaks": kind, "hbm_GBs": hbm_peak,
                       "tensor_TFs": tf_peak, "iters": args.iters}))
 
 
