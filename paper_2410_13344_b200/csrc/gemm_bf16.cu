@@ -451,7 +451,7 @@ struct GemmPlan {
   long long total;   // checked to fit 31 bits before launch
 };
 
-// Tuning switches (environment, read once): CERB_GEMM_WIDE, CERB_GEMM_GROUP, CERB_GEMM_HINT.
+// Tuning switches (environment, read once): CERB_GEMM_WIDE, CERB_GEMM_LOCK, CERB_GEMM_GROUP, CERB_GEMM_HINT.
 int tune(const char* name, int dflt) {
   const char* v = getenv(name);
   return v ? atoi(v) : dflt;
