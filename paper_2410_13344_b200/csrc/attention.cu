@@ -167,6 +167,22 @@ __device__ __forceinline__ float4 ld_cluster_v4(uint32_t a) {
 }
 __device__ __forceinline__ void compute_bar(int nthreads) { asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory"); }
 
+// Which of the 64 keys key0 .. key0 + 63 one query row may see, as a bit mask (bit j <-> key key0 + j): prefix keys
+// (position < L) always, tree keys by the row's ancestor words a0, a1, a2 (tree index = position - L).  Ancestor
+// words have no bits at or above the live node count, so keys past the last live tree key come out invisible.
+// Called only for tiles that reach past the prefix (key0 + 64 > L).
+__device__ __forceinline__ uint64_t tile_visibility(int key0, int L, uint64_t a0, uint64_t a1, uint64_t a2) {
+  const int base = key0 - L;                       // tree index of the tile's first key; negative: the tile starts in the prefix
+  if (base < 0) {
+    const int s = -base;                           // 1 .. 63 prefix keys, then tree keys 0 .. 63 - s
+    return (a0 << s) | ((1ull << s) - 1ull);
+  }
+  const int w = base >> 6, sh = base & 63;
+  const uint64_t lo = w == 0 ? a0 : w == 1 ? a1 : w == 2 ? a2 : 0ull;
+  const uint64_t hi = w == 0 ? a1 : w == 1 ? a2 : 0ull;
+  return sh ? (lo >> sh) | (hi << (64 - sh)) : lo;
+}
+
 struct AttnParams {
   const bf16* q;
   const int32_t* page_table;
@@ -352,6 +368,11 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
 
       // ---- mask, online softmax ----
       const bool need_mask = key_tile0 + TILE > L;
+      uint64_t vm0 = ~0ull, vm1 = ~0ull;             // visible keys of this tile for rows r0 and r1
+      if (need_mask) {
+        vm0 = tile_visibility(key_tile0, L, anc0[0], anc0[1], anc0[2]);
+        vm1 = tile_visibility(key_tile0, L, anc1[0], anc1[1], anc1[2]);
+      }
       float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
       for (int nt = 0; nt < NT; ++nt) {
@@ -359,14 +380,8 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
         for (int e = 0; e < 4; ++e) {
           float v = sc[nt][e] * p.scale_log2;
           if (need_mask) {
-            int kpos = key_tile0 + ki * KW + nt * 8 + tq * 2 + (e & 1);
-            bool vis = kpos < L;
-            if (!vis && kpos < kv_total) {
-              int j = kpos - L;
-              const uint64_t* a = (e < 2) ? anc0 : anc1;
-              vis = ((j < 64 ? a[0] : j < 128 ? a[1] : a[2]) >> (j & 63)) & 1ull;     // selects, not an indexed local array
-            }
-            if (!vis) v = -INFINITY;
+            const int j = ki * KW + nt * 8 + tq * 2 + (e & 1);          // key's index inside the tile
+            if (!((((e < 2) ? vm0 : vm1) >> j) & 1ull)) v = -INFINITY;
           }
           sc[nt][e] = v;
           if (e < 2) mx0 = fmaxf(mx0, v); else mx1 = fmaxf(mx1, v);
@@ -875,14 +890,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       const int key0 = (t0 + i) * TILE;
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
       if (key0 + TILE > L) {
+        const uint64_t vm = tile_visibility(key0, L, anc0, anc1, anc2);
+        const uint32_t vm_lo = (uint32_t)vm, vm_hi = (uint32_t)(vm >> 32);
 #pragma unroll
         for (int j = 0; j < 64; ++j) {
-          const int kpos = key0 + j;
-          bool vis = kpos < L;
-          if (!vis && kpos < kv_total) {
-            const int t = kpos - L;
-            vis = ((t < 64 ? anc0 : t < 128 ? anc1 : anc2) >> (t & 63)) & 1ull;
-          }
+          const bool vis = ((j < 32 ? vm_lo >> j : vm_hi >> (j - 32)) & 1u) != 0u;      // j is a constant after unrolling
           sc[j] = vis ? sc[j] * p.scale_log2 : -INFINITY;
           mx4[j & 3] = fmaxf(mx4[j & 3], sc[j]);
         }
