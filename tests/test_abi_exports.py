@@ -53,3 +53,32 @@ def test_threshold_from_samples_splits_the_requested_fraction():
     for frac, below in ((0.5, 5), (0.7, 7), (0.1, 1), (0.0, 1), (1.0, 9)):
         T = binding.threshold_from_samples(S, frac)
         assert sum(1 for v in S if v <= T) == below and T not in S
+
+
+def _slots_by_the_stated_schedule(M, N, K, sms=148):
+    """Partial slots per output element of the bf16 GEMM, from its schedule as documented: units are (256-row weight
+    tile, 64-wide k block) pairs; rows beyond 256 form row chunks; with 2..74 chunks the unit list of ONE chunk is cut
+    into floor(148 / chunks) contiguous shares (one CTA per chunk walks each share), otherwise the list over all
+    chunks is cut into 148 shares; a share has at least min(k blocks, 4) units; a tile's slots = shares it touches."""
+    tiles, kb, chunks = -(-N // 256), -(-K // 64), -(-M // 256)
+    grouped = 1 < chunks <= sms // 2
+    jobs = tiles if grouped else tiles * chunks
+    shares = sms // chunks if grouped else sms
+    per = max(-(-jobs * kb // shares), min(kb, 4))
+    return max((j * kb + kb - 1) // per - (j * kb) // per + 1 for j in range(jobs))
+
+
+def test_gemm_scratch_size_follows_the_documented_schedule():
+    import ctypes as C
+    from paper_2410_13344_b200 import binding
+    L = binding.lib()
+    shapes = [(1, 128, 64), (16, 22016, 4096), (64, 4096, 4096), (64, 22016, 4096), (64, 12288, 4096), (64, 32000, 4096),
+              (128, 4096, 11008), (256, 22016, 4096), (300, 384, 320), (512, 4096, 4096), (513, 1536, 384),
+              (1024, 12288, 4096), (1281, 300, 1024), (2048, 22016, 4096), (2048, 4096, 11008), (2048, 32000, 4096),
+              (19201, 128, 64), (64, 27648, 5120), (256, 5120, 13824)]
+    for M, N, K in shapes:
+        nb = C.c_size_t(0)
+        assert L.cerb_gemm_scratch_bytes(M, N, K, C.byref(nb)) == binding.OK
+        assert nb.value == 256 + _slots_by_the_stated_schedule(M, N, K) * M * N * 4, (M, N, K)
+    # weights leave HBM once at 2048 rows: 8 row chunks share 18 groups, a 64-block tile touches at most 2 shares
+    assert _slots_by_the_stated_schedule(2048, 22016, 4096) == 2
