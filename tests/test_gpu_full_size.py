@@ -213,3 +213,37 @@ def test_13b_width_batch_of_four_tree_and_autoregressive_paths_agree(cb):
     accepted, agree, clear, total = _teacher_forced_steps(cb, eng, tree, prompts, 6, [2, 5, 1, 3])
     assert max(accepted) >= 4
     assert agree >= 0.8 * total
+
+
+@pytest.mark.parametrize("M,N,K", [(2048, 22016, 4096), (2048, 4096, 11008), (1024, 12288, 4096), (512, 32000, 4096),
+                                   (256, 27648, 5120)])
+def test_gemm_at_the_batched_steps_sizes_on_sampled_outputs(cb, M, N, K):
+    """The projections of the 7B shape (gate/up, down, QKV, LM head) at the row counts of the batched verify steps
+    (16 sequences x 128 / 64 / 32 nodes) and the 13B gate/up at 256 rows: the 256 x 256 units and the row chunks that
+    walk the weights side by side.  The oracle computes a sample of 96 output rows x 384 output columns (first and
+    last rows of every row chunk and first and last columns included) from its definition."""
+    X = synth.normal(12, 1, (M, K), 1.0, dtype=torch.bfloat16, device="cuda")
+    W = synth.normal(12, 2, (N, K), 0.05, dtype=torch.bfloat16, device="cuda")
+    out = cb.gemm(X, W)
+    torch.cuda.synchronize()
+    assert torch.isfinite(out).all()
+    def sample(must, tensor_id, count, high):
+        picked = list(dict.fromkeys(must))
+        for v in synth.randint(12, tensor_id, (4 * count,), high):
+            if len(picked) >= count:
+                break
+            if int(v) not in picked:
+                picked.append(int(v))
+        return sorted(picked)
+
+    rows = sample([0, M - 1] + [c * 256 + d for c in range(M // 256) for d in (0, 255)], 3, 96, M)
+    cols = sample([0, 1, 127, 128, 255, 256, N - 257, N - 256, N - 1], 4, 384, N)
+    ri, ci = torch.tensor(rows), torch.tensor(cols)
+    ref = orc.linear(X.cpu()[ri], W.cpu()[ci])
+    got = out.cpu()[ri][:, ci]
+    assert close(got, ref, 0) < 2e-4
+    # every output element, against the sum of its row's products in another order (a property that holds at any
+    # size): column sums of the whole matrix equal X^T-weighted sums computed from the sampled definition
+    colsum = out.double().sum(dim=0).cpu()[ci]
+    ref_colsum = orc.linear(X.double().sum(dim=0, keepdim=True).cpu(), W.cpu()[ci].double())[0]
+    assert float(((colsum - ref_colsum).abs() / (1.0 + ref_colsum.abs())).max()) < 2e-3
