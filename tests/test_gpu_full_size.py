@@ -247,3 +247,41 @@ def test_gemm_at_the_batched_steps_sizes_on_sampled_outputs(cb, M, N, K):
     colsum = out.double().sum(dim=0).cpu()[ci]
     ref_colsum = orc.linear(X.double().sum(dim=0, keepdim=True).cpu(), W.cpu()[ci].double())[0]
     assert float(((colsum - ref_colsum).abs() / (1.0 + ref_colsum.abs())).max()) < 2e-3
+
+
+def test_7b_width_batch_of_16_with_128_node_trees_against_oracle(cb):
+    """The largest batched verify step (16 sequences x 128 nodes = 2048 rows) at the 7B width, two layers: GEMMs in
+    row chunks walked side by side, the 128-row tensor-core attention, ragged prompts.  One sequence of the batch is
+    checked against the oracle (prefill state, hidden states and logits of all its 128 nodes, every argmax decision)."""
+    ms = synth.shape_7b(n_layers=2)
+    topk = [10, 10, 10, 10]
+    B, pick = 16, 5
+    model, layout, heads, eng = _engine(cb, ms, 4, topk, 400, max_batch=B)
+    cmodel, sh = cpu(model), oracle_shape(ms)
+    lens = [60 + 17 * b for b in range(B)]
+    prompts = [[int(t) for t in synth.make_prompt(ms.vocab, L, seq=80 + b)] for b, L in enumerate(lens)]
+    tok = torch.zeros(B, max(lens), dtype=torch.int32, device="cuda")
+    for b, p in enumerate(prompts):
+        tok[b, :len(p)] = torch.tensor(p, dtype=torch.int32)
+    eng.prefill(tok, lens)
+    tree = synth.random_parent_tree(128, 6, tree_id=77)
+    th = eng.tree(synth.Tree(tree.parent, np.clip(tree.head, 0, 3), tree.rank))
+    tt = torch.stack([synth.make_prompt(ms.vocab, 128, seq=120 + b).to(torch.int32) for b in range(B)]).cuda().contiguous()
+    node_argmax, logits, hidden = eng.verify(th, tt, want_logits=True, want_hidden=True)
+    torch.cuda.synchronize()
+    assert eng.device_status() == 0
+    assert torch.equal(node_argmax.long().cpu(), torch.argmax(logits, dim=-1).cpu())
+    st = orc.prefill(cmodel, sh, prompts[pick], 600)
+    _, _, h_last = eng.read_state()
+    assert close(h_last[pick], st.h_last) < TOL
+    o_hidden, o_logits = orc.verify_tree(cmodel, sh, st, [int(t) for t in tt[pick]], tree.parent)
+    assert_close_large(hidden[pick], o_hidden, TOL, "hidden")
+    assert_close_large(logits[pick], o_logits, TOL, "logits")
+    o_arg = [int(a) for a in orc.argmax_f32(o_logits)]
+    flips = 0
+    for v in range(tree.n):
+        gv = int(node_argmax[pick, v])
+        if gv != o_arg[v]:
+            flips += 1
+            assert float(o_logits[v].max() - o_logits[v][gv]) < TOL, (v, gv, o_arg[v])
+    assert flips <= 6
