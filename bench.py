@@ -552,7 +552,7 @@ def run_sweep(args):
     points = []
     for B in batches:
         for L in lens:
-            eng = cb.Cerberus(ms, model, None, None, (), max_tokens=L + 16, max_batch=B, max_nodes=128)
+            eng = cb.Cerberus(ms, model, None, None, (), max_tokens=L + 16, max_batch=B, max_nodes=max(128, max(nodes)))
             prompts = torch.stack([synth.make_prompt(ms.vocab, L, seq=b).to(torch.int32) for b in range(B)]).cuda().contiguous()
             eng.prefill(prompts, [L] * B)
             torch.cuda.synchronize()
