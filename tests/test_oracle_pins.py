@@ -335,3 +335,107 @@ def test_threshold_calibration_splits_in_half():
     S = [0.1 * i for i in range(32)]
     T = orc.calibrate_threshold(S)
     assert sum(s > T for s in S) == 16
+
+
+# ------------------------------------------------------------------ decoder-layer wiring against an independent library model
+
+def _hf_llama(ms, model):
+    """The same weights inside the stock `transformers` LLaMA implementation, parameters in float64, eager
+    attention.  That implementation takes its norms, rotation angles and softmax in float32 whatever the
+    parameter type, so agreement is at float32 rounding (~1e-7 per operation), not float64."""
+    tr = pytest.importorskip("transformers")
+    cfg = tr.LlamaConfig(vocab_size=ms.vocab, hidden_size=ms.d_model, intermediate_size=ms.mlp_dim,
+                         num_hidden_layers=ms.n_layers, num_attention_heads=ms.n_heads,
+                         num_key_value_heads=ms.n_heads, head_dim=ms.head_dim, rms_norm_eps=ms.rms_eps,
+                         rope_theta=ms.rope_base, attention_bias=False, mlp_bias=False, tie_word_embeddings=False,
+                         max_position_embeddings=256, hidden_act="silu", attn_implementation="eager")
+    hf = tr.LlamaForCausalLM(cfg).to(torch.float64).eval()
+    hd, F = ms.n_heads * ms.head_dim, ms.mlp_dim
+    sd = {"model.embed_tokens.weight": model["embed"], "model.norm.weight": model["final_norm"],
+          "lm_head.weight": model["lm_head"]}
+    for l in range(ms.n_layers):
+        p = f"model.layers.{l}."
+        wqkv, wgu = model[f"wqkv.{l}"], model[f"wgu.{l}"]
+        sd[p + "self_attn.q_proj.weight"] = wqkv[:hd]
+        sd[p + "self_attn.k_proj.weight"] = wqkv[hd:2 * hd]
+        sd[p + "self_attn.v_proj.weight"] = wqkv[2 * hd:]
+        sd[p + "self_attn.o_proj.weight"] = model[f"wo.{l}"]
+        sd[p + "mlp.gate_proj.weight"] = wgu[:F]
+        sd[p + "mlp.up_proj.weight"] = wgu[F:]
+        sd[p + "mlp.down_proj.weight"] = model[f"wd.{l}"]
+        sd[p + "input_layernorm.weight"] = model[f"attn_norm.{l}"]
+        sd[p + "post_attention_layernorm.weight"] = model[f"mlp_norm.{l}"]
+    missing, unexpected = hf.load_state_dict({k: v.to(torch.float64) for k, v in sd.items()}, strict=False)
+    assert not unexpected and all("rotary" in k or "inv_freq" in k for k in missing), (missing, unexpected)
+    return hf
+
+
+def test_decoder_wiring_matches_transformers_llama():
+    """forward_full (pre-norm, fused QKV split, rotate-half RoPE, causal attention, o-projection + residual,
+    pre-norm SwiGLU with gate rows first, down-projection + residual, final norm, untied LM head) against the
+    LLaMA decoder of the `transformers` package holding the same weights: Section 5.1 names the base model as
+    a LLaMA fine-tune, and that package is an independent statement of the architecture."""
+    ms = synth.ModelShape(3, 64, 4, 16, 176, 96, "fp32")
+    model = synth.make_model(ms, seed=5, std=0.08)
+    sh = orc.Shape(ms.n_layers, ms.d_model, ms.n_heads, ms.head_dim, ms.mlp_dim, ms.vocab, "fp32")
+    tokens = [int(t) for t in synth.make_prompt(ms.vocab, 23, seq=3)]
+    hidden, logits, kv = orc.forward_full(model, sh, tokens)
+    hf = _hf_llama(ms, model)
+    with torch.no_grad():
+        out = hf(torch.tensor([tokens]), use_cache=True, output_hidden_states=True)
+        h_ref = hf.model(torch.tensor([tokens])).last_hidden_state[0]
+    tol = 3e-6          # the library's float32 norms, angles and softmax; a wiring mistake is > 1e-3 (next test)
+    assert float((logits - out.logits[0]).abs().max()) < tol
+    assert float((hidden - h_ref).abs().max()) < tol
+    # the residual stream entering every layer (hidden_states[l], before the final norm) is implied by the above
+    # for the last layer only; K and V of every layer pin the rest: post-rotation keys, unrotated values
+    for l in range(ms.n_layers):
+        layer = out.past_key_values.layers[l]
+        k_ref, v_ref = layer.keys[0].transpose(0, 1), layer.values[0].transpose(0, 1)     # [T][H][Dh]
+        assert float((kv[l][0] - k_ref).abs().max()) < tol
+        assert float((kv[l][1] - v_ref).abs().max()) < tol
+    assert float(logits.abs().max()) > 0.1      # the comparison is not between two near-zero tensors
+
+
+@pytest.mark.parametrize("mistake", ["no_attn_residual", "no_mlp_residual", "swap_gate_up", "post_norm", "no_final_norm"])
+def test_decoder_wiring_pin_catches_planted_mistakes(mistake, monkeypatch):
+    """The library comparison must turn red for each plausible wiring mistake, planted in the oracle."""
+    ms = synth.ModelShape(2, 64, 4, 16, 176, 96, "fp32")
+    model = synth.make_model(ms, seed=5, std=0.08)
+    sh = orc.Shape(ms.n_layers, ms.d_model, ms.n_heads, ms.head_dim, ms.mlp_dim, ms.vocab, "fp32")
+    tokens = [int(t) for t in synth.make_prompt(ms.vocab, 11, seq=4)]
+    hf = _hf_llama(ms, model)
+    with torch.no_grad():
+        ref = hf(torch.tensor([tokens])).logits[0]
+    good = orc.forward_full(model, sh, tokens)[1]
+    assert float((good - ref).abs().max()) < 3e-6
+
+    F = ms.mlp_dim
+    f64 = orc.f64
+
+    def post(x, a, m, l, s):
+        T = x.shape[0]
+        o = a.reshape(T, -1) @ f64(m[f"wo.{l}"]).T
+        x = o if mistake == "no_attn_residual" else x + o
+        if mistake == "post_norm":
+            xn = x
+        else:
+            xn = orc.rmsnorm(x, f64(m[f"mlp_norm.{l}"]), s.rms_eps)
+        gu = xn @ f64(m[f"wgu.{l}"]).T
+        g, u = (gu[:, F:], gu[:, :F]) if mistake == "swap_gate_up" else (gu[:, :F], gu[:, F:])
+        y = (orc.silu(g) * u) @ f64(m[f"wd.{l}"]).T
+        y = y if mistake == "no_mlp_residual" else x + y
+        if mistake == "post_norm":
+            y = orc.rmsnorm(y, f64(m[f"mlp_norm.{l}"]), s.rms_eps)
+        return y
+
+    def final(x, m, s, want_logits=True):
+        h = x if mistake == "no_final_norm" else orc.rmsnorm(x, f64(m["final_norm"]), s.rms_eps)
+        return h, h @ f64(m["lm_head"]).T
+
+    if mistake == "no_final_norm":
+        monkeypatch.setattr(orc, "_final", final)
+    else:
+        monkeypatch.setattr(orc, "_post_attention", post)
+    bad = orc.forward_full(model, sh, tokens)[1]
+    assert float((bad - ref).abs().max()) > 1e-3
