@@ -291,6 +291,14 @@ int cerb_device_status(cerb_ctx* ctx, void* stream);
 int cerb_profile_enable(cerb_ctx* ctx, int32_t on);
 int cerb_profile_read(cerb_ctx* ctx, double* ms_out, int64_t* groups_out, void* stream);
 
+/* Budget of every bounded device-side wait (mbarrier and cluster waits inside the kernels), in SM clock
+ * cycles, for all later launches of this process; the paper has no counterpart.  The default, 4e9 (about two
+ * seconds), is far beyond any legitimate wait.  A wait that runs out makes its CTA raise CERB_E_TIMEOUT in the
+ * status word, leave its loops, wait (bounded) for its own copies in flight, free its tensor memory and
+ * return; the results of that launch are then undefined and cerb_device_status reports the code.  Meant for
+ * testing that exit; CERB_E_ARG below 1000 cycles. */
+int cerb_set_wait_cycles(int64_t cycles);
+
 /* Number of kernel launches issued by this context since load (for accounting). */
 int64_t cerb_launch_count(const cerb_ctx* ctx);
 

@@ -26,7 +26,8 @@ def _stale(target: str, deps) -> bool:
 
 def build(verbose: bool = False, force: bool = False) -> str:
     os.makedirs(OBJ, exist_ok=True)
-    headers = [os.path.join(CSRC, "cerb_internal.cuh"), os.path.join(ROOT, "include", "cerb.h")]
+    headers = [os.path.join(CSRC, f) for f in sorted(os.listdir(CSRC)) if f.endswith(".cuh")]
+    headers.append(os.path.join(ROOT, "include", "cerb.h"))
     jobs = []
     for src in SOURCES:
         s = os.path.join(CSRC, src)

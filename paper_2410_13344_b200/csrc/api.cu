@@ -19,6 +19,10 @@ bool pdl_enabled() {
   }
   return v != 0;
 }
+namespace {
+long long g_wait_cycles = 4000000000ll;       // about 2 s of SM clock: far beyond any legitimate wait
+}
+long long wait_cycles() { return g_wait_cycles; }
 }  // namespace cerb
 
 namespace {
@@ -723,5 +727,11 @@ int cerb_profile_read(cerb_ctx* c, double* ms_out, int64_t* groups_out, void* st
 }
 
 int64_t cerb_launch_count(const cerb_ctx* c) { return c ? c->launches : -1; }
+
+int cerb_set_wait_cycles(int64_t cycles) {
+  if (cycles < 1000) return CERB_E_ARG;
+  cerb::g_wait_cycles = cycles;
+  return CERB_OK;
+}
 
 }  // extern "C"

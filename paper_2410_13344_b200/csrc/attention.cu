@@ -13,7 +13,7 @@
 // fp32 path (CERB_F32 models): plain FMA arithmetic, one CTA per (node, head, sequence).
 #include <stdlib.h>
 
-#include "cerb_internal.cuh"
+#include "tc_common.cuh"
 
 namespace cerb {
 
@@ -24,72 +24,12 @@ constexpr int PAGES_PER_TILE = TILE / CERB_PAGE;
 constexpr int kTargetCtas = 296;          // two CTAs per SM on a 148-SM part
 constexpr int kMaxSplit = 32;
 constexpr int kMaxPagesPerCta = 1024;
-constexpr long long kWaitCycles = 4000000000ll;   // about 2 s of SM clock: far beyond any legitimate wait
 constexpr size_t kCounterBytes = 4096;    // one ticket counter per (sequence, head)
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait: gives up after kWaitCycles SM clock cycles (a couple of seconds).  After the first
-// time-out in a CTA (or when an earlier kernel already reported one) every later wait gives up
-// almost at once, so the CTA still runs to its end in bounded time.  The budget is measured with
-// the SM-local cycle counter, which is cheap to read; the polls in between are back to back.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* aborted, int32_t* status) {
-  for (int i = 0; i < 1024; ++i)
-    if (mbar_try_wait(bar, parity)) return;
-  const long long t0 = clock64();
-  const long long budget = *aborted ? 40000ll : kWaitCycles;
-  for (;;) {
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_wait(bar, parity)) return;
-    if (clock64() - t0 > budget) break;
-  }
-  *aborted = 1;
-  atomicExch(status, CERB_E_TIMEOUT);
-}
-// Same bounded wait for a lane whose warp shares an issue port with busy warps: back off between polls.
-__device__ __forceinline__ void mbar_wait_polite(uint32_t bar, uint32_t parity, volatile int* aborted, int32_t* status) {
-  for (int i = 0; i < 4; ++i)
-    if (mbar_try_wait(bar, parity)) return;
-  const long long t0 = clock64();
-  const long long budget = *aborted ? 40000ll : kWaitCycles;
-  for (;;) {
-    for (int i = 0; i < 64; ++i) {
-      if (mbar_try_wait(bar, parity)) return;
-      __nanosleep(40);
-    }
-    if (clock64() - t0 > budget) break;
-  }
-  *aborted = 1;
-  atomicExch(status, CERB_E_TIMEOUT);
-}
 // K/V tiles are read once per step (the next layer's tiles, and 13 GB of weights, come before they are needed
 // again): they enter L2 with evict-first priority so that they do not push out activations and partial sums.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  uint64_t pol;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
-      ::"r"(dst), "l"((uint64_t)map), "r"(x), "r"(y), "r"(bar), "l"(pol)
-      : "memory");
+  tma_load_2d_hint(dst, map, x, y, bar, l2_policy(true));
 }
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -104,66 +44,6 @@ __device__ __forceinline__ void mma_bf16(float* c, uint32_t a0, uint32_t a1, uin
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
-// Thread-block cluster helpers: barrier over every thread of the cluster, and loads from another CTA's shared memory.
-// Rendezvous of the CTAs of a cluster with bounded waits.  Every CTA owns two mbarriers that expect one
-// arrival per member; to meet, one thread of every CTA arrives on that barrier of every member (remote
-// arrive, release at cluster scope) and whoever goes on to read the others' shared memory first waits on its
-// own copy (acquire at cluster scope) with the same cycle budget as every other wait of these kernels.  The
-// hardware cluster barrier is used once only, split in two: every thread arrives right after the barriers
-// are initialised and waits just before the first remote arrive, so that no arrival can reach a barrier that
-// is not initialised yet; that wait depends on nothing but the members having started.
-__device__ __forceinline__ void cluster_start_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
-__device__ __forceinline__ void cluster_start_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// `idx` numbers the calling threads of the CTA from 0: thread s signals member s (the arrivals leave in parallel).
-__device__ __forceinline__ void cluster_meet(uint64_t* bar, int members, int idx, volatile int* aborted, int32_t* status) {
-  const uint32_t local = (uint32_t)__cvta_generic_to_shared(bar);
-  if (idx < members) {
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"((uint32_t)idx));
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
-  }
-  for (int i = 0; i < 1024; ++i)
-    if (mbar_try_wait_cluster(local, 0)) return;
-  const long long t0 = clock64();
-  const long long budget = *aborted ? 40000ll : kWaitCycles;
-  for (;;) {
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_wait_cluster(local, 0)) return;
-    if (clock64() - t0 > budget) break;
-  }
-  *aborted = 1;
-  atomicExch(status, CERB_E_TIMEOUT);
-}
-__device__ __forceinline__ uint32_t mapa_u32(uint32_t saddr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ float ld_cluster_f32(uint32_t a) {
-  float v;
-  asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
-  return v;
-}
-__device__ __forceinline__ float4 ld_cluster_v4(uint32_t a) {
-  float4 v;
-  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a) : "memory");
-  return v;
 }
 __device__ __forceinline__ void compute_bar(int nthreads) { asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory"); }
 
@@ -200,6 +80,7 @@ struct AttnParams {
                             // (the row stride between sequences); only keys below row0 + rows can be ancestors of these rows.
   int rows_pad;             // rows per split in `partial` (16, 32, 64 or 128)
   uint32_t v_lbo, v_sbo;    // byte offsets of the V operand's descriptor (tensor-core path)
+  long long wait_cycles;    // budget of every bounded wait, SM clock cycles
   int cluster;              // tensor-core path: the splits of a (sequence, head) form one cluster and merge through shared memory
   float scale_log2;
 };
@@ -227,6 +108,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
   __shared__ unsigned int ticket_s;
   __shared__ __align__(8) uint64_t cl_bar[2];
   volatile int* aborted = &aborted_s;
+  const WaitCtx wc{p.wait_cycles, aborted, p.status};
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -278,7 +160,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
         if (i == early) { griddep_wait(); griddep_launch(); }
         int s = i % STAGES;
         uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-        mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, aborted, p.status);
+        mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, wc);
         uint32_t fb = smem_u32(&full_bar[s]);
         mbar_expect_tx(fb, STAGE_BYTES);
         uint32_t kdst = smem_base + (uint32_t)s * STAGE_BYTES, vdst = kdst + KV_BYTES;
@@ -332,7 +214,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
     for (int t = t0, it = 0; t < t_end; ++t, ++it) {
       const int s = it % STAGES;
       const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
-      mbar_wait(smem_u32(&full_bar[s]), ph, aborted, p.status);
+      mbar_wait(smem_u32(&full_bar[s]), ph, wc);
       const uint32_t kbase = smem_base + (uint32_t)s * STAGE_BYTES, vbase = kbase + KV_BYTES;
       const int key_tile0 = t * TILE;
       if (key_tile0 + TILE > kv_total) {
@@ -541,7 +423,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
     // in split order and writes the output.  Nobody leaves before the second meeting.
     cluster_start_wait();
     if (warp < NW) {
-      cluster_meet(&cl_bar[0], p.nsplit, (int)threadIdx.x, aborted, p.status);     // every member's rows are in place
+      cluster_meet(&cl_bar[0], p.nsplit, (int)threadIdx.x, wc);     // every member's rows are in place
       constexpr int C4 = DH / 4;
       const int ct = warp * 32 + lane, rows_per_pass = (NW * 32) / C4;
       const float LN2 = 0.6931471805599453f;
@@ -567,7 +449,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
         if (c4 == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
       }
       compute_bar(NW * 32);                                                          // this CTA has read all it needs
-      if (warp == 0) cluster_meet(&cl_bar[1], p.nsplit, lane, aborted, p.status);
+      if (warp == 0) cluster_meet(&cl_bar[1], p.nsplit, lane, wc);
     }
     __syncthreads();                           // nobody exits before warp 0 has seen every member done
   }
@@ -611,49 +493,9 @@ constexpr int TC_DH = 128, TC_ROWF = TC_DH + 4;
 constexpr int TC_THREADS = 352;                       // producer, QK^T issuer, two softmax groups of four warps, PV issuer
 constexpr float TC_RESCALE = 8.0f;                    // log2 of the growth of a row maximum that forces a rescale
 
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ uint64_t desc_k_sw128(uint32_t saddr) {      // K-major rows of 128 bytes, 128-byte swizzle
-  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024u >> 4) << 32) | ((uint64_t)1 << 46) |
-         ((uint64_t)2 << 61);
-}
-__device__ __forceinline__ uint64_t desc_mn_sw128(uint32_t saddr, uint32_t lbo, uint32_t sbo) {   // MN-major (V: [key][dh])
-  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | ((uint64_t)1 << 46) |
-         ((uint64_t)2 << 61);
-}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) { tmem_ld16_nowait(taddr, r); }
 __device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
+  umma_bf16(tmem_d, adesc, bdesc, idesc, acc);
 }
 
 template <int SK, int SV, int QROWS, bool UNI>
@@ -670,6 +512,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
   __shared__ unsigned int ticket_s;
   __shared__ __align__(8) uint64_t cl_bar[2];
   volatile int* aborted = &aborted_s;
+  const WaitCtx wc{p.wait_cycles, aborted, p.status};
 
   // Everything up to the first use of Q or of this step's tree keys runs before griddep_wait(): lengths,
   // live node counts and the page table were written at least two kernels ago, and so were the prefix
@@ -754,9 +597,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
         const int sk = i % SK, sv = i % SV;
         const uint32_t fk = smem_u32(&full_k[sk]), fv = smem_u32(&full_v[sv]);
         if (lane == 0) {
-          mbar_wait_polite(smem_u32(&empty_k[sk]), ((uint32_t)(i / SK) & 1u) ^ 1u, aborted, p.status);
+          mbar_wait_polite(smem_u32(&empty_k[sk]), ((uint32_t)(i / SK) & 1u) ^ 1u, wc);
           mbar_expect_tx(fk, TC_KV_BYTES);
-          mbar_wait_polite(smem_u32(&empty_v[sv]), ((uint32_t)(i / SV) & 1u) ^ 1u, aborted, p.status);
+          mbar_wait_polite(smem_u32(&empty_v[sv]), ((uint32_t)(i / SV) & 1u) ^ 1u, wc);
           mbar_expect_tx(fv, TC_KV_BYTES);
         }
         __syncwarp();
@@ -772,7 +615,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       for (int i = 0; i < T; ++i) {
         if (i == early) { griddep_wait(); griddep_launch(); }
         const int sv = i % SV;
-        mbar_wait_polite(smem_u32(&empty_v[sv]), ((uint32_t)(i / SV) & 1u) ^ 1u, aborted, p.status);
+        mbar_wait_polite(smem_u32(&empty_v[sv]), ((uint32_t)(i / SV) & 1u) ^ 1u, wc);
         const uint32_t fv = smem_u32(&full_v[sv]);
         mbar_expect_tx(fv, 2 * TC_KV_BYTES);
         const uint32_t kdst = k_ring + (uint32_t)sv * TC_KV_BYTES, vdst = v_ring + (uint32_t)sv * TC_KV_BYTES;
@@ -803,12 +646,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     if (lane == 0 && T > 0) {
       const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
       const uint64_t q_desc0 = desc_k_sw128(q_base), q_desc1 = desc_k_sw128(q_base + QHALF);
-      mbar_wait(smem_u32(&q_ready), 0, aborted, p.status);
+      mbar_wait(smem_u32(&q_ready), 0, wc);
       for (int i = 0; i < T; ++i) {
         const int g = i & 1, k = i >> 1;
-        if (!UNI) mbar_wait(smem_u32(&full_k[i % SK]), (uint32_t)(i / SK) & 1u, aborted, p.status);
-        else mbar_wait(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, aborted, p.status);
-        mbar_wait(smem_u32(&s_free[g]), ((uint32_t)k & 1u) ^ 1u, aborted, p.status);
+        if (!UNI) mbar_wait(smem_u32(&full_k[i % SK]), (uint32_t)(i / SK) & 1u, wc);
+        else mbar_wait(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, wc);
+        mbar_wait(smem_u32(&s_free[g]), ((uint32_t)k & 1u) ^ 1u, wc);
         tc_fence_after();
         const uint32_t kb = k_ring + (uint32_t)(i % SK) * TC_KV_BYTES;
         const uint64_t k_desc0 = desc_k_sw128(kb), k_desc1 = desc_k_sw128(kb + 8192u);
@@ -830,8 +673,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
       for (int j = 0; j < T; ++j) {
         const int g = j & 1, k = j >> 1;
-        mbar_wait(smem_u32(&p_ready[g]), (uint32_t)k & 1u, aborted, p.status);
-        mbar_wait(smem_u32(&full_v[j % SV]), (uint32_t)(j / SV) & 1u, aborted, p.status);
+        mbar_wait(smem_u32(&p_ready[g]), (uint32_t)k & 1u, wc);
+        mbar_wait(smem_u32(&full_v[j % SV]), (uint32_t)(j / SV) & 1u, wc);
         tc_fence_after();
         const uint32_t vb = v_ring + (uint32_t)(j % SV) * TC_KV_BYTES;
         const uint32_t d = tmem + 128u + (uint32_t)g * 128u;
@@ -878,7 +721,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     float m_used = -INFINITY, l = 0.f;
     int k = 0;
     for (int i = g; i < T; i += 2, ++k) {
-      mbar_wait(smem_u32(&s_full[g]), (uint32_t)k & 1u, aborted, p.status);
+      mbar_wait(smem_u32(&s_full[g]), (uint32_t)k & 1u, wc);
       tc_fence_after();
       float sc[64];
 #pragma unroll
@@ -916,7 +759,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       for (int j = 0; j < 64; ++j) { sc[j] = ex2(sc[j] - mu); rs4[j & 3] += sc[j]; }
       l = l * alpha + ((rs4[0] + rs4[1]) + (rs4[2] + rs4[3]));
       if (k > 0) {
-        mbar_wait(smem_u32(&pv_done[g]), (uint32_t)(k - 1) & 1u, aborted, p.status);   // P buffers free, O at rest
+        mbar_wait(smem_u32(&pv_done[g]), (uint32_t)(k - 1) & 1u, wc);   // P buffers free, O at rest
         tc_fence_after();
         if (__any_sync(0xffffffffu, rescale)) {
 #pragma unroll 1
@@ -937,7 +780,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
         // last, partial tile: rows past the end may hold anything (stale pool memory); zero V there so
         // that a zero probability times a non-finite value cannot poison the sum.  V travels apart
         // from K, so wait until it has landed.
-        mbar_wait(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, aborted, p.status);
+        mbar_wait(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, wc);
         const int first_bad = kv_total - key0;
         uint8_t* vgen = smem_gen + (v_ring - smem_base) + (size_t)(i % SV) * TC_KV_BYTES;
         for (int idx = gt; idx < (TILE - first_bad) * 16; idx += 128) {
@@ -970,7 +813,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     }
     // ---- this group's (m, l, O) rows into shared memory ----
     if (k > 0) {
-      mbar_wait(smem_u32(&pv_done[g]), (uint32_t)(k - 1) & 1u, aborted, p.status);
+      mbar_wait(smem_u32(&pv_done[g]), (uint32_t)(k - 1) & 1u, wc);
       tc_fence_after();
     }
     compute_bar(256);                               // every MMA has retired: all of shared memory can be reused
@@ -1082,7 +925,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     // before the second meeting, so no shared memory is read after its CTA has gone.
     cluster_start_wait();
     if (warp >= 2 && warp < 10) {
-      cluster_meet(&cl_bar[0], p.nsplit, (int)threadIdx.x - 64, aborted, p.status);  // every member's rows are in place
+      cluster_meet(&cl_bar[0], p.nsplit, (int)threadIdx.x - 64, wc);  // every member's rows are in place
       const int ct = threadIdx.x - 64;
       const float LN2 = 0.6931471805599453f;
       const uint32_t mine = smem_u32(smem_gen);
@@ -1115,7 +958,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
         if (c4 == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
       }
       compute_bar(256);                                                              // this CTA has read all it needs
-      if (warp == 2) cluster_meet(&cl_bar[1], p.nsplit, lane, aborted, p.status);
+      if (warp == 2) cluster_meet(&cl_bar[1], p.nsplit, lane, wc);
     }
   }
   tc_fence_before();
@@ -1124,6 +967,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
 }
 
 }  // namespace
+
+#include "attention_kt.cuh"
 
 // ---------------------------------------------------------------------------------------------
 // fp32 path
@@ -1244,6 +1089,7 @@ static int launch_attn_window(const cerb_attn_args* a, int row0, int rows, const
   p.counters = (unsigned int*)a->scratch;
   p.partial = (float*)((char*)a->scratch + kCounterBytes);
   p.status = status;
+  p.wait_cycles = wait_cycles();
   p.n = a->n;
   p.H = a->n_heads;
   p.max_pages = a->max_pages;
@@ -1274,7 +1120,37 @@ static int launch_attn_window(const cerb_attn_args* a, int row0, int rows, const
   p.v_lbo = 8192u;
   p.v_sbo = 1024u;
   int np = nq_pad(rows), rc = CERB_E_SHAPE;
-  if (tensor_path) {
+  // The keys-on-M tensor-core kernel (attention_kt.cuh): 128-key tiles, every MMA row in use whatever the tree's
+  // width.  CERB_ATTN_KT=0 / 1 switches it off / forces it for every head_dim-128 launch.
+  static const int force_kt = getenv("CERB_ATTN_KT") ? atoi(getenv("CERB_ATTN_KT")) : -1;
+  const bool kt_path = a->head_dim == 128 && force_tc < 0 && (force_kt < 0 ? true : force_kt != 0);
+  if (kt_path) {
+    const int tiles = (a->max_len + KT_TILE - 1) / KT_TILE;
+    int want = 148 / (a->B * a->n_heads);
+    const int max_split = use_cluster ? 8 : kMaxSplit;
+    if (want > max_split) want = max_split;
+    if (want > tiles) want = tiles;
+    if (want < 1) want = 1;
+    const int per = (tiles + want - 1) / want;
+    if (per * KT_PAGES > kMaxPagesPerCta) return CERB_E_SHAPE;
+    p.nsplit = (tiles + per - 1) / per;
+    p.cluster = (use_cluster && p.nsplit >= 2 && p.nsplit <= 8) ? 1 : 0;
+    // query blocks of 32: trees of up to 64 nodes take the two-block kernel (its MMAs are 64 queries wide anyway)
+    const int ncb = rows <= 64 ? 2 : (rows + 31) / 32;
+    static bool kt_configured = false;
+    if (!kt_configured) {
+      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_kt_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kt_smem(2)));
+      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_kt_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kt_smem(3)));
+      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_kt_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kt_smem(4)));
+      kt_configured = true;
+    }
+    auto kern = ncb == 2 ? tree_attn_kt_kernel<2> : ncb == 3 ? tree_attn_kt_kernel<3> : tree_attn_kt_kernel<4>;
+    const dim3 grid(p.nsplit, p.H, a->B), block(kt_threads(ncb));
+    if (p.cluster)
+      rc = launch_pdl_cluster(kern, grid, block, kt_smem(ncb), st, (unsigned)p.nsplit, *tmK, *tmV, p) == cudaSuccess ? CERB_OK : CERB_E_CUDA;
+    else
+      rc = launch_pdl(kern, grid, block, kt_smem(ncb), st, *tmK, *tmV, p) == cudaSuccess ? CERB_OK : CERB_E_CUDA;
+  } else if (tensor_path) {
     static bool configured = false;
     if (!configured) {
       CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_tc_kernel<2, 5, 128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tc_smem(2, 5, 128)));

@@ -29,13 +29,13 @@
 // owns a tile's last segment zero-fills the slots that tile does not use.
 //
 // Roles inside a CTA (224 threads): warp 0 = TMA producer (one lane) running ahead through the
-// whole share, warp 1 = TMEM allocator and MMA issuer (one lane), warp 6 = second MMA issuer in wide
-// mode, warps 2-5 = epilogue (each owns the 32 TMEM lanes of its warp quarter).  The accumulator is double-buffered in TMEM so a segment's
+// whole share, warp 1 = TMEM allocator and MMA issuer (one lane), warp 6 = second MMA issuer,
+// warps 2-5 = epilogue (each owns the 32 TMEM lanes of its warp quarter).  The accumulator is double-buffered in TMEM so a segment's
 // epilogue overlaps the next segment's MMAs.  Stages and accumulators are handed over with
 // mbarriers; every wait is bounded and reports CERB_E_TIMEOUT through a status word.
 #include <stdlib.h>
 
-#include "cerb_internal.cuh"
+#include "tc_common.cuh"
 
 namespace cerb {
 
@@ -45,106 +45,11 @@ constexpr int BM = 128;          // weight rows per CTA (MMA M)
 constexpr int BK = 64;           // k elements per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int MAX_STAGES = 8;
 constexpr uint32_t A_STAGE_BYTES = BM * BK * 2;
-constexpr long long kWaitCycles = 4000000000ll;   // about 2 s of SM clock: far beyond any legitimate wait
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait: gives up after kWaitCycles SM clock cycles (a couple of seconds).  After the first
-// time-out in a CTA (or when an earlier kernel already reported one) every later wait gives up
-// almost at once, so the CTA still runs to its end in bounded time.  The budget is measured with
-// the SM-local cycle counter, which is cheap to read; the polls in between are back to back.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* aborted, int32_t* status) {
-  for (int i = 0; i < 1024; ++i)
-    if (mbar_try_wait(bar, parity)) return;
-  const long long t0 = clock64();
-  const long long budget = *aborted ? 40000ll : kWaitCycles;
-  for (;;) {
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_wait(bar, parity)) return;
-    if (clock64() - t0 > budget) break;
-  }
-  *aborted = 1;
-  atomicExch(status, CERB_E_TIMEOUT);
-}
-
-__device__ __forceinline__ uint64_t l2_policy(bool evict_first) {
-  uint64_t pol;
-  if (evict_first) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-  else asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-  return pol;
-}
-__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar, uint64_t pol) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
-      ::"r"(dst), "l"((uint64_t)map), "r"(x), "r"(y), "r"(bar), "l"(pol)
-      : "memory");
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"((uint64_t)map), "r"(x), "r"(y), "r"(bar)
-      : "memory");
-}
-
-// Shared-memory matrix descriptor for a K-major operand tile stored as rows of 128 bytes with the
-// 128-byte swizzle (what TMA writes): 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);        // start address, 16-byte units
-  d |= (uint64_t)1 << 16;                           // leading byte offset (unused for swizzled K-major)
-  d |= (uint64_t)(1024u >> 4) << 32;                // stride byte offset between 8-row groups
-  d |= (uint64_t)1 << 46;                           // descriptor version for this architecture
-  d |= (uint64_t)2 << 61;                           // layout: 128-byte swizzle
-  return d;
-}
-
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
-      : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
+// Loads 16 accumulator columns of this warp's 32 lanes and waits for them.
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+  tmem_ld16_nowait(taddr, r);
+  tmem_ld_wait();
 }
 
 struct GemmParams {
@@ -161,10 +66,7 @@ struct GemmParams {
                       // part of the list
   int nslots;         // partial slots per output element
   int stages;
-  int wide;           // 1: a CTA works on 256 weight rows at a time (two MMA tiles sharing one activation stage)
-  int group;          // stages are released to the producer in groups of this many (1 or 2)
-  int hint;           // 1: weights evict-first, activations evict-last in L2
-  int issuers;        // MMA-issuing threads: 2 in wide mode (one per weight tile of a unit), else 1
+  long long wait_cycles;   // budget of every bounded wait, SM clock cycles
   uint32_t idesc;
   uint32_t acc_cols;  // TMEM columns of one accumulator buffer
   int acc_bufs;       // accumulator buffers in TMEM: 2 (a segment's epilogue overlaps the next segment's MMAs), or 1 when
@@ -205,12 +107,12 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
   __shared__ int aborted_s;
   __shared__ unsigned int ticket_s;
   volatile int* aborted = &aborted_s;
+  const WaitCtx wc{p.wait_cycles, aborted, p.status};
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t b_bytes = (uint32_t)p.n_mma * BK * 2;
-  const uint32_t a_bytes = A_STAGE_BYTES * (uint32_t)(1 + p.wide);
+  const uint32_t a_bytes = 2 * A_STAGE_BYTES;        // two weight tiles of 128 rows per unit
   const uint32_t stage_bytes = a_bytes + b_bytes;
-  const int rows_per_tile = BM * (1 + p.wide);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int share = (int)blockIdx.x / p.lock;          // which contiguous share of the unit list
   const int my_chunk = (int)blockIdx.x % p.lock;       // with lock > 1: the row chunk this CTA computes
@@ -221,10 +123,10 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
     aborted_s = 0;
     for (int s = 0; s < p.stages; ++s) {
       mbar_init(smem_u32(&full_bar[s]), 1);
-      mbar_init(smem_u32(&empty_bar[s]), (uint32_t)p.issuers);
+      mbar_init(smem_u32(&empty_bar[s]), 2);
     }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(smem_u32(&acc_full[i]), (uint32_t)p.issuers);
+      mbar_init(smem_u32(&acc_full[i]), 2);
       mbar_init(smem_u32(&acc_empty[i]), 4);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -240,7 +142,6 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
 
-  griddep_launch();
   if (warp == 0) {
     if (lane == 0) {
       const int n_units = u1 - u0;
@@ -254,13 +155,8 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
         const uint32_t fb = smem_u32(&full_bar[s]);
         const uint32_t a_dst = smem_base + (uint32_t)s * stage_bytes;
         mbar_expect_tx(fb, stage_bytes);
-        if (p.hint) {
-          tma_load_2d_hint(a_dst, &tmW, w_kb * BK, tile * p.tile_rows, fb, pol_w);
-          if (p.wide) tma_load_2d_hint(a_dst + A_STAGE_BYTES, &tmW, w_kb * BK, tile * p.tile_rows + p.half_off, fb, pol_w);
-        } else {
-          tma_load_2d(a_dst, &tmW, w_kb * BK, tile * p.tile_rows, fb);
-          if (p.wide) tma_load_2d(a_dst + A_STAGE_BYTES, &tmW, w_kb * BK, tile * p.tile_rows + p.half_off, fb);
-        }
+        tma_load_2d_hint(a_dst, &tmW, w_kb * BK, tile * p.tile_rows, fb, pol_w);
+        tma_load_2d_hint(a_dst + A_STAGE_BYTES, &tmW, w_kb * BK, tile * p.tile_rows + p.half_off, fb, pol_w);
         if (++w_kb == p.num_kb) { w_kb = 0; ++w_job; }
       };
       auto load_x = [&](int i) {
@@ -268,8 +164,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
         const int s = i % p.stages;
         const uint32_t fb = smem_u32(&full_bar[s]);
         const uint32_t x_dst = smem_base + (uint32_t)s * stage_bytes + a_bytes;
-        if (p.hint) tma_load_2d_hint(x_dst, &tmX, x_kb * BK, mchunk * kGemmRowsPerPass, fb, pol_x);
-        else tma_load_2d(x_dst, &tmX, x_kb * BK, mchunk * kGemmRowsPerPass, fb);
+        tma_load_2d_hint(x_dst, &tmX, x_kb * BK, mchunk * kGemmRowsPerPass, fb, pol_x);
         if (++x_kb == p.num_kb) { x_kb = 0; ++x_job; }
       };
       // Weights do not depend on the kernel before this one: fill the whole ring with weight tiles
@@ -279,57 +174,49 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
       // the activation map's descriptor is fetched now, not by the first load after the wait
       asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tmX) : "memory");
       griddep_wait();
+      // Dependents are released only now, after this CTA's own wait: when the kernel after this one starts,
+      // the kernel before this one is complete, which is what lets kernels read, ahead of their own wait,
+      // anything written at least two launches earlier.
+      griddep_launch();
       if (p.clk) atomicMin(p.clk, globaltimer_ns());
       for (int i = 0; i < pre; ++i) load_x(i);
       for (int i = pre; i < n_units; ++i) {
         const int s = i % p.stages;
         const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
-        mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, aborted, p.status);
+        mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, wc);
         load_w(i);
         load_x(i);
       }
     }
   } else if (warp == 1 || warp == 6) {
     // MMA issuers.  Issuing one tcgen05.mma occupies its thread for ~100 cycles whatever the MMA's size, and
-    // a 64-row step needs eight of them per 32 KB of weights, so in wide mode each of the two weight
-    // tiles of a unit has its own issuing thread (warp 1: first tile, warp 6: second tile).  A stage is
-    // free, and an accumulator complete, once both have committed.
-    const int mine = warp == 6 ? 1 : 0;
-    if (lane == 0 && mine < p.issuers) {
-      const int hf0 = mine, hf1 = (p.issuers == 2) ? mine : p.wide;     // weight tiles of a unit this thread issues
+    // a 64-row step needs eight of them per 32 KB of weights, so each of the two weight tiles of a unit has
+    // its own issuing thread (warp 1: first tile, warp 6: second tile).  A stage is free, and an accumulator
+    // complete, once both have committed.
+    const int hf = warp == 6 ? 1 : 0;
+    if (lane == 0) {
       int u = u0;
       Segment sg;
       int i = 0, g = 0;
       while (next_segment(u, u1, p.num_kb, sg)) {
         const int buf = p.acc_bufs == 2 ? (g & 1) : 0;
         const uint32_t use = (uint32_t)(p.acc_bufs == 2 ? g >> 1 : g);      // how often this buffer was used before
-        mbar_wait(smem_u32(&acc_empty[buf]), (use & 1u) ^ 1u, aborted, p.status);
+        mbar_wait(smem_u32(&acc_empty[buf]), (use & 1u) ^ 1u, wc);
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)buf * p.acc_cols;
-        int held = -1;                                // stage whose release is deferred to pair it with the next
         for (int k = 0; k < sg.nkb; ++k, ++i) {
           int s = i % p.stages;
           uint32_t ph = (uint32_t)(i / p.stages) & 1u;
-          mbar_wait(smem_u32(&full_bar[s]), ph, aborted, p.status);
+          mbar_wait(smem_u32(&full_bar[s]), ph, wc);
           tc_fence_after();
           uint32_t a_src = smem_base + (uint32_t)s * stage_bytes;
-          uint64_t bdesc = umma_desc_sw128(a_src + a_bytes);
-          for (int hf = hf0; hf <= hf1; ++hf) {
-            const uint64_t adesc = umma_desc_sw128(a_src + (uint32_t)hf * A_STAGE_BYTES);
-            const uint32_t d = tmem_d + (uint32_t)(hf * p.n_mma);
+          uint64_t bdesc = desc_k_sw128(a_src + a_bytes);
+          const uint64_t adesc = desc_k_sw128(a_src + (uint32_t)hf * A_STAGE_BYTES);
+          const uint32_t d = tmem_d + (uint32_t)(hf * p.n_mma);
 #pragma unroll
-            for (int kk = 0; kk < BK / 16; ++kk)    // advance 16 k elements = 32 bytes inside the swizzled row: +2 in 16-byte units
-              umma_bf16(d, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), p.idesc, (k > 0 || kk > 0) ? 1u : 0u);
-          }
-          // Release stages once the MMAs have read them.  Releasing two neighbouring k blocks together
-          // makes the producer request 256 contiguous bytes of every weight row at once.
-          if (p.group == 2 && held < 0 && k + 1 < sg.nkb) {
-            held = s;
-          } else {
-            if (held >= 0) umma_commit(smem_u32(&empty_bar[held]));
-            umma_commit(smem_u32(&empty_bar[s]));
-            held = -1;
-          }
+          for (int kk = 0; kk < BK / 16; ++kk)    // advance 16 k elements = 32 bytes inside the swizzled row: +2 in 16-byte units
+            umma_bf16(d, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), p.idesc, (k > 0 || kk > 0) ? 1u : 0u);
+          umma_commit(smem_u32(&empty_bar[s]));     // the stage is free once the MMAs have read it
         }
         umma_commit(smem_u32(&acc_full[buf]));       // this thread's part of the segment's accumulator is complete
         ++g;
@@ -344,7 +231,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
     while (next_segment(u, u1, p.num_kb, sg)) {
       const int buf = p.acc_bufs == 2 ? (g & 1) : 0;
       const int tile = sg.job % p.tiles, mchunk = p.lock > 1 ? my_chunk : sg.job / p.tiles;
-      mbar_wait(smem_u32(&acc_full[buf]), (uint32_t)(p.acc_bufs == 2 ? g >> 1 : g) & 1u, aborted, p.status);
+      mbar_wait(smem_u32(&acc_full[buf]), (uint32_t)(p.acc_bufs == 2 ? g >> 1 : g) & 1u, wc);
       tc_fence_after();
       // slot = how many CTAs before this one also work on this job
       const int job_u0 = sg.job * p.num_kb;
@@ -377,7 +264,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
         ++g;
         continue;
       }
-      for (int hf = 0; hf <= p.wide; ++hf) {
+      for (int hf = 0; hf < 2; ++hf) {
         const int n_out = tile * p.tile_rows + hf * p.half_off + quarter * 32 + lane;
         const bool n_ok = n_out < p.N;
         // consecutive lanes hold consecutive output columns: every store instruction writes 128 contiguous bytes
@@ -402,7 +289,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
       if (p.epi == 0 && share == last_cta) {
-        for (int hf = 0; hf <= p.wide; ++hf) {
+        for (int hf = 0; hf < 2; ++hf) {
           const int n_out = tile * p.tile_rows + hf * p.half_off + quarter * 32 + lane;
           if (n_out >= p.N) continue;
           for (int z = last_cta - first_cta + 1; z < p.nslots; ++z) {
@@ -451,21 +338,9 @@ struct GemmPlan {
   long long total;   // checked to fit 31 bits before launch
 };
 
-// Tuning switches (environment, read once): CERB_GEMM_WIDE, CERB_GEMM_LOCK, CERB_GEMM_GROUP, CERB_GEMM_HINT.
-int tune(const char* name, int dflt) {
-  const char* v = getenv(name);
-  return v ? atoi(v) : dflt;
-}
-// 0: never; 1: only for passes of at most 128 activation rows; 2: for 256-row passes as well (the accumulator is then
-// single-buffered: two weight tiles x 256 rows fill tensor memory)
-bool use_wide(int M) {
-  static int w = tune("CERB_GEMM_WIDE", 2);
-  return w && (w >= 2 || bucket_rows(row_bucket(M < kGemmRowsPerPass ? M : kGemmRowsPerPass)) <= 128);
-}
-
 GemmPlan make_plan(int sm_count, int M, int N, int K) {
   GemmPlan g;
-  const int rows_per_tile = BM * (use_wide(M) ? 2 : 1);
+  const int rows_per_tile = 2 * BM;            // a unit is two weight tiles of 128 rows
   g.tiles = (N + rows_per_tile - 1) / rows_per_tile;
   g.mchunks = (M + kGemmRowsPerPass - 1) / kGemmRowsPerPass;
   g.num_kb = (K + BK - 1) / BK;
@@ -473,8 +348,7 @@ GemmPlan make_plan(int sm_count, int M, int N, int K) {
   // share is walked by mchunks CTAs side by side, one per row chunk.  They ask for the same weight tiles at the
   // same time, so HBM delivers every weight byte once instead of once per row chunk (measured at 2048 rows x
   // 22016 x 4096 before this: 1.58 GB of DRAM reads for 180 MB of weights, the kernel at 70 % of DRAM throughput).
-  static int lockstep = tune("CERB_GEMM_LOCK", 1);
-  g.lock = (lockstep && g.mchunks > 1 && g.mchunks * 2 <= sm_count) ? g.mchunks : 1;
+  g.lock = (g.mchunks > 1 && g.mchunks * 2 <= sm_count) ? g.mchunks : 1;
   const int jobs = g.lock > 1 ? g.tiles : g.tiles * g.mchunks;
   const int shares = sm_count / g.lock;
   g.total = (long long)jobs * g.num_kb;
@@ -500,11 +374,6 @@ EncodeTiledFn g_encode = nullptr;
 // bytes of every row as well, i.e. the next (or previous) k block of the same rows, which the same CTA asks
 // for right afterwards: DRAM bursts twice as long.  Measured on the 7B decoding step: 4.23 -> 4.02 ms per
 // 64-node forward, 3.49 -> 3.31 ms per one-node forward (128-byte promotion and none are equal).
-CUtensorMapL2promotion l2_promotion() {
-  static int v = getenv("CERB_TMA_PROMO") ? atoi(getenv("CERB_TMA_PROMO")) : 256;
-  return v == 256 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : v == 64 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B
-         : v == 0 ? CU_TENSOR_MAP_L2_PROMOTION_NONE : CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
-}
 
 int encode_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer, uint64_t row_bytes, uint32_t box_inner,
               uint32_t box_outer) {
@@ -515,7 +384,7 @@ int encode_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer
   cuuint32_t box[2] = {box_inner, box_outer};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = g_encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, l2_promotion(),
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? CERB_OK : CERB_E_CUDA;
 }
@@ -555,8 +424,7 @@ int make_pool_map(CUtensorMap* out, const void* pool, int n_pool_pages, int H, i
 // tile's slots with its 128 epilogue threads, which at 64 rows took 55 us per layer against the
 // 6.6 us of the separate kernel that spreads the same bytes over every SM (measured).
 bool gemm_swiglu_fusable(int M, int F) {
-  static int on = tune("CERB_GEMM_SWIGLU", 1);
-  return on && M >= 1 && M <= 16 && use_wide(M) && F % BM == 0;
+  return M >= 1 && M <= 16 && F % BM == 0;
 }
 int gemm_plan_split(int sm_count, int M, int N, int K) { return make_plan(sm_count, M, N, K).nslots; }
 
@@ -587,9 +455,8 @@ int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, fl
   p.total = (int)g.total;
   p.lock = g.lock;
   p.nslots = g.nslots;
-  static int group = tune("CERB_GEMM_GROUP", 1), hint = tune("CERB_GEMM_HINT", 1);
-  p.wide = use_wide(M) ? 1 : 0;
-  p.tile_rows = BM * (1 + p.wide);
+  p.tile_rows = 2 * BM;
+  p.wait_cycles = wait_cycles();
   p.half_off = BM;
   p.epi = 0; p.F = 0; p.act = nullptr; p.tickets = nullptr;
   p.clk = clock_slot;
@@ -599,18 +466,14 @@ int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, fl
     p.tile_rows = BM;            // a unit = gate tile t (rows t*128..) and up tile t (rows F + t*128..)
     p.half_off = p.F;
   }
-  p.group = group == 2 ? 2 : 1;
-  p.hint = hint ? 1 : 0;
-  static int issuers = tune("CERB_GEMM_ISSUERS", 2);
-  p.issuers = (p.wide && issuers == 2) ? 2 : 1;
-  uint32_t stage_bytes = A_STAGE_BYTES * (1 + p.wide) + (uint32_t)p.n_mma * BK * 2;
+  uint32_t stage_bytes = 2 * A_STAGE_BYTES + (uint32_t)p.n_mma * BK * 2;
   p.stages = (int)((216u * 1024u) / stage_bytes);
   if (p.stages > MAX_STAGES) p.stages = MAX_STAGES;
   if (p.stages < 2) return CERB_E_SHAPE;
-  p.acc_cols = (uint32_t)p.n_mma * (1 + p.wide) < 32 ? 32u : (uint32_t)p.n_mma * (1 + p.wide);
+  p.acc_cols = 2u * (uint32_t)p.n_mma;            // two weight tiles side by side (at least 32 columns)
   p.acc_bufs = 2u * p.acc_cols <= 512u ? 2 : 1;
   // instruction descriptor: D fp32, A and B bf16, both K-major, N = n_mma, M = 128
-  p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n_mma >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+  p.idesc = idesc_bf16(BM, (uint32_t)p.n_mma, false, false);
   size_t smem = (size_t)p.stages * stage_bytes + 1024;
   if (smem < 120 * 1024) smem = 120 * 1024;    // one CTA per SM: a CTA may then own all of tensor memory
   static bool configured = false;

@@ -10,6 +10,7 @@ if ROOT not in sys.path:
 
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200); deselected on CPU-only boxes")
+    config.addinivalue_line("markers", "slow: minutes of host time for the oracle; deselect with -m 'gpu and not slow'")
 
 
 def pytest_collection_modifyitems(config, items):

@@ -11,11 +11,26 @@ import torch
 
 from oracle import cerberus_oracle as orc
 from paper_2410_13344_b200 import synth
-from tests.helpers import assert_close_large, close, concat_src, cpu, deepest_path, oracle_shape, top2_margin
+from tests.helpers import (assert_close_large, check_argmax_flips, close, concat_src, cpu, deepest_path, oracle_shape,
+                           parity_stats, record, top2_margin)
 
 pytestmark = pytest.mark.gpu
 TOL = 2e-2
 TIE = 1e-3
+# Allowances of the large-tensor criterion, set to about twice what was measured (the raw figures are recorded by
+# every run, see tests/helpers.py: record): fraction of elements outside |a-b| <= TOL * (1 + |b|), largest oracle
+# margin of a node whose argmax differs, and how many of 64 nodes may differ.
+# Measured (two-layer models at the 7B / 13B widths): K/V 9e-6, hidden states 1.5e-5 (3.8e-5 over 128 nodes), logits
+# 4.2e-4 / 1.2e-3; one node of 64 differing with an oracle margin of 5e-3 (one of 128 with 1.5e-2).  At all 32 layers,
+# against the depth-scaled bound: K/V 6.8e-4, hidden states 1.5e-4, logits 1.0e-3.
+OUTLIERS_KV = 2e-5
+OUTLIERS_HIDDEN = 8e-5
+OUTLIERS_LOGITS = 2.5e-3
+OUTLIERS_KV_DEEP = 1.4e-3
+OUTLIERS_HIDDEN_DEEP = 3e-4
+OUTLIERS_LOGITS_DEEP = 2e-3
+FLIP_MARGIN = 2e-2
+MAX_FLIPS_64 = 2
 
 
 @pytest.fixture(scope="module")
@@ -32,58 +47,98 @@ def _engine(cb, ms, n_cheads, topk, max_tokens, max_batch=1):
     return model, layout, heads, eng
 
 
-def test_7b_width_two_layers_against_oracle(cb):
-    ms = synth.shape_7b(n_layers=2)
-    topk = [10, 10, 10, 10]
-    model, layout, heads, eng = _engine(cb, ms, 4, topk, 512)
+def _two_layer_width_against_oracle(cb, ms, n_cheads, prompt_len, seq, what):
+    """Prefill, gate, draft, one 64-node verification forward, acceptance: values and decisions against the oracle."""
+    topk = [10] * n_cheads
+    model, layout, heads, eng = _engine(cb, ms, n_cheads, topk, 512)
     cmodel, cheads, sh, csrc = cpu(model), cpu(heads), oracle_shape(ms), concat_src(layout)
-    prompt = [int(t) for t in synth.make_prompt(ms.vocab, 200, seq=7)]
+    prompt = [int(t) for t in synth.make_prompt(ms.vocab, prompt_len, seq=seq)]
     tree = synth.best_first_tree(64, topk)
     th = eng.tree(tree)
     eng.prefill(torch.tensor([prompt], dtype=torch.int32, device="cuda"), [len(prompt)])
     st = orc.prefill(cmodel, sh, prompt, 512)
     lens, roots, h_last = eng.read_state()
     assert lens[0] == len(prompt)
+    record(what + " h_last", tol=TOL, **parity_stats(h_last[0], st.h_last, TOL))
     assert close(h_last[0], st.h_last) < TOL
-    for l in range(2):
+    for l in range(ms.n_layers):
         k, v = eng.gather_kv(0, l, len(prompt))
-        assert_close_large(k, st.k[l][:len(prompt)], TOL, f"K[{l}]")
-        assert_close_large(v, st.v[l][:len(prompt)], TOL, f"V[{l}]")
+        assert_close_large(k, st.k[l][:len(prompt)], TOL, f"{what} K[{l}]", outliers=OUTLIERS_KV)
+        assert_close_large(v, st.v[l][:len(prompt)], TOL, f"{what} V[{l}]", outliers=OUTLIERS_KV)
     lm = orc.linear(st.h_last[None], cmodel["lm_head"])[0]
     assert roots[0] == st.root or top2_margin(lm) < TIE
     if roots[0] != st.root:
         pytest.skip("argmax near-tie at the prompt's last position")
     S, _ = eng.gate(0.0)
+    record(what + " gate S", gpu=float(S[0]), oracle=orc.gate_entropy(st.h_last))
     assert abs(float(S[0]) - orc.gate_entropy(st.h_last)) < 2e-2
     # draft: head logits from the GPU's own h_last (the inputs must be identical to compare decisions)
     tree_tok, topk_ids, hlog = eng.draft(th, want_logits=True)
     olog = orc.heads_forward(h_last[0].double(), cheads, csrc)
-    for h in range(4):
+    for h in range(n_cheads):
         assert close(hlog[0, h], olog[h]) < 5e-3
         assert [int(t) for t in topk_ids[0, h, :10]] == list(orc.topk_ids(hlog[0, h].cpu().double(), 10))
     want_tok = [int(roots[0])] + [int(topk_ids[0, tree.head[v], tree.rank[v]]) for v in range(1, tree.n)]
     assert [int(t) for t in tree_tok[0]] == want_tok
-    # verify: hidden states of all 64 nodes, logits of a sample of nodes, every argmax
+    # verify: hidden states and logits of all 64 nodes, every argmax
     node_argmax, logits, hidden = eng.verify(th, tree_tok, want_logits=True, want_hidden=True)
     o_hidden, o_logits = orc.verify_tree(cmodel, sh, st, want_tok, tree.parent)
-    assert_close_large(hidden[0], o_hidden, TOL, "hidden")
-    assert_close_large(logits[0], o_logits, TOL, "logits")
-    o_arg = [int(a) for a in orc.argmax_f32(o_logits)]
+    assert_close_large(hidden[0], o_hidden, TOL, what + " hidden", outliers=OUTLIERS_HIDDEN)
+    assert_close_large(logits[0], o_logits, TOL, what + " logits", outliers=OUTLIERS_LOGITS)
     # decisions: exact on the kernel's own logits; against the oracle's logits a different token is
-    # admissible only where the oracle itself scores it within the logit tolerance of its best one
+    # admissible only where the oracle itself scores it within FLIP_MARGIN of its best one
     assert torch.equal(node_argmax[0].long().cpu(), torch.argmax(logits[0], dim=-1).cpu())
-    flips = 0
-    for v in range(tree.n):
-        gv = int(node_argmax[0, v])
-        if gv != o_arg[v]:
-            flips += 1
-            assert float(o_logits[v].max() - o_logits[v][gv]) < TOL, (v, gv, o_arg[v])
-    assert flips <= 3
+    check_argmax_flips(node_argmax[0], o_logits, FLIP_MARGIN, MAX_FLIPS_64, what)
     # accept + compaction against the oracle on the GPU's own decisions
     n_acc, gpath, gtok = eng.accept(th, tree_tok, node_argmax)
     opath = orc.accept_longest(want_tok, [int(a) for a in node_argmax[0]], tree.parent)
     assert [int(p) for p in gpath[0, :int(n_acc[0])]] == opath
     assert eng.device_status() == 0
+
+
+def test_7b_width_two_layers_against_oracle(cb):
+    _two_layer_width_against_oracle(cb, synth.shape_7b(n_layers=2), 4, 200, 7, "7B width, 2 layers")
+
+
+def test_13b_width_two_layers_against_oracle(cb):
+    """d_model 5120, 40 heads, MLP 13824, five decoding heads: the widths of the 13B configuration."""
+    _two_layer_width_against_oracle(cb, synth.shape_13b(n_layers=2), 5, 200, 11, "13B width, 2 layers")
+
+
+@pytest.mark.slow
+def test_7b_full_depth_prefill_and_verify_against_oracle(cb):
+    """All 32 layers of the 7B shape against the oracle: a 64-token prompt through cerb_prefill, then one 64-node
+    verification forward (about two minutes of host time for the oracle).  The raw error is recorded next to the
+    depth-scaled bound; decisions are compared as for the two-layer models."""
+    ms = synth.shape_7b()
+    topk = [10, 10, 10, 10]
+    model, layout, heads, eng = _engine(cb, ms, 4, topk, 256)
+    cmodel, sh = cpu(model), oracle_shape(ms)
+    prompt = [int(t) for t in synth.make_prompt(ms.vocab, 64, seq=21)]
+    tree = synth.best_first_tree(64, topk)
+    th = eng.tree(tree)
+    eng.prefill(torch.tensor([prompt], dtype=torch.int32, device="cuda"), [len(prompt)])
+    tree_tok, _, _ = eng.draft(th)
+    node_argmax, logits, hidden = eng.verify(th, tree_tok, want_logits=True, want_hidden=True)
+    lens, roots, h_last = eng.read_state()
+    kv = {l: eng.gather_kv(0, l, len(prompt)) for l in (0, 15, 31)}
+    torch.cuda.synchronize()
+    assert eng.device_status() == 0
+    st = orc.prefill(cmodel, sh, prompt, 256)
+    tol = _depth_tol(ms.n_layers)
+    record("7B, 32 layers h_last", tol=TOL, depth_tol=tol, **parity_stats(h_last[0], st.h_last, TOL))
+    assert close(h_last[0], st.h_last) < tol
+    for l, (k, v) in kv.items():
+        assert_close_large(k, st.k[l][:len(prompt)], tol, f"7B, 32 layers K[{l}]", outliers=OUTLIERS_KV_DEEP)
+        assert_close_large(v, st.v[l][:len(prompt)], tol, f"7B, 32 layers V[{l}]", outliers=OUTLIERS_KV_DEEP)
+    want_tok = [int(t) for t in tree_tok[0]]
+    # the oracle verifies the GPU's own tree (the root may sit at a near-tie after 32 layers; the candidates come
+    # from the GPU's h_last): what is compared is the forward over identical tokens
+    o_hidden, o_logits = orc.verify_tree(cmodel, sh, st, want_tok, tree.parent)
+    assert_close_large(hidden[0], o_hidden, tol, "7B, 32 layers hidden", outliers=OUTLIERS_HIDDEN_DEEP)
+    assert_close_large(logits[0], o_logits, tol, "7B, 32 layers logits", outliers=OUTLIERS_LOGITS_DEEP)
+    assert torch.equal(node_argmax[0].long().cpu(), torch.argmax(logits[0], dim=-1).cpu())
+    check_argmax_flips(node_argmax[0], o_logits, tol, 8, "7B, 32 layers")
 
 
 def test_7b_width_one_node_step_against_oracle(cb):
@@ -102,7 +157,7 @@ def test_7b_width_one_node_step_against_oracle(cb):
     node_argmax, logits, hidden = eng.verify(th1, tok, want_logits=True, want_hidden=True)
     o_hidden, o_logits = orc.verify_tree(cmodel, sh, st, [int(roots[0])], synth.single_node_tree().parent)
     assert close(hidden[0], o_hidden) < TOL
-    assert_close_large(logits[0], o_logits, TOL, "logits")
+    assert_close_large(logits[0], o_logits, TOL, "7B width, one-node step logits", outliers=OUTLIERS_LOGITS)
     assert int(node_argmax[0, 0]) == int(torch.argmax(logits[0, 0]))
     assert eng.device_status() == 0
 
@@ -275,13 +330,6 @@ def test_7b_width_batch_of_16_with_128_node_trees_against_oracle(cb):
     _, _, h_last = eng.read_state()
     assert close(h_last[pick], st.h_last) < TOL
     o_hidden, o_logits = orc.verify_tree(cmodel, sh, st, [int(t) for t in tt[pick]], tree.parent)
-    assert_close_large(hidden[pick], o_hidden, TOL, "hidden")
-    assert_close_large(logits[pick], o_logits, TOL, "logits")
-    o_arg = [int(a) for a in orc.argmax_f32(o_logits)]
-    flips = 0
-    for v in range(tree.n):
-        gv = int(node_argmax[pick, v])
-        if gv != o_arg[v]:
-            flips += 1
-            assert float(o_logits[v].max() - o_logits[v][gv]) < TOL, (v, gv, o_arg[v])
-    assert flips <= 6
+    assert_close_large(hidden[pick], o_hidden, TOL, "7B width, batch 16 x 128 nodes hidden", outliers=OUTLIERS_HIDDEN)
+    assert_close_large(logits[pick], o_logits, TOL, "7B width, batch 16 x 128 nodes logits", outliers=OUTLIERS_LOGITS)
+    check_argmax_flips(node_argmax[pick], o_logits, FLIP_MARGIN, 2 * MAX_FLIPS_64, "7B width, batch 16 x 128 nodes")
