@@ -274,6 +274,13 @@ int cerb_read_state(cerb_ctx* ctx, int32_t* len_host, int32_t* root_host, void* 
  * function: CERB_OK, or CERB_E_TIMEOUT.  Synchronises `stream`. */
 int cerb_device_status(cerb_ctx* ctx, void* stream);
 
+/* Diagnosis of a CERB_E_TIMEOUT (the paper has no counterpart): copies the four status words to out4_host
+ * without clearing them: [0] the status cerb_device_status reports, [1] a number naming the wait inside the
+ * kernel that ran out first, [2] the block that waited (x + 1000 y + 1000000 z), [3] a number naming the
+ * launch (GEMM: output columns + 100000 x rows).  Synchronises
+ * `stream`. */
+int cerb_wait_diagnosis(cerb_ctx* ctx, int32_t* out4_host, void* stream);
+
 /* Per-kernel-family device timing, for measurement only (the paper has no counterpart).  While
  * enabled, the host controller brackets each family's launches with CUDA events on the caller's
  * stream; cerb_profile_read synchronises the stream, adds up the elapsed times and launch-group

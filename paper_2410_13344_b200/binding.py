@@ -31,7 +31,7 @@ EXPORTS = [
     "cerb_prefill", "cerb_gate", "cerb_draft", "cerb_verify", "cerb_accept", "cerb_step",
     "cerb_attn_scratch_bytes", "cerb_tree_attention", "cerb_tree_ancestors", "cerb_gemm_scratch_bytes", "cerb_gemm",
     "cerb_read_state", "cerb_device_status", "cerb_launch_count", "cerb_strerror", "cerb_profile_enable",
-    "cerb_profile_read", "cerb_tree_attention_noalloc", "cerb_set_wait_cycles",
+    "cerb_profile_read", "cerb_tree_attention_noalloc", "cerb_set_wait_cycles", "cerb_wait_diagnosis",
 ]
 
 
@@ -118,6 +118,7 @@ def lib():
         L.cerb_device_status.argtypes = [C.c_void_p, C.c_void_p]
         L.cerb_profile_enable.argtypes = [C.c_void_p, C.c_int32]
         L.cerb_set_wait_cycles.argtypes = [C.c_int64]
+        L.cerb_wait_diagnosis.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.cerb_profile_read.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
@@ -319,7 +320,9 @@ class Cerberus:
     def step(self, th: TreeHandle, T: float, plant: Optional[torch.Tensor] = None):
         """One decoding step; results land in the pinned mirrors (h_S, h_mode, h_n_accept, h_tokens)
         once the stream is synchronised."""
-        _check(lib().cerb_step(self.ctx, th.handle, T, _ptr(plant), C.byref(self._step_out), _stream()), "cerb_step")
+        rc = lib().cerb_step(self.ctx, th.handle, T, _ptr(plant), C.byref(self._step_out), _stream())
+        if rc != OK:
+            raise CerbError(rc, "cerb_step (device status words %s)" % self.wait_diagnosis())
 
     def read_state(self):
         lens = np.zeros(self.B, np.int32)
@@ -345,6 +348,11 @@ class Cerberus:
         return lib().cerb_device_status(self.ctx, _stream())
 
     PROF_KINDS = ("gemm", "attention", "heads", "glue", "gate", "accept")
+
+    def wait_diagnosis(self):
+        out = (C.c_int32 * 4)()
+        _check(lib().cerb_wait_diagnosis(self.ctx, out, _stream()), "cerb_wait_diagnosis")
+        return list(out)
 
     def profile(self, on):
         """False / 0: off; True / 1: CUDA-event brackets per kernel family; 2: the GEMM kernels stamp their own

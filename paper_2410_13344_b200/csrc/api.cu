@@ -686,6 +686,13 @@ int cerb_device_status(cerb_ctx* c, void* stream) {
   return s;
 }
 
+int cerb_wait_diagnosis(cerb_ctx* c, int32_t* out4_host, void* stream) {
+  if (!c || !out4_host) return CERB_E_ARG;
+  CERB_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
+  CERB_CUDA_OK(cudaMemcpy(out4_host, c->d_status, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost));
+  return CERB_OK;
+}
+
 int cerb_profile_enable(cerb_ctx* c, int32_t on) {
   if (!c || on < 0 || on > 2) return CERB_E_ARG;
   c->prof_on = on != 0;

@@ -160,7 +160,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
         if (i == early) { griddep_wait(); griddep_launch(); }
         int s = i % STAGES;
         uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-        mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, wc);
+        mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, wc, 301);
         uint32_t fb = smem_u32(&full_bar[s]);
         mbar_expect_tx(fb, STAGE_BYTES);
         uint32_t kdst = smem_base + (uint32_t)s * STAGE_BYTES, vdst = kdst + KV_BYTES;
@@ -214,7 +214,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
     for (int t = t0, it = 0; t < t_end; ++t, ++it) {
       const int s = it % STAGES;
       const uint32_t ph = (uint32_t)(it / STAGES) & 1u;
-      mbar_wait(smem_u32(&full_bar[s]), ph, wc);
+      mbar_wait(smem_u32(&full_bar[s]), ph, wc, 302);
       const uint32_t kbase = smem_base + (uint32_t)s * STAGE_BYTES, vbase = kbase + KV_BYTES;
       const int key_tile0 = t * TILE;
       if (key_tile0 + TILE > kv_total) {
@@ -423,7 +423,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
     // in split order and writes the output.  Nobody leaves before the second meeting.
     cluster_start_wait();
     if (warp < NW) {
-      cluster_meet(&cl_bar[0], p.nsplit, (int)threadIdx.x, wc);     // every member's rows are in place
+      cluster_meet(&cl_bar[0], p.nsplit, (int)threadIdx.x, wc, 303);     // every member's rows are in place
       constexpr int C4 = DH / 4;
       const int ct = warp * 32 + lane, rows_per_pass = (NW * 32) / C4;
       const float LN2 = 0.6931471805599453f;
@@ -449,7 +449,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
         if (c4 == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
       }
       compute_bar(NW * 32);                                                          // this CTA has read all it needs
-      if (warp == 0) cluster_meet(&cl_bar[1], p.nsplit, lane, wc);
+      if (warp == 0) cluster_meet(&cl_bar[1], p.nsplit, lane, wc, 304);
     }
     __syncthreads();                           // nobody exits before warp 0 has seen every member done
   }
@@ -597,9 +597,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
         const int sk = i % SK, sv = i % SV;
         const uint32_t fk = smem_u32(&full_k[sk]), fv = smem_u32(&full_v[sv]);
         if (lane == 0) {
-          mbar_wait_polite(smem_u32(&empty_k[sk]), ((uint32_t)(i / SK) & 1u) ^ 1u, wc);
+          mbar_wait_polite(smem_u32(&empty_k[sk]), ((uint32_t)(i / SK) & 1u) ^ 1u, wc, 305);
           mbar_expect_tx(fk, TC_KV_BYTES);
-          mbar_wait_polite(smem_u32(&empty_v[sv]), ((uint32_t)(i / SV) & 1u) ^ 1u, wc);
+          mbar_wait_polite(smem_u32(&empty_v[sv]), ((uint32_t)(i / SV) & 1u) ^ 1u, wc, 306);
           mbar_expect_tx(fv, TC_KV_BYTES);
         }
         __syncwarp();
@@ -615,7 +615,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       for (int i = 0; i < T; ++i) {
         if (i == early) { griddep_wait(); griddep_launch(); }
         const int sv = i % SV;
-        mbar_wait_polite(smem_u32(&empty_v[sv]), ((uint32_t)(i / SV) & 1u) ^ 1u, wc);
+        mbar_wait_polite(smem_u32(&empty_v[sv]), ((uint32_t)(i / SV) & 1u) ^ 1u, wc, 307);
         const uint32_t fv = smem_u32(&full_v[sv]);
         mbar_expect_tx(fv, 2 * TC_KV_BYTES);
         const uint32_t kdst = k_ring + (uint32_t)sv * TC_KV_BYTES, vdst = v_ring + (uint32_t)sv * TC_KV_BYTES;
@@ -646,12 +646,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     if (lane == 0 && T > 0) {
       const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
       const uint64_t q_desc0 = desc_k_sw128(q_base), q_desc1 = desc_k_sw128(q_base + QHALF);
-      mbar_wait(smem_u32(&q_ready), 0, wc);
+      mbar_wait(smem_u32(&q_ready), 0, wc, 308);
       for (int i = 0; i < T; ++i) {
         const int g = i & 1, k = i >> 1;
-        if (!UNI) mbar_wait(smem_u32(&full_k[i % SK]), (uint32_t)(i / SK) & 1u, wc);
-        else mbar_wait(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, wc);
-        mbar_wait(smem_u32(&s_free[g]), ((uint32_t)k & 1u) ^ 1u, wc);
+        if (!UNI) mbar_wait(smem_u32(&full_k[i % SK]), (uint32_t)(i / SK) & 1u, wc, 309);
+        else mbar_wait(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, wc, 310);
+        mbar_wait(smem_u32(&s_free[g]), ((uint32_t)k & 1u) ^ 1u, wc, 311);
         tc_fence_after();
         const uint32_t kb = k_ring + (uint32_t)(i % SK) * TC_KV_BYTES;
         const uint64_t k_desc0 = desc_k_sw128(kb), k_desc1 = desc_k_sw128(kb + 8192u);
@@ -673,8 +673,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
       for (int j = 0; j < T; ++j) {
         const int g = j & 1, k = j >> 1;
-        mbar_wait(smem_u32(&p_ready[g]), (uint32_t)k & 1u, wc);
-        mbar_wait(smem_u32(&full_v[j % SV]), (uint32_t)(j / SV) & 1u, wc);
+        mbar_wait(smem_u32(&p_ready[g]), (uint32_t)k & 1u, wc, 312);
+        mbar_wait(smem_u32(&full_v[j % SV]), (uint32_t)(j / SV) & 1u, wc, 313);
         tc_fence_after();
         const uint32_t vb = v_ring + (uint32_t)(j % SV) * TC_KV_BYTES;
         const uint32_t d = tmem + 128u + (uint32_t)g * 128u;
@@ -721,7 +721,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     float m_used = -INFINITY, l = 0.f;
     int k = 0;
     for (int i = g; i < T; i += 2, ++k) {
-      mbar_wait(smem_u32(&s_full[g]), (uint32_t)k & 1u, wc);
+      mbar_wait(smem_u32(&s_full[g]), (uint32_t)k & 1u, wc, 314);
       tc_fence_after();
       float sc[64];
 #pragma unroll
@@ -759,7 +759,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       for (int j = 0; j < 64; ++j) { sc[j] = ex2(sc[j] - mu); rs4[j & 3] += sc[j]; }
       l = l * alpha + ((rs4[0] + rs4[1]) + (rs4[2] + rs4[3]));
       if (k > 0) {
-        mbar_wait(smem_u32(&pv_done[g]), (uint32_t)(k - 1) & 1u, wc);   // P buffers free, O at rest
+        mbar_wait(smem_u32(&pv_done[g]), (uint32_t)(k - 1) & 1u, wc, 315);   // P buffers free, O at rest
         tc_fence_after();
         if (__any_sync(0xffffffffu, rescale)) {
 #pragma unroll 1
@@ -780,7 +780,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
         // last, partial tile: rows past the end may hold anything (stale pool memory); zero V there so
         // that a zero probability times a non-finite value cannot poison the sum.  V travels apart
         // from K, so wait until it has landed.
-        mbar_wait(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, wc);
+        mbar_wait(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, wc, 316);
         const int first_bad = kv_total - key0;
         uint8_t* vgen = smem_gen + (v_ring - smem_base) + (size_t)(i % SV) * TC_KV_BYTES;
         for (int idx = gt; idx < (TILE - first_bad) * 16; idx += 128) {
@@ -813,7 +813,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     }
     // ---- this group's (m, l, O) rows into shared memory ----
     if (k > 0) {
-      mbar_wait(smem_u32(&pv_done[g]), (uint32_t)(k - 1) & 1u, wc);
+      mbar_wait(smem_u32(&pv_done[g]), (uint32_t)(k - 1) & 1u, wc, 317);
       tc_fence_after();
     }
     compute_bar(256);                               // every MMA has retired: all of shared memory can be reused
@@ -925,7 +925,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     // before the second meeting, so no shared memory is read after its CTA has gone.
     cluster_start_wait();
     if (warp >= 2 && warp < 10) {
-      cluster_meet(&cl_bar[0], p.nsplit, (int)threadIdx.x - 64, wc);  // every member's rows are in place
+      cluster_meet(&cl_bar[0], p.nsplit, (int)threadIdx.x - 64, wc, 318);  // every member's rows are in place
       const int ct = threadIdx.x - 64;
       const float LN2 = 0.6931471805599453f;
       const uint32_t mine = smem_u32(smem_gen);
@@ -958,7 +958,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
         if (c4 == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
       }
       compute_bar(256);                                                              // this CTA has read all it needs
-      if (warp == 2) cluster_meet(&cl_bar[1], p.nsplit, lane, wc);
+      if (warp == 2) cluster_meet(&cl_bar[1], p.nsplit, lane, wc, 319);
     }
   }
   tc_fence_before();

@@ -12,7 +12,7 @@
 //
 // Softmax.  Thread = key means a row maximum would be a reduction across threads, so none is taken per tile:
 // every query keeps a reference exponent m[q] in shared memory and p = 2^(s - m[q]) is used as long as no
-// visible score of the tile exceeds m[q] by more than 2^8 (fp32 and the two-term bf16 split of p have the
+// visible score of the tile exceeds m[q] by more than 2^30 (fp32 and the two-term bf16 split of p have the
 // exponent range for that); only when one does (the first visible key always does: m[q] starts at -1e30) the
 // four warps that share the query block agree (one named barrier per tile) to raise m[q] to the largest score
 // seen, rescale those columns of O^T and their running sums, and take the tile's scores again.  The result after the final normalisation is exact for any reference.
@@ -42,16 +42,20 @@ constexpr int KT_PAGES = KT_TILE / CERB_PAGE;      // 8 pages per tile
 constexpr uint32_t KT_UNIT = 32768;                // K (or V) of one tile: [2 halves of head_dim][128 keys][128 bytes]
 constexpr uint32_t KT_HALF = 16384;
 constexpr int KT_DH = 128, KT_ROWF = KT_DH + 4;
-constexpr float KT_RAISE = 8.0f;                   // log2 of the excess over the reference that forces a new reference
+// log2 of the excess over the reference that forces a new reference.  Everything downstream is relative (the
+// exponential, the two-term bf16 split, the fp32 sums), so the bound only has to keep 2^30 x (keys per split) x |v|
+// far inside the fp32 range.
+constexpr float KT_RAISE = 30.0f;
 constexpr float KT_UNSET = -1.0e30f;               // reference of a query that has seen no key yet: any real score exceeds it
 
 __host__ __device__ constexpr int kt_nq(int ncb) { return ncb <= 2 ? 64 : 128; }           // query columns of the MMAs
-__host__ __device__ constexpr int kt_units(int ncb) { return ncb <= 2 ? 5 : 3; }           // ring depth in 32 KB units
+__host__ __device__ constexpr int kt_units(int ncb) { return ncb <= 2 ? 4 : 3; }           // ring depth in 32 KB units
+__host__ __device__ constexpr int kt_pbufs(int ncb) { return ncb <= 2 ? 2 : 1; }           // P^T buffers
 __host__ __device__ constexpr int kt_producers(int ncb) { return ncb <= 2 ? 4 : 2; }      // TMA-issuing warps
 __host__ __device__ constexpr int kt_threads(int ncb) { return 128 * ncb + 32 * (kt_producers(ncb) + 2); }
 __host__ __device__ constexpr size_t kt_smem(int ncb) {
   // P^T (hi | lo), Q, ring, alignment slack
-  return (size_t)2 * kt_nq(ncb) * 256 + (size_t)kt_nq(ncb) * 256 + (size_t)kt_units(ncb) * KT_UNIT + 1024;
+  return (size_t)kt_pbufs(ncb) * 2 * kt_nq(ncb) * 256 + (size_t)kt_nq(ncb) * 256 + (size_t)kt_units(ncb) * KT_UNIT + 1024;
 }
 
 // Order-preserving map float -> int (for integer atomicMax on floats) and back.
@@ -68,6 +72,7 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
   constexpr int DH = KT_DH, ROWF = KT_ROWF;
   constexpr int NQ = kt_nq(NCB);                   // query columns of S^T; O^T has 2 * NQ (hi | lo)
   constexpr int NU = kt_units(NCB);
+  constexpr int PB = kt_pbufs(NCB);                // P^T buffers: with two, the stores of tile t need not wait for PV of tile t - 1
   constexpr int NSW = 4 * NCB;                     // softmax warps
   constexpr int NPROD = kt_producers(NCB);         // producer warps NSW .. NSW + NPROD - 1; then QK^T issuer, PV issuer
   constexpr int W_QK = NSW + NPROD, W_PV = W_QK + 1;
@@ -76,7 +81,7 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
   constexpr uint32_t TMEM_COLS = NQ == 64 ? 256u : 512u;           // S^T x 2 buffers, then O^T hi | lo
   constexpr uint32_t O_COL = 2u * NQ;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_u[NU], empty_u[NU], s_full[2], s_free[2], p_ready, pv_done, q_ready;
+  __shared__ __align__(8) uint64_t full_u[2][NU], empty_u[NU], s_full[2], s_free[2], p_ready[PB], pv_done[PB], q_ready;
   __shared__ __align__(8) uint64_t cl_bar[2];
   __shared__ int page_list[kMaxPagesPerCta];
   __shared__ uint32_t desc_t[CERB_MAX_NODES][4];   // per tree key: which queries of this launch see it, 32 per word
@@ -92,8 +97,8 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t p_base = smem_base;                                 // [hi, lo][64-query block][128 keys][128 B]
-  const uint32_t q_base = p_base + 2 * P_TERM;                       // [half of head_dim][NQ rows][128 B]
+  const uint32_t p_base = smem_base;                                 // [buffer][hi, lo][64-query block][128 keys][128 B]
+  const uint32_t q_base = p_base + PB * 2 * P_TERM;                       // [half of head_dim][NQ rows][128 B]
   const uint32_t ring = q_base + 2 * QHALF;                          // NU units
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
@@ -114,16 +119,19 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
   if (threadIdx.x == 0) {
     aborted_s = (*p.status != 0);
     for (int s = 0; s < NU; ++s) {
-      mbar_init(smem_u32(&full_u[s]), NPROD);
+      mbar_init(smem_u32(&full_u[0][s]), NPROD);
+      mbar_init(smem_u32(&full_u[1][s]), NPROD);
       mbar_init(smem_u32(&empty_u[s]), 1);
     }
     for (int g = 0; g < 2; ++g) {
       mbar_init(smem_u32(&s_full[g]), 1);
       mbar_init(smem_u32(&s_free[g]), NSW);
     }
-    mbar_init(smem_u32(&p_ready), NSW);
-    mbar_init(smem_u32(&pv_done), 1);
-    mbar_init(smem_u32(&q_ready), NQ / 32);
+    for (int g = 0; g < PB; ++g) {
+      mbar_init(smem_u32(&p_ready[g]), NSW);
+      mbar_init(smem_u32(&pv_done[g]), 1);
+    }
+    mbar_init(smem_u32(&q_ready), NSW);
     mbar_init(smem_u32(&cl_bar[0]), (uint32_t)p.nsplit);
     mbar_init(smem_u32(&cl_bar[1]), (uint32_t)p.nsplit);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -144,6 +152,14 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
   const uint32_t tmem = tmem_slot;                   // columns [0, 2 NQ): S^T buffers 0 / 1; [2 NQ, 4 NQ): O^T hi | lo
   float* mrg = reinterpret_cast<float*>(smem_gen);   // [NQ][ROWF] over the operand buffers, once the key loop is over
 
+  // Waiting for unit u (K units are even, V units odd) to have landed.  A parity wait only tells "the phase before
+  // the current one is complete", so every barrier needs ONE waiter that sees each of its phases in turn.  With
+  // an odd ring depth a slot holds K and V units alternately, and a K consumer looking at every other phase of a
+  // shared barrier returned at once when its wait began before the V unit in between had landed (a rare
+  // dead-lock, measured).  Hence one "landed" barrier per slot and per kind of unit: full_u[kind][slot], whose
+  // phases the one consumer of that kind sees in order.
+  auto unit_parity = [](int u) { return (uint32_t)((NU & 1) ? (u / NU) >> 1 : u / NU) & 1u; };
+  auto wait_unit = [&](int u, int site) { mbar_wait(smem_u32(&full_u[u & 1][u % NU]), unit_parity(u), wc, site); };
   if (warp >= NSW && warp < NSW + NPROD) {
     // ---------------- TMA producers ----------------
     // producer w issues boxes w, w + NPROD, ... of every unit (box = page * 2 + half of head_dim), one per lane
@@ -168,9 +184,9 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
     for (int u = 0; u < 2 * T; ++u) {
       if (u == early_units) { griddep_wait(); griddep_launch(); }
       const int slot = u % NU, t = u >> 1;
-      const uint32_t fb = smem_u32(&full_u[slot]);
+      const uint32_t fb = smem_u32(&full_u[u & 1][slot]);
       if (lane == 0) {
-        mbar_wait_polite(smem_u32(&empty_u[slot]), ((uint32_t)(u / NU) & 1u) ^ 1u, wc);
+        mbar_wait_polite(smem_u32(&empty_u[slot]), ((uint32_t)(u / NU) & 1u) ^ 1u, wc, 101);
         mbar_expect_tx(fb, KT_UNIT / NPROD);
       }
       __syncwarp();
@@ -189,11 +205,11 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
     if (lane == 0 && T > 0) {
       constexpr uint32_t idesc_s = idesc_bf16(128, NQ, false, false);
       const uint64_t q_desc0 = desc_k_sw128(q_base), q_desc1 = desc_k_sw128(q_base + QHALF);
-      mbar_wait(smem_u32(&q_ready), 0, wc);
+      mbar_wait(smem_u32(&q_ready), 0, wc, 102);
       for (int t = 0; t < T; ++t) {
         const int u = 2 * t, slot = u % NU, sb = t & 1;
-        mbar_wait(smem_u32(&full_u[slot]), (uint32_t)(u / NU) & 1u, wc);
-        mbar_wait(smem_u32(&s_free[sb]), ((uint32_t)(t >> 1) & 1u) ^ 1u, wc);
+        wait_unit(u, 103);
+        mbar_wait(smem_u32(&s_free[sb]), ((uint32_t)(t >> 1) & 1u) ^ 1u, wc, 104);
         tc_fence_after();
         const uint32_t kb = ring + (uint32_t)slot * KT_UNIT;
         const uint64_t k_desc0 = desc_k_sw128(kb), k_desc1 = desc_k_sw128(kb + KT_HALF);
@@ -216,17 +232,18 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
       constexpr uint32_t idesc_pv = idesc_bf16(128, 2 * NQ, true, true);
       for (int t = 0; t < T; ++t) {
         const int u = 2 * t + 1, slot = u % NU;
-        mbar_wait(smem_u32(&p_ready), (uint32_t)t & 1u, wc);
-        mbar_wait(smem_u32(&full_u[slot]), (uint32_t)(u / NU) & 1u, wc);
+        const int pb = t % PB;
+        mbar_wait(smem_u32(&p_ready[pb]), (uint32_t)(t / PB) & 1u, wc, 105);
+        wait_unit(u, 106);
         tc_fence_after();
         const uint32_t vb = ring + (uint32_t)slot * KT_UNIT;
         const uint32_t d = tmem + O_COL;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
-          umma_bf16(d, desc_mn_sw128(vb + ks * 2048u, KT_HALF, 1024u), desc_mn_sw128(p_base + ks * 2048u, KT_HALF, 1024u),
+          umma_bf16(d, desc_mn_sw128(vb + ks * 2048u, KT_HALF, 1024u), desc_mn_sw128(p_base + (uint32_t)pb * 2u * P_TERM + ks * 2048u, KT_HALF, 1024u),
                     idesc_pv, (t == 0 && ks == 0) ? 0u : 1u);
         umma_commit(smem_u32(&empty_u[slot]));
-        umma_commit(smem_u32(&pv_done));
+        umma_commit(smem_u32(&pv_done[pb]));
       }
     }
   } else {
@@ -238,27 +255,38 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
     const bool tree_keys = t1 * KT_TILE > L && T > 0;           // this CTA's range reaches past the prefix
     if (tree_keys) {
       // transposed ancestor masks: bit q of desc_t[j] <-> tree key j is visible to query row0 + q
-      for (int j = st; j < n_tree; j += nst) {
-        uint32_t w[4] = {0u, 0u, 0u, 0u};
-        for (int q = 0; q < nq; ++q) {
-          const uint64_t a = p.anc[(size_t)q * CERB_ANC_WORDS + (j >> 6)];
-          w[q >> 5] |= (uint32_t)((a >> (j & 63)) & 1ull) << (q & 31);
+      // A bit-matrix transposition by warp votes: a warp takes one block of 32 queries (lane = query) and one
+      // 64-bit ancestor word, and one ballot per tree key of that word gives the key's 32 visibility bits.
+      const int n_qb = (nq + 31) >> 5, n_kw = (n_tree + 63) >> 6;
+      for (int item = warp; item < n_qb * n_kw; item += NSW) {
+        const int qb = item % n_qb, kw = item / n_qb;
+        const int q = qb * 32 + lane;
+        const uint64_t a = q < nq ? p.anc[(size_t)q * CERB_ANC_WORDS + kw] : 0ull;
+        const int j_end = min(64, n_tree - kw * 64);
+        for (int jj = 0; jj < j_end; ++jj) {
+          const uint32_t bits = __ballot_sync(0xffffffffu, (a >> jj) & 1ull);
+          if (lane == (jj & 31)) desc_t[kw * 64 + jj][qb] = bits;
         }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) desc_t[j][i] = w[i];
       }
     }
     griddep_wait();
     griddep_launch();
-    if (st < NQ) {
-      // stage row `st` of Q (zeros past the last live node) in the swizzled K-major layout
-      const bool valid = st < nq;
-      const uint4* src = reinterpret_cast<const uint4*>(p.q + (((size_t)b * p.n + (valid ? st : 0)) * p.H + h) * DH);
+    {
+      // stage Q (zeros past the last live node) in the swizzled K-major layout: 16-byte pieces, NQ * 16 of them,
+      // spread over all softmax threads so that every thread has its loads in flight at once
+      constexpr int PIECES = (NQ * 16 + 128 * NCB - 1) / (128 * NCB);
+      uint4 v[PIECES];
 #pragma unroll
-      for (int c = 0; c < 16; ++c) {
-        const uint4 v = valid ? src[c] : make_uint4(0, 0, 0, 0);
-        *reinterpret_cast<uint4*>(smem_gen + (q_base - smem_base) + (uint32_t)(c >> 3) * QHALF + (uint32_t)st * 128u +
-                                  (uint32_t)(((c & 7) ^ (st & 7)) << 4)) = v;
+      for (int i = 0; i < PIECES; ++i) {
+        const int piece = st + i * nst, row = piece >> 4, c = piece & 15;
+        v[i] = row < nq ? reinterpret_cast<const uint4*>(p.q + (((size_t)b * p.n + row) * p.H + h) * DH)[c] : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int i = 0; i < PIECES; ++i) {
+        const int piece = st + i * nst, row = piece >> 4, c = piece & 15;
+        if (piece < NQ * 16)
+          *reinterpret_cast<uint4*>(smem_gen + (q_base - smem_base) + (uint32_t)(c >> 3) * QHALF + (uint32_t)row * 128u +
+                                  (uint32_t)(((c & 7) ^ (row & 7)) << 4)) = v[i];
       }
       proxy_fence();
       __syncwarp();
@@ -273,10 +301,10 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
     float l_acc[32];
 #pragma unroll
     for (int j = 0; j < 32; ++j) l_acc[j] = 0.f;
-    uint8_t* prow = smem_gen + (p_base - smem_base) + (uint32_t)(cb >> 1) * KT_HALF + (uint32_t)r * 128u;
+    uint8_t* prow0 = smem_gen + (p_base - smem_base) + (uint32_t)(cb >> 1) * KT_HALF + (uint32_t)r * 128u;
     for (int t = 0; t < T; ++t) {
       const int sb = t & 1;
-      mbar_wait(smem_u32(&s_full[sb]), (uint32_t)(t >> 1) & 1u, wc);
+      mbar_wait(smem_u32(&s_full[sb]), (uint32_t)(t >> 1) & 1u, wc, 107);
       tc_fence_after();
       float sc[32];
       const uint32_t s_addr = tmem + lane_base + (uint32_t)sb * NQ + (uint32_t)cb * 32u;
@@ -286,6 +314,16 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
       const int kpos = (t0 + t) * KT_TILE + r;
       const bool masked = (t0 + t + 1) * KT_TILE > L;           // the tile reaches past the prefix (uniform over the CTA)
       const uint32_t vis = !masked ? 0xffffffffu : kpos < L ? qmask : kpos < kv_total ? (desc_t[kpos - L][cb] & qmask) : 0u;
+      if (t == 0 && !masked) {
+        // First tile, all keys visible: the scores of its first key serve as the reference (any value within the
+        // exponent range of the true maximum does; whatever exceeds it by 2^8 later raises it the usual way).
+        if (r == 0) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if ((qmask >> j) & 1u) mr[j] = sc[j] * p.scale_log2;
+        }
+        asm volatile("bar.sync %0, 128;" ::"r"(4 + cb) : "memory");
+      }
       // scores relative to the reference, in bits: t = s * scale - m[q]; the largest decides whether m must rise
       float tmax = -INFINITY;
       if (!masked) {
@@ -338,7 +376,7 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
           }
         }
         if (t > 0 && any_change) {
-          mbar_wait(smem_u32(&pv_done), (uint32_t)(t - 1) & 1u, wc);      // O^T at rest
+          mbar_wait(smem_u32(&pv_done[(t - 1) % PB]), (uint32_t)((t - 1) / PB) & 1u, wc, 108);      // O^T at rest (PV retires in order)
           tc_fence_after();
           waited_pv = true;
           // rows of O^T = head-dim lanes of this warp's quarter; columns of this query block, both terms
@@ -383,15 +421,16 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
         const float r0 = p0 - __uint_as_float(b0 & 0xffff0000u), r1 = p1 - __uint_as_float(b1 & 0xffff0000u);
         lo[j >> 1] = __byte_perm(__float_as_uint(r0), __float_as_uint(r1), 0x7632);
       }
-      if (t > 0 && !waited_pv) {
-        mbar_wait(smem_u32(&pv_done), (uint32_t)(t - 1) & 1u, wc);        // the P^T buffer is free
+      if (t >= PB && !(PB == 1 && waited_pv)) {
+        mbar_wait(smem_u32(&pv_done[t % PB]), (uint32_t)(t / PB - 1) & 1u, wc, 109);        // this tile's P^T buffer is free
         tc_fence_after();
       }
+      uint8_t* prow = prow0 + (size_t)(t % PB) * (2 * P_TERM);
       if (cb == 0 && kpos >= kv_total) {
         // Keys past the end (only in the last tile): the row of V may hold anything (stale pool memory); zero it
         // so that a zero probability times a non-finite value cannot poison the sum.  V must have landed first.
         const int u = 2 * t + 1;
-        mbar_wait(smem_u32(&full_u[u % NU]), (uint32_t)(u / NU) & 1u, wc);
+        wait_unit(u, 110);
         uint8_t* vrow = smem_gen + (ring - smem_base) + (size_t)(u % NU) * KT_UNIT + (size_t)r * 128;
 #pragma unroll
         for (int c = 0; c < 16; ++c) *reinterpret_cast<uint4*>(vrow + (size_t)(c >> 3) * KT_HALF + (c & 7) * 16) = make_uint4(0, 0, 0, 0);
@@ -406,11 +445,11 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
       proxy_fence();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&p_ready));
+      if (lane == 0) mbar_arrive(smem_u32(&p_ready[t % PB]));
     }
     // ---- this CTA's rows (O, m, l) into shared memory ----
     if (T > 0) {
-      mbar_wait(smem_u32(&pv_done), (uint32_t)(T - 1) & 1u, wc);
+      mbar_wait(smem_u32(&pv_done[(T - 1) % PB]), (uint32_t)((T - 1) / PB) & 1u, wc, 111);
       tc_fence_after();
     }
     // row sums: transpose-reduce the 32 partials of a warp (lane q ends up with the sum for query q)
@@ -523,24 +562,37 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
     cluster_start_wait();
     if (warp < NSW) {
       const int ct = (int)threadIdx.x, nwarps = NSW;
-      cluster_meet(&cl_bar[0], p.nsplit, ct, wc);              // every member's rows are in place
+      cluster_meet(&cl_bar[0], p.nsplit, ct, wc, 112);              // every member's rows are in place
       const float LN2 = 0.6931471805599453f;
       const uint32_t mine = smem_u32(smem_gen);
       const int c4 = ct & 31;
       for (int rr = split + p.nsplit * (ct >> 5); rr < nq; rr += p.nsplit * nwarps) {
         const uint32_t row_off = (uint32_t)rr * (ROWF * 4);
+        // every member's (m, l) and this thread's four output columns, all loads in flight at once (a cluster
+        // has at most 8 members)
+        float ms[8], ls[8];
+        float4 vs[8];
+#pragma unroll
+        for (int s2 = 0; s2 < 8; ++s2) {
+          if (s2 < p.nsplit) {
+            const uint32_t base = mapa_u32(mine, (uint32_t)s2) + row_off;
+            ms[s2] = ld_cluster_f32(base + DH * 4);
+            ls[s2] = ld_cluster_f32(base + DH * 4 + 4);
+            vs[s2] = ld_cluster_v4(base + (uint32_t)c4 * 16u);
+          } else {
+            ms[s2] = -INFINITY; ls[s2] = 0.f; vs[s2] = make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+        }
         float M = -INFINITY;
-        for (int s2 = 0; s2 < p.nsplit; ++s2) M = fmaxf(M, ld_cluster_f32(mapa_u32(mine, (uint32_t)s2) + row_off + DH * 4));
-        const float u = M == -INFINITY ? 0.f : M;
+#pragma unroll
+        for (int s2 = 0; s2 < 8; ++s2) M = fmaxf(M, ms[s2]);
         float Lsum = 0.f;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s2 = 0; s2 < p.nsplit; ++s2) {
-          const uint32_t base = mapa_u32(mine, (uint32_t)s2) + row_off;
-          const float ms = ld_cluster_f32(base + DH * 4);
-          const float w = ex2(ms - u);
-          Lsum += ld_cluster_f32(base + DH * 4 + 4) * w;
-          const float4 v = ld_cluster_v4(base + (uint32_t)c4 * 16u);
-          acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+#pragma unroll
+        for (int s2 = 0; s2 < 8; ++s2) {          // split order: the sum does not depend on timing
+          const float w = ex2(ms[s2] - M);
+          Lsum += ls[s2] * w;
+          acc.x += vs[s2].x * w; acc.y += vs[s2].y * w; acc.z += vs[s2].z * w; acc.w += vs[s2].w * w;
         }
         const float inv = 1.0f / Lsum;
         *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.n + rr) * p.H + h) * DH + c4 * 4) =
@@ -548,7 +600,7 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
         if (c4 == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + rr] = (M + log2f(Lsum)) * LN2;
       }
       asm volatile("bar.sync 2, %0;" ::"r"(128 * NCB) : "memory");            // this CTA has read all it needs
-      if (warp == 0) cluster_meet(&cl_bar[1], p.nsplit, lane, wc);
+      if (warp == 0) cluster_meet(&cl_bar[1], p.nsplit, lane, wc, 113);
     }
   }
   tc_fence_before();

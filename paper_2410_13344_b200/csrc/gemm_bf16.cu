@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
   __shared__ int aborted_s;
   __shared__ unsigned int ticket_s;
   volatile int* aborted = &aborted_s;
-  const WaitCtx wc{p.wait_cycles, aborted, p.status};
+  const WaitCtx wc{p.wait_cycles, aborted, p.status, p.N + 100000 * (p.M > 999 ? 999 : p.M)};
 
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t b_bytes = (uint32_t)p.n_mma * BK * 2;
@@ -183,7 +183,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
       for (int i = pre; i < n_units; ++i) {
         const int s = i % p.stages;
         const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
-        mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, wc);
+        mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, wc, 201);
         load_w(i);
         load_x(i);
       }
@@ -201,13 +201,13 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
       while (next_segment(u, u1, p.num_kb, sg)) {
         const int buf = p.acc_bufs == 2 ? (g & 1) : 0;
         const uint32_t use = (uint32_t)(p.acc_bufs == 2 ? g >> 1 : g);      // how often this buffer was used before
-        mbar_wait(smem_u32(&acc_empty[buf]), (use & 1u) ^ 1u, wc);
+        mbar_wait(smem_u32(&acc_empty[buf]), (use & 1u) ^ 1u, wc, 202);
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)buf * p.acc_cols;
         for (int k = 0; k < sg.nkb; ++k, ++i) {
           int s = i % p.stages;
           uint32_t ph = (uint32_t)(i / p.stages) & 1u;
-          mbar_wait(smem_u32(&full_bar[s]), ph, wc);
+          mbar_wait(smem_u32(&full_bar[s]), ph, wc, 203);
           tc_fence_after();
           uint32_t a_src = smem_base + (uint32_t)s * stage_bytes;
           uint64_t bdesc = desc_k_sw128(a_src + a_bytes);
@@ -231,7 +231,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
     while (next_segment(u, u1, p.num_kb, sg)) {
       const int buf = p.acc_bufs == 2 ? (g & 1) : 0;
       const int tile = sg.job % p.tiles, mchunk = p.lock > 1 ? my_chunk : sg.job / p.tiles;
-      mbar_wait(smem_u32(&acc_full[buf]), (uint32_t)(p.acc_bufs == 2 ? g >> 1 : g) & 1u, wc);
+      mbar_wait(smem_u32(&acc_full[buf]), (uint32_t)(p.acc_bufs == 2 ? g >> 1 : g) & 1u, wc, 204);
       tc_fence_after();
       // slot = how many CTAs before this one also work on this job
       const int job_u0 = sg.job * p.num_kb;

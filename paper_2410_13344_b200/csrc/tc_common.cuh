@@ -35,15 +35,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 struct WaitCtx {
   long long budget;          // SM clock cycles a wait may take (about 2 s by default: far beyond any legitimate wait)
   volatile int* aborted;     // shared-memory flag of the CTA: set by the first wait that ran out
-  int32_t* status;           // device status word: receives CERB_E_TIMEOUT
+  int32_t* status;           // device status words: [0] receives CERB_E_TIMEOUT, [1] the site of the first wait that ran
+                             // out (a number chosen by the kernel, for diagnosis), [2] its block index (x + 1000 y),
+                             // [3] `tag`
+  int tag = 0;               // a number identifying the launch (for diagnosis)
 };
+__device__ __forceinline__ void wait_ran_out(const WaitCtx& w, int site) {
+  *w.aborted = 1;
+  if (atomicExch(w.status, CERB_E_TIMEOUT) == 0) {
+    w.status[1] = site;
+    w.status[2] = (int)(blockIdx.x + 1000u * blockIdx.y + 1000000u * blockIdx.z);
+    w.status[3] = w.tag;
+  }
+}
 // Once one wait in a CTA has run out (or an earlier kernel already reported a time-out), every later wait
 // of that CTA gives up after this many cycles, so the CTA still runs to its end in bounded time.
 constexpr long long kAbortedWaitCycles = 40000ll;
 
 // Bounded wait: gives up after the budget.  The budget is measured with the SM-local cycle counter, which is
 // cheap to read; the polls in between are back to back.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w) {
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w, int site = 0) {
   for (int i = 0; i < 1024; ++i)
     if (mbar_try_wait(bar, parity)) return;
   const long long t0 = clock64();
@@ -53,11 +64,10 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const W
       if (mbar_try_wait(bar, parity)) return;
     if (clock64() - t0 > budget) break;
   }
-  *w.aborted = 1;
-  atomicExch(w.status, CERB_E_TIMEOUT);
+  wait_ran_out(w, site);
 }
 // Same bounded wait for a lane whose warp shares an issue port with busy warps: back off between polls.
-__device__ __forceinline__ void mbar_wait_polite(uint32_t bar, uint32_t parity, const WaitCtx& w) {
+__device__ __forceinline__ void mbar_wait_polite(uint32_t bar, uint32_t parity, const WaitCtx& w, int site = 0) {
   for (int i = 0; i < 4; ++i)
     if (mbar_try_wait(bar, parity)) return;
   const long long t0 = clock64();
@@ -69,8 +79,7 @@ __device__ __forceinline__ void mbar_wait_polite(uint32_t bar, uint32_t parity, 
     }
     if (clock64() - t0 > budget) break;
   }
-  *w.aborted = 1;
-  atomicExch(w.status, CERB_E_TIMEOUT);
+  wait_ran_out(w, site);
 }
 
 // ---- TMA tile loads (no multicast anywhere) ----
@@ -175,7 +184,7 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
   return ok != 0;
 }
 // `idx` numbers the calling threads of the CTA from 0: thread s signals member s (the arrivals leave in parallel).
-__device__ __forceinline__ void cluster_meet(uint64_t* bar, int members, int idx, const WaitCtx& w) {
+__device__ __forceinline__ void cluster_meet(uint64_t* bar, int members, int idx, const WaitCtx& w, int site = 0) {
   const uint32_t local = (uint32_t)__cvta_generic_to_shared(bar);
   if (idx < members) {
     uint32_t remote;
@@ -191,8 +200,7 @@ __device__ __forceinline__ void cluster_meet(uint64_t* bar, int members, int idx
       if (mbar_try_wait_cluster(local, 0)) return;
     if (clock64() - t0 > budget) break;
   }
-  *w.aborted = 1;
-  atomicExch(w.status, CERB_E_TIMEOUT);
+  wait_ran_out(w, site);
 }
 __device__ __forceinline__ uint32_t mapa_u32(uint32_t saddr, uint32_t rank) {
   uint32_t r;

@@ -47,7 +47,7 @@ def test_gemm_f32_matches_definition(cb, M, N, K):
     assert close(out, orc.linear(X.cpu(), W.cpu()), 0) < 1e-5
 
 
-def _attention_case(cb, dtype, B, n, H, Dh, lens, max_depth, seed_id, shuffled=True, n_active=None):
+def _attention_case(cb, dtype, B, n, H, Dh, lens, max_depth, seed_id, shuffled=True, n_active=None, k_growth=0.0):
     """Builds a paged cache + tree queries, runs the kernel and the oracle, returns the two results."""
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     max_len = max(lens) + n
@@ -59,6 +59,14 @@ def _attention_case(cb, dtype, B, n, H, Dh, lens, max_depth, seed_id, shuffled=T
     q = synth.normal(synth.SEED_ATTN, 10 + seed_id, (B, n, H, Dh), 1.0, dtype=tdt, device="cuda")
     kpool = synth.normal(synth.SEED_ATTN, 20 + seed_id, (n_pool, H, 16, Dh), 1.0, dtype=tdt, device="cuda")
     vpool = synth.normal(synth.SEED_ATTN, 30 + seed_id, (n_pool, H, 16, Dh), 1.0, dtype=tdt, device="cuda")
+    if k_growth:
+        # keys grow with their position, so that scores keep rising along the cache: the running reference of an
+        # online softmax has to move many times, far beyond what N(0,1) keys ever ask for
+        for b in range(B):
+            slots = torch.arange(lens[b] + n)
+            pages = torch.from_numpy(pt[b].astype(np.int64))[slots // 16].cuda()
+            f = (1.0 + k_growth * slots.float() / float(lens[b] + n)).to(tdt).cuda()
+            kpool[pages, :, (slots % 16).cuda()] = kpool[pages, :, (slots % 16).cuda()] * f[:, None, None]
     # the unused tail of the pool holds non-finite garbage: the kernel must never let it leak
     kpool[n_pool - 3:] = float("nan")
     vpool[n_pool - 3:] = float("inf")
@@ -123,6 +131,18 @@ ATTN_CASES = [
 def test_tree_attention_bf16(cb, case):
     B, n, H, Dh, lens, md = case
     for got_o, got_l, O, l in _attention_case(cb, "bf16", B, n, H, Dh, lens, md, seed_id=ATTN_CASES.index(case)):
+        assert torch.isfinite(got_o.float()).all()
+        assert close(got_o, O, 0) < TOL_BF16
+        assert close(got_l, l, 0) < 2e-3
+
+
+@pytest.mark.parametrize("case", [(2, 64, 4, 128, [1500, 700], 5), (1, 128, 2, 128, [900], 6), (1, 16, 4, 128, [3000], 4),
+                                  (1, 64, 2, 64, [600], 5)])
+def test_tree_attention_bf16_rising_scores(cb, case):
+    """Scores that grow by tens of bits along the cache: every kernel's running softmax reference must follow
+    (rescaling what it has accumulated) without losing the early keys' share or overflowing."""
+    B, n, H, Dh, lens, md = case
+    for got_o, got_l, O, l in _attention_case(cb, "bf16", B, n, H, Dh, lens, md, seed_id=70 + n, k_growth=40.0):
         assert torch.isfinite(got_o.float()).all()
         assert close(got_o, O, 0) < TOL_BF16
         assert close(got_l, l, 0) < 2e-3
