@@ -238,21 +238,35 @@ int cerb_attn_scratch_bytes(int32_t B, int32_t n, int32_t n_heads, int32_t head_
 int cerb_tree_attention(const cerb_attn_args* args, void* stream);
 
 /* cerb_tree_attention for callers that cannot allocate device memory (the paper has no
- * counterpart; this is a packaging variant of the same kernel).  Typical cases: code running
+ * counterpart; this is a packaging variant of the same kernels).  Typical cases: code running
  * inside an allocator or memory-pool callback, a plug-in that only receives fixed buffers from its
  * host application, a process whose device-memory budget is fixed at start-up.  The split-KV
  * scratch that the caller would otherwise provide lives in a static device array inside the
  * library, CERB_STATIC_ATTN_SCRATCH_BYTES large; every GPU that loads the library holds it until
  * the process exits.  args->scratch and args->scratch_bytes are ignored; inputs and outputs are
- * still the caller's.  bf16 only.  Returns CERB_E_NOMEM when cerb_attn_scratch_bytes() for the
- * problem exceeds the static array (roughly: B * n_heads beyond a few hundred with 128-node trees).
- * This call never allocates or frees device memory.
- * The first call on each device looks up the array's device address (one runtime query); make that
- * first call outside any stream capture.  All calls share the one array and each call clears the
- * part that must start at zero on `stream`, so two calls that may overlap on the GPU (different
- * streams, no dependency) race with each other: serialise them. */
+ * still the caller's.  bf16 only.  This call never allocates or frees device memory.
+ *
+ * Limit.  CERB_E_NOMEM when cerb_attn_scratch_bytes() for the problem exceeds the static array.
+ * That size is 4096 + (328 + B * n_heads) * P * (head_dim + 4) * 4 bytes with P = the tree's node
+ * count padded to 16 / 32 / 64 / 128 (every tree above 64 nodes counts as 128).  With 16 MiB:
+ *   head_dim 128: trees of up to 16 nodes B * n_heads <= 1020 (the ticket counters' limit, CERB_E_SHAPE
+ *                 beyond it, as for the ordinary entry); up to 32 nodes <= 664; up to 64
+ *                 nodes <= 168 (batch 5 at 32 heads); trees above 64 nodes are always rejected;
+ *   head_dim  64: up to 64 nodes B * n_heads <= 635; above 64 nodes <= 153.
+ *
+ * Set-up.  The first call on each device looks up the array's device address (one runtime query,
+ * with that device current); make that first call outside any stream capture.
+ * Sharing.  All calls share the one array and each call clears, on `stream`, the part that must
+ * start at zero, so two calls that may overlap on the GPU (different streams, no dependency) race
+ * with each other: serialise them.
+ * Errors found on the device (a bounded wait that ran out, max_len smaller than a sequence's
+ * len + n) land in status words inside the array, which no call clears:
+ * cerb_tree_attention_noalloc_status synchronises `stream`, returns the first word (CERB_OK,
+ * CERB_E_TIMEOUT or CERB_E_SHAPE; the output of the call that raised it is undefined) and clears
+ * it.  Until it has been read, later calls through this entry run with shortened waits. */
 #define CERB_STATIC_ATTN_SCRATCH_BYTES (16u << 20)
 int cerb_tree_attention_noalloc(const cerb_attn_args* args, void* stream);
+int cerb_tree_attention_noalloc_status(void* stream);
 
 /* Ancestor bitmasks of a tree, the form cerb_tree_attention takes: anc_out host [n][CERB_ANC_WORDS]. */
 int cerb_tree_ancestors(const int32_t* parent, int32_t n, uint64_t* anc_out);

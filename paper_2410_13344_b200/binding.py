@@ -31,7 +31,7 @@ EXPORTS = [
     "cerb_prefill", "cerb_gate", "cerb_draft", "cerb_verify", "cerb_accept", "cerb_step",
     "cerb_attn_scratch_bytes", "cerb_tree_attention", "cerb_tree_ancestors", "cerb_gemm_scratch_bytes", "cerb_gemm",
     "cerb_read_state", "cerb_device_status", "cerb_launch_count", "cerb_strerror", "cerb_profile_enable",
-    "cerb_profile_read", "cerb_tree_attention_noalloc", "cerb_set_wait_cycles", "cerb_wait_diagnosis",
+    "cerb_profile_read", "cerb_tree_attention_noalloc", "cerb_set_wait_cycles", "cerb_wait_diagnosis", "cerb_tree_attention_noalloc_status",
 ]
 
 
@@ -111,6 +111,7 @@ def lib():
         L.cerb_tree_attention.argtypes = [C.POINTER(AttnArgs), C.c_void_p]
         L.cerb_tree_ancestors.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
         L.cerb_tree_attention_noalloc.argtypes = [C.POINTER(AttnArgs), C.c_void_p]
+        L.cerb_tree_attention_noalloc_status.argtypes = [C.c_void_p]
         L.cerb_gemm_scratch_bytes.argtypes = [C.c_int32] * 3 + [C.POINTER(C.c_size_t)]
         L.cerb_gemm.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                 C.c_void_p, C.c_size_t, C.c_void_p]
@@ -411,6 +412,11 @@ def tree_attention_noalloc(q: torch.Tensor, k_pool: torch.Tensor, v_pool: torch.
                  page_table.data_ptr(), lens.data_ptr(), _ptr(n_active), anc.data_ptr(), out.data_ptr(), _ptr(lse),
                  scale, max_len, k_pool.shape[0], None, 0)
     return lib().cerb_tree_attention_noalloc(C.byref(a), _stream())
+
+
+def tree_attention_noalloc_status() -> int:
+    """Device-side status of the calls made through tree_attention_noalloc since the last read (synchronises)."""
+    return lib().cerb_tree_attention_noalloc_status(_stream())
 
 
 def gemm(X: torch.Tensor, W: torch.Tensor, scratch: Optional[torch.Tensor] = None) -> torch.Tensor:

@@ -240,8 +240,21 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
                  cudaStream_t st) {
   const cerb_config& g = c->cfg;
   const int B = c->B, M = B * n, d = g.d_model, HD = g.n_heads * g.head_dim, F = g.mlp_dim;
+  // The host knows an upper bound of every committed length (cerb_accept adds the deepest possible path).  When
+  // that bound reaches the end of the page table, the true lengths are fetched once before giving up.
+  bool refreshed = false;
   int max_len = 0;
   for (int b = 0; b < B; ++b) {
+    if (c->h_len[b] + n > c->max_pos && !refreshed) {
+      int32_t tmp[CERB_MAX_BATCH];
+      CERB_CUDA_OK(cudaStreamSynchronize(st));
+      CERB_CUDA_OK(cudaMemcpy(tmp, c->d_len, B * sizeof(int32_t), cudaMemcpyDeviceToHost));
+      for (int i = 0; i < B; ++i) c->h_len[i] = tmp[i];
+      refreshed = true;
+      max_len = 0;
+      b = -1;
+      continue;
+    }
     if (c->h_len[b] + n > c->max_pos) return CERB_E_STATE;
     if (c->h_len[b] + n > max_len) max_len = c->h_len[b] + n;
   }
@@ -682,7 +695,11 @@ int cerb_device_status(cerb_ctx* c, void* stream) {
   CERB_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
   int32_t s = 0;
   CERB_CUDA_OK(cudaMemcpy(&s, c->d_status, sizeof(s), cudaMemcpyDeviceToHost));
-  if (s != 0) CERB_CUDA_OK(cudaMemset(c->d_status, 0, sizeof(s)));
+  if (s != 0) {
+    // a launch that gave up may have left the arrival counters of the GEMM's fused epilogue half-way
+    CERB_CUDA_OK(cudaMemset(c->d_status, 0, 4 * sizeof(int32_t)));
+    CERB_CUDA_OK(cudaMemset(c->d_gemm_tickets, 0, kGemmTickets * sizeof(unsigned int)));
+  }
   return s;
 }
 

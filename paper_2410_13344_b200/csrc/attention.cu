@@ -13,6 +13,8 @@
 // fp32 path (CERB_F32 models): plain FMA arithmetic, one CTA per (node, head, sequence).
 #include <stdlib.h>
 
+#include <atomic>
+
 #include "tc_common.cuh"
 
 namespace cerb {
@@ -1225,7 +1227,23 @@ static __device__ __align__(256) unsigned char g_static_attn_scratch[CERB_STATIC
 
 namespace {
 constexpr int kMaxDevices = 64;
-void* g_static_scratch_addr[kMaxDevices];      // device address of the array, per device, once known
+std::atomic<void*> g_static_scratch_addr[kMaxDevices];      // device address of the array, per device, once known
+
+// Set-up, once per device, with that device current.  In host code the array's name is only a handle; the
+// address a kernel can use has to be asked for.  Two threads racing here both get the same answer from the
+// runtime, so the slot is simply an atomic pointer.
+int static_scratch(void** out) {
+  int dev = -1;
+  CERB_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return CERB_E_SHAPE;
+  void* ptr = g_static_scratch_addr[dev].load(std::memory_order_acquire);
+  if (!ptr) {
+    if (cudaGetSymbolAddress(&ptr, g_static_attn_scratch) != cudaSuccess || !ptr) return CERB_E_CUDA;
+    g_static_scratch_addr[dev].store(ptr, std::memory_order_release);
+  }
+  *out = ptr;
+  return CERB_OK;
+}
 }  // namespace
 
 extern "C" int cerb_tree_attention_noalloc(const cerb_attn_args* a, void* stream) {
@@ -1236,21 +1254,13 @@ extern "C" int cerb_tree_attention_noalloc(const cerb_attn_args* a, void* stream
   if (a->head_dim != 64 && a->head_dim != 128) return CERB_E_SHAPE;
   const size_t need = attn_scratch_bytes(a->B, a->n, a->n_heads, a->head_dim);
   if (need > (size_t)CERB_STATIC_ATTN_SCRATCH_BYTES) return CERB_E_NOMEM;     // problem too large for the built-in scratch
-  int dev = -1;
-  CERB_CUDA_OK(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= kMaxDevices) return CERB_E_SHAPE;
-  if (!g_static_scratch_addr[dev]) {
-    // In host code the array's name is only a handle; the address a kernel can use has to be asked
-    // for, once per device, while that device is current.
-    void* ptr = nullptr;
-    if (cudaGetSymbolAddress(&ptr, g_static_attn_scratch) != cudaSuccess || !ptr) return CERB_E_CUDA;
-    g_static_scratch_addr[dev] = ptr;
-  }
-  void* scratch = g_static_scratch_addr[dev];
+  void* scratch = nullptr;
+  CERB_TRY(static_scratch(&scratch));
   cudaStream_t st = (cudaStream_t)stream;
-  // The array keeps whatever the previous call left: the ticket counters and the status word (the
-  // first 4 KB) must start at zero.  The partials behind them are fully rewritten before being read.
-  CERB_CUDA_OK(cudaMemsetAsync(scratch, 0, kCounterBytes, st));
+  // The array keeps whatever the previous call left.  The ticket counters must start at zero; the partials behind
+  // them are fully rewritten before being read.  The status words (the last 16 bytes of the first 4 KB) are NOT
+  // cleared here: a time-out stays visible until cerb_tree_attention_noalloc_status has read it.
+  CERB_CUDA_OK(cudaMemsetAsync(scratch, 0, kCounterBytes - 16, st));
   CUtensorMap tk, tv;
   CERB_TRY(make_pool_map(&tk, a->k_pool, a->n_pool_pages, a->n_heads, a->head_dim));
   CERB_TRY(make_pool_map(&tv, a->v_pool, a->n_pool_pages, a->n_heads, a->head_dim));
@@ -1261,3 +1271,13 @@ extern "C" int cerb_tree_attention_noalloc(const cerb_attn_args* a, void* stream
   return launch_tree_attention(nullptr, &b, &tk, &tv, 148, status, st);
 }
 
+extern "C" int cerb_tree_attention_noalloc_status(void* stream) {
+  using namespace cerb;
+  void* scratch = nullptr;
+  CERB_TRY(static_scratch(&scratch));
+  CERB_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
+  int32_t words[4] = {0, 0, 0, 0};
+  CERB_CUDA_OK(cudaMemcpy(words, (char*)scratch + kCounterBytes - 16, sizeof(words), cudaMemcpyDeviceToHost));
+  if (words[0] != 0) CERB_CUDA_OK(cudaMemset((char*)scratch + kCounterBytes - 16, 0, 16));
+  return words[0];
+}

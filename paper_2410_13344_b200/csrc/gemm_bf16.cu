@@ -103,6 +103,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
   __shared__ __align__(8) uint64_t empty_bar[MAX_STAGES];
   __shared__ __align__(8) uint64_t acc_full[2];
   __shared__ __align__(8) uint64_t acc_empty[2];
+  __shared__ __align__(8) uint64_t drain_bar[2];       // one per MMA issuer: "everything I issued has retired" (give-up path only)
   __shared__ uint32_t tmem_base_slot;
   __shared__ int aborted_s;
   __shared__ unsigned int ticket_s;
@@ -128,6 +129,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&acc_full[i]), 2);
       mbar_init(smem_u32(&acc_empty[i]), 4);
+      mbar_init(smem_u32(&drain_bar[i]), 1);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -180,12 +182,20 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
       griddep_launch();
       if (p.clk) atomicMin(p.clk, globaltimer_ns());
       for (int i = 0; i < pre; ++i) load_x(i);
+      int issued = pre;
       for (int i = pre; i < n_units; ++i) {
         const int s = i % p.stages;
         const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
         mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, wc, 201);
+        if (*aborted) break;                       // a wait ran out somewhere in this CTA: issue nothing more
         load_w(i);
         load_x(i);
+        issued = i + 1;
+      }
+      if (*aborted) {
+        // give-up path: the copies already issued still land in this CTA's shared memory; see each of them in
+        for (int i = issued > p.stages ? issued - p.stages : 0; i < issued; ++i)
+          mbar_wait_drain(smem_u32(&full_bar[i % p.stages]), (uint32_t)(i / p.stages) & 1u);
       }
     }
   } else if (warp == 1 || warp == 6) {
@@ -202,12 +212,14 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
         const int buf = p.acc_bufs == 2 ? (g & 1) : 0;
         const uint32_t use = (uint32_t)(p.acc_bufs == 2 ? g >> 1 : g);      // how often this buffer was used before
         mbar_wait(smem_u32(&acc_empty[buf]), (use & 1u) ^ 1u, wc, 202);
+        if (*aborted) break;
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)buf * p.acc_cols;
         for (int k = 0; k < sg.nkb; ++k, ++i) {
           int s = i % p.stages;
           uint32_t ph = (uint32_t)(i / p.stages) & 1u;
           mbar_wait(smem_u32(&full_bar[s]), ph, wc, 203);
+          if (*aborted) break;
           tc_fence_after();
           uint32_t a_src = smem_base + (uint32_t)s * stage_bytes;
           uint64_t bdesc = desc_k_sw128(a_src + a_bytes);
@@ -218,8 +230,14 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
             umma_bf16(d, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), p.idesc, (k > 0 || kk > 0) ? 1u : 0u);
           umma_commit(smem_u32(&empty_bar[s]));     // the stage is free once the MMAs have read it
         }
+        if (*aborted) break;
         umma_commit(smem_u32(&acc_full[buf]));       // this thread's part of the segment's accumulator is complete
         ++g;
+      }
+      if (*aborted) {
+        // give-up path: the MMAs already issued still read shared memory and write tensor memory; see them retire
+        umma_commit(smem_u32(&drain_bar[hf]));
+        mbar_wait_drain(smem_u32(&drain_bar[hf]), 0);
       }
     }
   } else {
@@ -232,6 +250,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
       const int buf = p.acc_bufs == 2 ? (g & 1) : 0;
       const int tile = sg.job % p.tiles, mchunk = p.lock > 1 ? my_chunk : sg.job / p.tiles;
       mbar_wait(smem_u32(&acc_full[buf]), (uint32_t)(p.acc_bufs == 2 ? g >> 1 : g) & 1u, wc, 204);
+      if (*aborted) break;                         // the launch's output is undefined from here on
       tc_fence_after();
       // slot = how many CTAs before this one also work on this job
       const int job_u0 = sg.job * p.num_kb;

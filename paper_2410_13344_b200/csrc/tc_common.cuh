@@ -52,19 +52,45 @@ __device__ __forceinline__ void wait_ran_out(const WaitCtx& w, int site) {
 // of that CTA gives up after this many cycles, so the CTA still runs to its end in bounded time.
 constexpr long long kAbortedWaitCycles = 40000ll;
 
-// Bounded wait: gives up after the budget.  The budget is measured with the SM-local cycle counter, which is
-// cheap to read; the polls in between are back to back.
+// mbarrier.try_wait may suspend the thread for a system-dependent time before it answers "not yet"; with a hint
+// it comes back after about that many nanoseconds, which bounds how late a time-out can be noticed.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after the budget.  A few plain polls first (almost every wait ends there); then the
+// budget is measured with the SM-local cycle counter, which is cheap to read, between short runs of polls
+// that each return after two microseconds at the latest.
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w, int site = 0) {
-  for (int i = 0; i < 1024; ++i)
+  for (int i = 0; i < 8; ++i)
     if (mbar_try_wait(bar, parity)) return;
   const long long t0 = clock64();
   const long long budget = *w.aborted ? kAbortedWaitCycles : w.budget;
   for (;;) {
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_wait(bar, parity)) return;
+    for (int i = 0; i < 16; ++i)
+      if (mbar_try_wait_hint(bar, parity, 2000u)) return;
     if (clock64() - t0 > budget) break;
   }
   wait_ran_out(w, site);
+}
+// Wait used on the way out of a CTA that has given up: for copies and MMAs that are already in flight, so that
+// none of them outlives the CTA's shared and tensor memory.  It keeps a budget of its own (what it waits for
+// was issued and will complete; the limit only guards against the unforeseen) and reports nothing.
+constexpr long long kDrainCycles = 4000000000ll;
+__device__ __forceinline__ void mbar_wait_drain(uint32_t bar, uint32_t parity) {
+  const long long t0 = clock64();
+  for (;;) {
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return;
+    if (clock64() - t0 > kDrainCycles) return;
+  }
 }
 // Same bounded wait for a lane whose warp shares an issue port with busy warps: back off between polls.
 __device__ __forceinline__ void mbar_wait_polite(uint32_t bar, uint32_t parity, const WaitCtx& w, int site = 0) {

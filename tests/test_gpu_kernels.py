@@ -201,6 +201,37 @@ def test_tree_attention_f32(cb, case):
         assert close(got_o, O, 0) < TOL_F32 and close(got_l, l, 0) < TOL_F32
 
 
+def test_bounded_wait_runs_out_cleanly_and_the_next_call_is_correct(cb):
+    """Every device-side wait has a cycle budget.  With the budget set to a thousand cycles, the epilogue warps of
+    a long GEMM (2048 rows x 256 x 262144: each CTA accumulates ~230 k blocks, about half a millisecond, before its
+    epilogue may read) run out of it by the limit alone -- nothing is skipped or broken.  The launch must report CERB_E_TIMEOUT in its status word, come
+    back (its CTAs stop issuing, see their copies and MMAs in flight retire, free their tensor memory), and the
+    same call with the default budget must then give the right result."""
+    L = cb.lib()
+    M, N, K = 2048, 256, 262144
+    X = synth.normal(13, 1, (M, K), 1.0, dtype=torch.bfloat16, device="cuda")
+    W = synth.normal(13, 2, (N, K), 0.05, dtype=torch.bfloat16, device="cuda")
+    nb = cb.C.c_size_t(0)
+    assert L.cerb_gemm_scratch_bytes(M, N, K, cb.C.byref(nb)) == cb.OK
+    scratch = torch.zeros(nb.value + 512, dtype=torch.uint8, device="cuda")
+    off = (-scratch.data_ptr()) % 256                      # where the binding places the status word
+    assert L.cerb_set_wait_cycles(100) == cb.E_ARG
+    assert L.cerb_set_wait_cycles(1000) == cb.OK
+    try:
+        cb.gemm(X, W, scratch=scratch)
+        torch.cuda.synchronize()
+        status = int(scratch[off:off + 4].view(torch.int32).item())
+    finally:
+        assert L.cerb_set_wait_cycles(4_000_000_000) == cb.OK
+    assert status == cb.E_TIMEOUT
+    out = cb.gemm(X, W, scratch=scratch)
+    torch.cuda.synchronize()
+    assert int(scratch[off:off + 4].view(torch.int32).item()) == 0
+    ri, ci = torch.arange(0, M, 197), torch.arange(0, N, 37)
+    ref = orc.linear(X[ri].cpu(), W[ci].cpu())
+    assert close(out[ri][:, ci].cpu(), ref, 0) < 2e-3          # 262144 products per element
+
+
 def test_abi_rejects_bad_arguments(cb):
     L = cb.lib()
     assert L.cerb_tree_attention(None, None) == cb.E_ARG

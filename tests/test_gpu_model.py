@@ -422,6 +422,34 @@ def test_151_node_trees(cb, dtype):
     assert eng.device_status() == 0
 
 
+def test_verify_accept_loop_runs_to_the_true_capacity(cb):
+    """The stand-alone calls keep only an upper bound of the committed length on the host (every cerb_accept adds
+    the deepest possible path).  A loop of draft / verify / accept must still run until the sequence really fills
+    its pages: the library fetches the true lengths once its bound reaches the end of the page table."""
+    ms = synth.tiny_shape("fp32")
+    rig = Rig(cb, ms, max_tokens=96, max_nodes=16)
+    eng = rig.eng
+    tree = synth.best_first_tree(16, rig.topk)
+    th = eng.tree(tree)
+    eng.prefill(torch.zeros(1, 8, dtype=torch.int32, device="cuda"), [8])
+    capacity = 16 * eng.max_pages
+    steps = 0
+    while True:
+        try:
+            tree_tok, _, _ = eng.draft(th)
+            am, _, _ = eng.verify(th, tree_tok)
+            eng.accept(th, tree_tok, am)
+        except cb.CerbError as e:
+            assert e.code == cb.E_STATE
+            break
+        steps += 1
+        assert steps < 200
+    lens, _, _ = eng.read_state()
+    # untrained heads: one token per step; the loop must have used the pages up, not stopped at the drifting bound
+    assert int(lens[0]) + tree.n > capacity and int(lens[0]) >= capacity - tree.n - 4 and steps >= 60
+    assert eng.device_status() == 0
+
+
 def test_error_codes(cb):
     ms = synth.tiny_shape("fp32")
     rig = Rig(cb, ms, max_tokens=128)
