@@ -1095,16 +1095,13 @@ static int launch_attn_window(const cerb_attn_args* a, int row0, int rows, const
   p.n = a->n;
   p.H = a->n_heads;
   p.max_pages = a->max_pages;
-  // The tcgen05 kernel's MMAs are 128 rows tall: it takes the 65..128-node trees, and the 33..64-node trees
-  // from about 1K keys per sequence (measured inside the 7B decoding step, batch 1, ms per 64-node forward,
-  // tcgen05 against warp-MMA: 4.18 / 4.18 at 512 keys, 4.20 / 4.29 at 1K, 4.21 / 4.31 at 2K, 4.50 / 4.99 at
-  // 4K, 5.02 / 6.20 at 8K; kernel alone at 2 x 2K keys 29 / 45 us), and so do the 17..32-node trees (kernel
-  // alone 20 / 30 us at 2K keys, 43 / 68 us at 8K, 523 / 552 us at 16 x 8K).  Trees of up to 16 nodes and
-  // one-node steps stay on the warp-MMA kernel, whose 16-row layout wastes no tensor work and which streams
-  // at 7.0 TB/s at batch 16 x 8K keys (the tcgen05 kernel: 4.2).  CERB_ATTN_TC=0 / 1 forces one.
+  // Which kernel: windows of 65 .. 128 rows take the tcgen05 kernel whose MMAs are 128 query rows tall; 17 .. 64 rows
+  // the keys-on-M kernel (below); up to 16 rows and one-node steps the warp-MMA kernel, whose 16-row layout wastes
+  // no tensor work and streams at 7.0 TB/s at batch 16 x 8K keys.  Short caches and head_dim 64 stay on the
+  // warp-MMA kernel too.  CERB_ATTN_TC=0 / 1 forces the warp-MMA / the query-rows-on-M tcgen05 kernel (tests).
   static const int force_tc = getenv("CERB_ATTN_TC") ? atoi(getenv("CERB_ATTN_TC")) : -1;
   const int np_ = nq_pad(rows);
-  const bool auto_tc = np_ == 128 || ((np_ == 64 || np_ == 32) && a->max_len >= 1024);
+  const bool auto_tc = np_ == 128;
   const bool tensor_path = a->head_dim == 128 && (force_tc < 0 ? auto_tc : force_tc != 0);
   // With clusters the splits of a (sequence, head) merge through distributed shared memory: at most 8 of them
   // (the portable cluster size).  CERB_ATTN_CLUSTER=0 keeps the merge through global partials (up to 32 splits).
@@ -1122,10 +1119,14 @@ static int launch_attn_window(const cerb_attn_args* a, int row0, int rows, const
   p.v_lbo = 8192u;
   p.v_sbo = 1024u;
   int np = nq_pad(rows), rc = CERB_E_SHAPE;
-  // The keys-on-M tensor-core kernel (attention_kt.cuh): 128-key tiles, every MMA row in use whatever the tree's
-  // width.  CERB_ATTN_KT=0 / 1 switches it off / forces it for every head_dim-128 launch.
+  // The keys-on-M tensor-core kernel (attention_kt.cuh; 128-key tiles, every MMA row in use whatever the tree's
+  // width) takes the trees of 17 to 64 nodes.  Measured inside the 7B decoding step, batch 1, 2K keys, this kernel
+  // against the others: 64-node steps 4.33 / 4.47 ms, one-node steps 3.39 / 3.27 ms (the 16-row warp-MMA layout has
+  // less to set up); alone at batch 16 x 8K keys: 64 nodes 403 / 537 us, 16 nodes 392 / 308 us, 128 nodes (its
+  // 128-query form, not built any more) 654 / 572 us.  CERB_ATTN_KT=0 / 1 keeps it off / uses it for every launch of
+  // up to 64 rows (tests).
   static const int force_kt = getenv("CERB_ATTN_KT") ? atoi(getenv("CERB_ATTN_KT")) : -1;
-  const bool kt_path = a->head_dim == 128 && force_tc < 0 && (force_kt < 0 ? true : force_kt != 0);
+  const bool kt_path = a->head_dim == 128 && force_tc < 0 && rows <= 64 && (force_kt < 0 ? rows > 16 : force_kt != 0);
   if (kt_path) {
     const int tiles = (a->max_len + KT_TILE - 1) / KT_TILE;
     int want = 148 / (a->B * a->n_heads);
@@ -1137,16 +1138,13 @@ static int launch_attn_window(const cerb_attn_args* a, int row0, int rows, const
     if (per * KT_PAGES > kMaxPagesPerCta) return CERB_E_SHAPE;
     p.nsplit = (tiles + per - 1) / per;
     p.cluster = (use_cluster && p.nsplit >= 2 && p.nsplit <= 8) ? 1 : 0;
-    // query blocks of 32: trees of up to 64 nodes take the two-block kernel (its MMAs are 64 queries wide anyway)
-    const int ncb = rows <= 64 ? 2 : (rows + 31) / 32;
+    constexpr int ncb = 2;             // two blocks of 32 queries: the MMAs are 64 queries wide
     static bool kt_configured = false;
     if (!kt_configured) {
       CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_kt_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kt_smem(2)));
-      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_kt_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kt_smem(3)));
-      CERB_CUDA_OK(cudaFuncSetAttribute(tree_attn_kt_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kt_smem(4)));
       kt_configured = true;
     }
-    auto kern = ncb == 2 ? tree_attn_kt_kernel<2> : ncb == 3 ? tree_attn_kt_kernel<3> : tree_attn_kt_kernel<4>;
+    auto kern = tree_attn_kt_kernel<2>;
     const dim3 grid(p.nsplit, p.H, a->B), block(kt_threads(ncb));
     if (p.cluster)
       rc = launch_pdl_cluster(kern, grid, block, kt_smem(ncb), st, (unsigned)p.nsplit, *tmK, *tmV, p) == cudaSuccess ? CERB_OK : CERB_E_CUDA;

@@ -148,14 +148,17 @@ def test_tree_attention_bf16_rising_scores(cb, case):
         assert close(got_l, l, 0) < 2e-3
 
 
-def test_global_partial_merge_path_in_a_child_process():
-    """By default the key splits merge inside a thread-block cluster.  The older route (partials in the
-    scratch buffer, merged by the CTA that arrives last) stays selectable by an environment switch that is
-    read once per process: run the bf16 attention cases again in a child process with it set."""
+@pytest.mark.parametrize("switch", ["CERB_ATTN_CLUSTER=0", "CERB_ATTN_KT=1", "CERB_ATTN_KT=0"])
+def test_other_attention_routes_in_a_child_process(switch):
+    """Environment switches that are read once per process select other routes through the attention kernels: the
+    key splits merged through partials in the scratch buffer instead of inside a thread-block cluster; the
+    keys-on-M tensor-core kernel for every launch of up to 64 query rows (by default it takes 17..64); that kernel
+    off.  Each route runs the bf16 attention cases again in a child process."""
     import os
     import subprocess
     import sys
-    env = dict(os.environ, CERB_ATTN_CLUSTER="0")
+    name, value = switch.split("=")
+    env = dict(os.environ, **{name: value})
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     r = subprocess.run([sys.executable, "-m", "pytest", "tests/test_gpu_kernels.py", "-q", "-x", "-m", "gpu", "-k",
                         "test_tree_attention_bf16"], cwd=root, env=env, capture_output=True, text=True, timeout=1200)
