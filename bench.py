@@ -368,6 +368,10 @@ def run_cerb(args, rank, world):
         "profiled_ms_per_step": ms_b / prof_steps,
         "clocks": clocks, "device_status": status, "setup_s": setup_s,
     }
+    if rank == 0 and world == 1 and args.workload == "7b" and not args.no_corner:
+        eng.close()
+        torch.cuda.empty_cache()
+        line["batched_corner"] = batched_corner(cb, ms, model, hbm_peak, tf_peak)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(ms, model, heads, layout, tree, prompt_len, tok_a / max(1, args.steps),
                                             len(par_steps) / max(1, len(modes_a)), budget_s=20.0)
@@ -403,9 +407,11 @@ def cpu_baseline(ms, model, heads, layout, tree, prompt_len, tokens_per_step, pa
     t0 = time.time()
     ns = 4 if ms.n_layers >= 8 else ms.n_layers        # 4 layers in float64 = 6.5 GB of host memory at the 7B shape
     orc, sub, sh, st, tok = _oracle_sample(ms, model, heads, layout, tree, prompt_len, ns)
+    reps = 2
     t1 = time.time()
-    orc.verify_tree(sub, sh, st, tok, tree.parent)
-    t_sample = time.time() - t1
+    for _ in range(reps):
+        orc.verify_tree(sub, sh, st, tok, tree.parent)
+    t_sample = (time.time() - t1) / reps
     t2 = time.time()
     orc.linear(torch.zeros(tree.n, ms.d_model, dtype=torch.float64), sub["lm_head"])
     t_lm = time.time() - t2
@@ -419,7 +425,7 @@ def cpu_baseline(ms, model, heads, layout, tree, prompt_len, tokens_per_step, pa
     t_step = (t_sample - t_lm) * ms.n_layers / ns + t_lm + par_fraction * t_heads
     return {"value": tokens_per_step / t_step, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
             "sample": f"one 64-node verify step through {ns} of {ms.n_layers} layers plus the LM head on a synthetic "
-                      f"{prompt_len}-token cache ({t_sample:.1f} s), layers scaled to {ms.n_layers}; heads scaled from one FC "
+                      f"{prompt_len}-token cache (mean of {reps} runs: {t_sample:.1f} s), layers scaled to {ms.n_layers}; heads scaled from one FC "
                       f"({t_fc:.2f} s); weight conversion to float64 excluded; extrapolated step {t_step:.1f} s",
             "seconds": time.time() - t0}
 
@@ -431,20 +437,24 @@ def run_reference(args, rank, world):
     n_ch, topk, n_nodes = draft_setup(args.workload)
     layout = synth.cerberus_layout(n_ch, 4)
     tree = synth.best_first_tree(n_nodes, topk)
-    # one layer of the model (the sample) plus embedding / LM head, generated on the host
+    # four layers of the model (the sample) plus embedding / LM head, generated on the host
     # (values do not matter for timing; a seeded torch generator is much faster on the host than the
     # counter-based generator the parity tests use)
-    ms1 = synth.ModelShape(1, ms.d_model, ms.n_heads, ms.head_dim, ms.mlp_dim, ms.vocab, ms.dtype)
+    # layers per step sample: four when the requested step count leaves room for it, one for long runs, so that the
+    # whole run stays within a few minutes (a sample layer costs about 0.7 s on 16 cores)
+    NS = min(ms.n_layers, 4 if args.steps + args.warmup <= 40 else 1)
+    ms1 = synth.ModelShape(NS, ms.d_model, ms.n_heads, ms.head_dim, ms.mlp_dim, ms.vocab, ms.dtype)
     g = torch.Generator().manual_seed(0)
     d_, F_, V_, HD_ = ms.d_model, ms.mlp_dim, ms.vocab, ms.n_heads * ms.head_dim
 
     def rnd(*shape, std=0.02, mean=0.0):
         return (torch.randn(*shape, generator=g) * std + mean).to(ms.torch_dtype)
 
-    model = {"embed": rnd(V_, d_), "final_norm": rnd(d_, std=0.1, mean=1.0), "lm_head": rnd(V_, d_),
-             "attn_norm.0": rnd(d_, std=0.1, mean=1.0), "wqkv.0": rnd(3 * HD_, d_), "wo.0": rnd(d_, HD_),
-             "mlp_norm.0": rnd(d_, std=0.1, mean=1.0), "wgu.0": rnd(2 * F_, d_), "wd.0": rnd(d_, F_)}
-    orc, sub, sh, st, tok = _oracle_sample(ms1, model, {}, layout, tree, prompt_len, 1)
+    model = {"embed": rnd(V_, d_), "final_norm": rnd(d_, std=0.1, mean=1.0), "lm_head": rnd(V_, d_)}
+    for l in range(NS):
+        model.update({f"attn_norm.{l}": rnd(d_, std=0.1, mean=1.0), f"wqkv.{l}": rnd(3 * HD_, d_), f"wo.{l}": rnd(d_, HD_),
+                      f"mlp_norm.{l}": rnd(d_, std=0.1, mean=1.0), f"wgu.{l}": rnd(2 * F_, d_), f"wd.{l}": rnd(d_, F_)})
+    orc, sub, sh, st, tok = _oracle_sample(ms1, model, {}, layout, tree, prompt_len, NS)
     lm_t0 = time.time()
     orc.linear(torch.zeros(tree.n, ms.d_model, dtype=torch.float64), sub["lm_head"])
     t_lm = time.time() - lm_t0
@@ -455,9 +465,9 @@ def run_reference(args, rank, world):
         if i >= args.warmup:
             times.append(time.time() - t0)
     t_sample = sum(times) / len(times)
-    t_step = t_sample * ms.n_layers + t_lm
+    t_step = t_sample * ms.n_layers / NS + t_lm
     value = 1.0 / t_step
-    sample = (f"per step: one {n_nodes}-node verify step of the oracle through 1 of {ms.n_layers} layers on a "
+    sample = (f"per step: one {n_nodes}-node verify step of the oracle through {NS} of {ms.n_layers} layers on a "
               f"synthetic {prompt_len}-token cache ({t_sample:.2f} s), scaled to {ms.n_layers} layers, plus the LM head timed once ({t_lm:.2f} s); heads and gate excluded; "
               f"one token per step")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -530,6 +540,69 @@ def run_kernel(args):
     print(json.dumps(out))
 
 
+def _verify_point(eng, ms, params, B, L, n, iters, hbm_peak, tf_peak):
+    """One point of the verify-step sweep on an engine whose B sequences hold L committed tokens: step latency
+    (undisturbed launch sequence), attention GB/s (event brackets), GEMM TFLOP/s (the kernels' own device-clock spans)."""
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    th = eng.tree(synth.random_parent_tree(n, 6, tree_id=n))
+    tok = torch.stack([synth.make_prompt(ms.vocab, n, seq=1000 + b).to(torch.int32) for b in range(B)]).cuda().contiguous()
+    run = lambda: eng.verify(th, tok)          # verify without accept leaves the committed state as it is
+    for _ in range(3):
+        run()
+    torch.cuda.synchronize()
+    e0, e1 = ev(), ev()
+    e0.record()
+    for _ in range(iters):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    step_ms = e0.elapsed_time(e1) / iters
+    k = max(2, iters // 2)
+    eng.profile(1); eng.profile_read()
+    for _ in range(k):
+        run()
+    prof = eng.profile_read()
+    eng.profile(2)
+    for _ in range(k):
+        run()
+    clk = eng.profile_read()
+    eng.profile(False)
+    M = B * n
+    gemm_b, attn_b, _ = algorithmic_bytes(ms, M, L, n, 0)
+    attn_b *= B
+    attn_ms = prof["attention"][0] / k
+    gemm_ev_ms, gemm_ck_ms = prof["gemm"][0] / k, clk["gemm"][0] / k
+    flops = 2.0 * M * params
+    bound_ms = max(flops / (tf_peak * 1e9), gemm_b / (hbm_peak * 1e6))
+    pt = {"B": B, "len": L, "n": n, "rows": M, "step_us": step_ms * 1e3,
+          "attn_us_per_layer": attn_ms / ms.n_layers * 1e3, "attn_GBs": attn_b / attn_ms / 1e6,
+          "attn_frac_of_measured": attn_b / attn_ms / 1e6 / hbm_peak, "attn_frac_of_8TBs": attn_b / attn_ms / 1e6 / HBM_NOMINAL_GBS,
+          "gemm_ms_events": gemm_ev_ms, "gemm_ms_device_clock": gemm_ck_ms,
+          "gemm_TFs": flops / gemm_ck_ms / 1e9, "gemm_frac_of_tensor_peak": flops / gemm_ck_ms / 1e9 / tf_peak,
+          "gemm_weight_GBs": gemm_b / gemm_ck_ms / 1e6, "gemm_bound": "tensor" if flops / (tf_peak * 1e9) > gemm_b / (hbm_peak * 1e6) else "hbm",
+          "gemm_frac_of_binding_roofline": bound_ms / gemm_ck_ms, "glue_ms_events": prof["glue"][0] / k}
+    eng.free_tree(th)
+    return pt
+
+
+def batched_corner(cb, ms, model, hbm_peak, tf_peak):
+    """The batched corner of the verify step: 16 sequences x 128-node trees (2048 rows per GEMM) on 512-token caches.
+    The batch-1 headline keeps the GEMMs HBM-bound; here they are bound by the tensor pipe."""
+    B, L, n = 16, 512, 128
+    HD = ms.n_heads * ms.head_dim
+    params = ms.n_layers * (3 * HD * ms.d_model + ms.d_model * HD + 3 * ms.mlp_dim * ms.d_model) + ms.vocab * ms.d_model
+    eng = cb.Cerberus(ms, model, None, None, (), max_tokens=L + 16, max_batch=B, max_nodes=128)
+    prompts = torch.stack([synth.make_prompt(ms.vocab, L, seq=b).to(torch.int32) for b in range(B)]).cuda().contiguous()
+    eng.prefill(prompts, [L] * B)
+    torch.cuda.synchronize()
+    pt = _verify_point(eng, ms, params, B, L, n, 4, hbm_peak, tf_peak)
+    pt["device_status"] = eng.device_status()
+    pt["note"] = ("one verify step, batch 16 x 128 nodes x 512 committed tokens; GEMM TFLOP/s from the kernels' own "
+                  "device-clock spans, against the measured bf16 tensor peak")
+    eng.close()
+    return pt
+
+
 def run_sweep(args):
     """The verify step alone (row a5 + a6: embedding .. LM head + argmax over every tree node) at the 7B shape over
     batch x committed KV length x tree nodes, random-parent trees of depth <= 6, KV produced by a real prefill of
@@ -557,47 +630,10 @@ def run_sweep(args):
             eng.prefill(prompts, [L] * B)
             torch.cuda.synchronize()
             for n in nodes:
-                th = eng.tree(synth.random_parent_tree(n, 6, tree_id=n))
-                tok = torch.stack([synth.make_prompt(ms.vocab, n, seq=1000 + b).to(torch.int32) for b in range(B)]).cuda().contiguous()
-                run = lambda: eng.verify(th, tok)          # verify without accept leaves the committed state as it is
-                for _ in range(3):
-                    run()
-                torch.cuda.synchronize()
-                e0, e1 = ev(), ev()
-                e0.record()
-                for _ in range(args.iters):
-                    run()
-                e1.record()
-                torch.cuda.synchronize()
-                step_ms = e0.elapsed_time(e1) / args.iters
-                k = max(2, args.iters // 2)
-                eng.profile(1); eng.profile_read()
-                for _ in range(k):
-                    run()
-                prof = eng.profile_read()
-                eng.profile(2)
-                for _ in range(k):
-                    run()
-                clk = eng.profile_read()
-                eng.profile(False)
-                M = B * n
-                gemm_b, attn_b, _ = algorithmic_bytes(ms, M, L, n, 0)
-                attn_b *= B
-                attn_ms = prof["attention"][0] / k
-                gemm_ev_ms, gemm_ck_ms = prof["gemm"][0] / k, clk["gemm"][0] / k
-                flops = 2.0 * M * params
-                bound_ms = max(flops / (tf_peak * 1e9), gemm_b / (hbm_peak * 1e6))
-                pt = {"B": B, "len": L, "n": n, "rows": M, "step_us": step_ms * 1e3,
-                      "attn_us_per_layer": attn_ms / ms.n_layers * 1e3, "attn_GBs": attn_b / attn_ms / 1e6,
-                      "attn_frac_of_measured": attn_b / attn_ms / 1e6 / hbm_peak, "attn_frac_of_8TBs": attn_b / attn_ms / 1e6 / HBM_NOMINAL_GBS,
-                      "gemm_ms_events": gemm_ev_ms, "gemm_ms_device_clock": gemm_ck_ms,
-                      "gemm_TFs": flops / gemm_ck_ms / 1e9, "gemm_frac_of_tensor_peak": flops / gemm_ck_ms / 1e9 / tf_peak,
-                      "gemm_weight_GBs": gemm_b / gemm_ck_ms / 1e6, "gemm_bound": "tensor" if flops / (tf_peak * 1e9) > gemm_b / (hbm_peak * 1e6) else "hbm",
-                      "gemm_frac_of_binding_roofline": bound_ms / gemm_ck_ms, "glue_ms_events": prof["glue"][0] / k}
+                pt = _verify_point(eng, ms, params, B, L, n, args.iters, hbm_peak, tf_peak)
                 assert eng.device_status() == 0
                 print(json.dumps(pt), flush=True)
                 points.append(pt)
-                eng.free_tree(th)
             eng.close()
             del eng, prompts
             torch.cuda.empty_cache()
@@ -624,6 +660,7 @@ def main():
     ap.add_argument("--n", type=int, default=64)
     ap.add_argument("--len", type=int, default=2048)
     ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--no-corner", action="store_true", help="skip the batched corner (batch 16 x 128 nodes) of the default line")
     ap.add_argument("--sweep", action="store_true", help="verify step alone over batch x KV length x tree nodes (7B shape)")
     ap.add_argument("--sweep-B", default="1,2,4,8,16")
     ap.add_argument("--sweep-len", default="512,2048,8192")

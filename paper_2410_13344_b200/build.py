@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libcerb.so")
-SOURCES = ["api.cu", "glue.cu", "gemm_f32.cu", "gemm_bf16.cu", "attention.cu", "heads.cu", "gate_accept.cu"]
+SOURCES = ["api.cu", "glue.cu", "gemm_f32.cu", "gemm_bf16.cu", "attention.cu", "heads.cu", "gate_accept.cu", "launch_order.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
          "-I", os.path.join(ROOT, "include"), "-I", CSRC]

@@ -234,6 +234,21 @@ int gemm(cerb_ctx* c, const void* X, const ActMaps* xm, const void* W, const CUt
   return launch_gemm_f32(c, (const float*)X, (const float*)W, c->d_part, M, N, K, st);
 }
 
+// Steps through the layer sequence of launch_order.cu while forward_rows launches: a kernel announced out of
+// turn means the table of pre-wait reads no longer describes the code.
+struct OrderCheck {
+  const int* ids;
+  int n, pos;
+  explicit OrderCheck(bool fused) : pos(0) { n = launch_order_layer(fused ? 1 : 0, &ids); }
+  bool next(int id) {
+    if (id == LO_NORM_FINAL) return pos == 0;
+    const bool ok = ids[pos] == id;
+    pos = (pos + 1) % n;
+    return ok;
+  }
+};
+#define CERB_ORDER(oc, id) do { if (!(oc).next(id)) return CERB_E_STATE; } while (0)
+
 // The base-model forward over B*n rows (tokens tok[b*stride + off + v]); ends with the final norm
 // in d_hidden.  d_nactive must already hold the live node count of every sequence.
 int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok_stride, int tok_off, int n,
@@ -258,7 +273,9 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
     if (c->h_len[b] + n > c->max_pos) return CERB_E_STATE;
     if (c->h_len[b] + n > max_len) max_len = c->h_len[b] + n;
   }
+  OrderCheck oc(c->bf16 && gemm_swiglu_fusable(M, F));
   // embedding gather fused with the first layer's attention norm
+  CERB_ORDER(oc, LO_NORM_ATTN);
   { ProfScope ps(c, K_GLUE, st);
     CERB_TRY(launch_fused_norm(c, nullptr, 0, 0, tok, tok_stride, tok_off, n, c->attn_norm[0], c->d_xn, M, st)); }
   cerb_attn_args a;
@@ -269,19 +286,25 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
   a.n_pool_pages = g.n_pool_pages; a.scratch = c->d_attn_scratch; a.scratch_bytes = c->attn_scratch_bytes;
   int ns = 1;
   for (int l = 0; l < g.n_layers; ++l) {
+    CERB_ORDER(oc, LO_GEMM_QKV);
     { ProfScope ps(c, K_GEMM, st);
       CERB_TRY(gemm(c, c->d_xn, &c->tm_xn, c->wqkv[l], c->bf16 ? &c->tm_wqkv[l] : nullptr, M, 3 * HD, d, &ns, st)); }
+    CERB_ORDER(oc, LO_ROPE);
     { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_rope_append(c, l, tree->dev, c->d_part, ns, (size_t)M * 3 * HD, B, n, st)); }
     a.k_pool = c->k_pool + (size_t)l * c->pool_layer_bytes;
     a.v_pool = c->v_pool + (size_t)l * c->pool_layer_bytes;
+    CERB_ORDER(oc, LO_ATTN);
     { ProfScope ps(c, K_ATTN, st);
       CERB_TRY(launch_tree_attention(c, &a, c->bf16 ? &c->tm_kpool[l] : nullptr, c->bf16 ? &c->tm_vpool[l] : nullptr,
                                      c->sm_count, c->d_status, st)); }
+    CERB_ORDER(oc, LO_GEMM_WO);
     { ProfScope ps(c, K_GEMM, st);
       CERB_TRY(gemm(c, c->d_attn, &c->tm_attn, c->wo[l], c->bf16 ? &c->tm_wo[l] : nullptr, M, d, HD, &ns, st)); }
     // residual add fused with the MLP norm
+    CERB_ORDER(oc, LO_NORM_MLP);
     { ProfScope ps(c, K_GLUE, st);
       CERB_TRY(launch_fused_norm(c, c->d_part, ns, (size_t)M * d, nullptr, 0, 0, n, c->mlp_norm[l], c->d_xn, M, st)); }
+    CERB_ORDER(oc, LO_GEMM_GU);
     if (c->bf16 && gemm_swiglu_fusable(M, F)) {
       // SwiGLU runs in the GEMM's epilogue: no separate kernel, no second pass over the partial sums
       ProfScope ps(c, K_GEMM, st);
@@ -292,11 +315,14 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
     } else {
       { ProfScope ps(c, K_GEMM, st);
         CERB_TRY(gemm(c, c->d_xn, &c->tm_xn, c->wgu[l], c->bf16 ? &c->tm_wgu[l] : nullptr, M, 2 * F, d, &ns, st)); }
+      CERB_ORDER(oc, LO_SWIGLU);
       { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_swiglu(c, c->d_part, ns, (size_t)M * 2 * F, c->d_act, M, st)); }
     }
+    CERB_ORDER(oc, LO_GEMM_DOWN);
     { ProfScope ps(c, K_GEMM, st);
       CERB_TRY(gemm(c, c->d_act, &c->tm_act, c->wd[l], c->bf16 ? &c->tm_wd[l] : nullptr, M, d, F, &ns, st)); }
     // residual add fused with the next layer's attention norm, or with the final norm
+    CERB_ORDER(oc, l + 1 == g.n_layers ? LO_NORM_FINAL : LO_NORM_ATTN);
     { ProfScope ps(c, K_GLUE, st);
       const bool last = l + 1 == g.n_layers;
       CERB_TRY(launch_fused_norm(c, c->d_part, ns, (size_t)M * d, nullptr, 0, 0, n, last ? c->final_norm : c->attn_norm[l + 1],

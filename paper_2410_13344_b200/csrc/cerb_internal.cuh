@@ -184,6 +184,12 @@ constexpr int kGemmTickets = 4096;
 constexpr int kGemmClockSlots = 4096;
 constexpr int kTopkChunks = 16;     // the vocabulary is cut into this many chunks for the heads' top-k
 
+// launch_order.cu: the forward's launch sequence and what each kernel reads ahead of its dependency wait
+enum { LO_SET_ACTIVE = 0, LO_NORM_ATTN, LO_GEMM_QKV, LO_ROPE, LO_ATTN, LO_GEMM_WO, LO_NORM_MLP, LO_GEMM_GU, LO_SWIGLU,
+       LO_GEMM_DOWN, LO_NORM_FINAL, LO_GEMM_LM, LO_ARGMAX };
+int launch_order_layer(int variant, const int** ids_out);     // variant 0: separate SwiGLU kernel, 1: fused into the GEMM
+int launch_order_violations(int variant);
+
 // ---- launch wrappers implemented across the .cu files (all asynchronous on `st`) ----
 
 // glue.cu

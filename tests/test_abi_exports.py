@@ -82,3 +82,52 @@ def test_gemm_scratch_size_follows_the_documented_schedule():
         assert nb.value == 256 + _slots_by_the_stated_schedule(M, N, K) * M * N * 4, (M, N, K)
     # weights leave HBM once at 2048 rows: 8 row chunks share 18 groups, a 64-block tile touches at most 2 shares
     assert _slots_by_the_stated_schedule(2048, 22016, 4096) == 2
+
+
+def _launch_table(variant):
+    from paper_2410_13344_b200 import binding
+    buf = ctypes.create_string_buffer(1 << 14)
+    rc = binding.lib().cerb_launch_order_table(variant, buf, len(buf))
+    rows = [line.split("|") for line in buf.value.decode().strip().split("\n")]
+    return rc, [(int(r[0]), r[1], int(r[2]), int(r[3])) for r in rows]
+
+
+def test_no_kernel_reads_before_its_wait_what_the_kernel_in_front_writes():
+    """Kernels of the forward start while their predecessor still runs and wait before touching its output.  Ahead of
+    the wait they may read only what is at least two launches old.  The library exports its launch sequence with,
+    per kernel, the buffers written and the buffers read ahead of the wait; the rule is recomputed here."""
+    from paper_2410_13344_b200 import binding
+    CONST = 1 << 9
+    for variant in (0, 1):
+        rc, rows = _launch_table(variant)
+        assert rc == binding.OK
+        names = [r[1] for r in rows]
+        assert sum("gemm" in n for n in names) == 3 * 4 + 1 and sum(n == "tree attention" for n in names) == 3
+        assert ("swiglu" in names) == (variant == 0)
+        for i, (_, name, _, reads) in enumerate(rows):
+            for bit in range(9):
+                if not reads >> bit & 1:
+                    continue
+                writers = [j for j in range(i) if rows[j][2] >> bit & 1]
+                assert not writers or i - writers[-1] >= 2, (variant, name, bit, rows[writers[-1]][1])
+        # nothing claims to write the constants, and every GEMM reads only constants (its weights) ahead of its wait
+        assert all(not w & CONST for _, _, w, _ in rows)
+        assert all(r == CONST for _, n, _, r in rows if n.startswith("gemm"))
+
+
+def test_every_forward_kernel_releases_its_dependents_after_its_own_wait():
+    """The two-launches rule above rests on every kernel calling griddepcontrol.launch_dependents only after its
+    own griddepcontrol.wait: checked on the sources, kernel by kernel (first trigger after first wait)."""
+    src = os.path.join(ROOT, "paper_2410_13344_b200", "csrc")
+    seen = 0
+    for fn in sorted(os.listdir(src)):
+        if not fn.endswith((".cu", ".cuh")) or fn == "cerb_internal.cuh":
+            continue
+        text = open(os.path.join(src, fn)).read()
+        text = re.sub(r"//[^\n]*", "", text)
+        for body in re.split(r"__global__", text)[1:]:
+            w, t = body.find("griddep_wait()"), body.find("griddep_launch()")
+            if t >= 0:
+                seen += 1
+                assert 0 <= w < t, (fn, body[:80])
+    assert seen >= 8
