@@ -202,8 +202,9 @@ typedef struct cerb_step_out {
 } cerb_step_out;
 
 /* One decoding step, Algorithm 1: gate; sequences with S > T verify a one-node
- * tree (their root token), the others draft and verify `tree`; then accept and
- * commit.  Waits once inside, after the gate, to learn whether any sequence
+ * tree (their root token), the others draft and verify `tree` (the rows of a batch
+ * are ragged: one row for an auto-regressive sequence, n for a drafting one); then
+ * accept and commit.  Waits once inside, after the gate, to learn whether any sequence
  * drafts; everything else is asynchronous on `stream`.  plant_tok_dev: optional
  * [B][n] int32 with -1 = keep the drafted token, used to exercise acceptance with
  * untrained heads; NULL in normal use. */
@@ -330,6 +331,10 @@ int cerb_launch_order_table(int32_t variant, char* buf_host, size_t cap);
 
 /* Number of kernel launches issued by this context since load (for accounting). */
 int64_t cerb_launch_count(const cerb_ctx* ctx);
+
+/* Activation rows of the last base-model forward this context launched (for accounting): B * n for cerb_verify and
+ * the prefill chunks; for cerb_step the sum over the sequences of n (drafting) or 1 (auto-regressive). */
+int32_t cerb_last_forward_rows(const cerb_ctx* ctx);
 
 const char* cerb_strerror(int code);
 

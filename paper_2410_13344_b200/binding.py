@@ -31,7 +31,7 @@ EXPORTS = [
     "cerb_prefill", "cerb_gate", "cerb_draft", "cerb_verify", "cerb_accept", "cerb_step",
     "cerb_attn_scratch_bytes", "cerb_tree_attention", "cerb_tree_ancestors", "cerb_gemm_scratch_bytes", "cerb_gemm",
     "cerb_read_state", "cerb_device_status", "cerb_launch_count", "cerb_strerror", "cerb_profile_enable",
-    "cerb_profile_read", "cerb_tree_attention_noalloc", "cerb_set_wait_cycles", "cerb_wait_diagnosis", "cerb_tree_attention_noalloc_status", "cerb_launch_order_table",
+    "cerb_profile_read", "cerb_tree_attention_noalloc", "cerb_set_wait_cycles", "cerb_wait_diagnosis", "cerb_tree_attention_noalloc_status", "cerb_launch_order_table", "cerb_last_forward_rows",
 ]
 
 
@@ -119,6 +119,7 @@ def lib():
         L.cerb_device_status.argtypes = [C.c_void_p, C.c_void_p]
         L.cerb_profile_enable.argtypes = [C.c_void_p, C.c_int32]
         L.cerb_set_wait_cycles.argtypes = [C.c_int64]
+        L.cerb_last_forward_rows.argtypes = [C.c_void_p]
         L.cerb_launch_order_table.argtypes = [C.c_int32, C.c_char_p, C.c_size_t]
         L.cerb_wait_diagnosis.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         L.cerb_profile_read.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -367,6 +368,9 @@ class Cerberus:
         gr = (C.c_int64 * 6)()
         _check(lib().cerb_profile_read(self.ctx, ms, gr, _stream()), "cerb_profile_read")
         return {k: (ms[i], gr[i]) for i, k in enumerate(self.PROF_KINDS)}
+
+    def last_forward_rows(self) -> int:
+        return int(lib().cerb_last_forward_rows(self.ctx))
 
     def launch_count(self) -> int:
         return lib().cerb_launch_count(self.ctx)

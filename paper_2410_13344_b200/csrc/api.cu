@@ -129,6 +129,7 @@ size_t carve(cerb_ctx* c, char* base) {
   c->d_mode = b.take<int32_t>(MB);
   c->d_naccept = b.take<int32_t>(MB);
   c->d_kper = b.take<int32_t>(CERB_MAX_HEADS);
+  c->d_rowoff = b.take<int32_t>(CERB_MAX_BATCH + 1);
   c->d_S = b.take<float>(MB);
   c->d_path = b.take<int32_t>(MB * kPathMax);
   c->d_outtok = b.take<int32_t>(MB * kPathMax);
@@ -251,10 +252,14 @@ struct OrderCheck {
 
 // The base-model forward over B*n rows (tokens tok[b*stride + off + v]); ends with the final norm
 // in d_hidden.  d_nactive must already hold the live node count of every sequence.
+// rows / row_off: with ragged rows (cerb_step on a batch whose sequences chose different modes) sequence b owns the
+// rows row_off[b] .. row_off[b] + n_active[b] - 1 of every activation buffer and `rows` is their total; otherwise
+// row_off is null and sequence b owns rows b * n .. b * n + n - 1.
 int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok_stride, int tok_off, int n,
-                 cudaStream_t st) {
+                 cudaStream_t st, int rows = 0, const int32_t* row_off = nullptr) {
   const cerb_config& g = c->cfg;
-  const int B = c->B, M = B * n, d = g.d_model, HD = g.n_heads * g.head_dim, F = g.mlp_dim;
+  const int B = c->B, M = row_off ? rows : B * n, d = g.d_model, HD = g.n_heads * g.head_dim, F = g.mlp_dim;
+  c->last_rows = M;
   // The host knows an upper bound of every committed length (cerb_accept adds the deepest possible path).  When
   // that bound reaches the end of the page table, the true lengths are fetched once before giving up.
   bool refreshed = false;
@@ -277,7 +282,7 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
   // embedding gather fused with the first layer's attention norm
   CERB_ORDER(oc, LO_NORM_ATTN);
   { ProfScope ps(c, K_GLUE, st);
-    CERB_TRY(launch_fused_norm(c, nullptr, 0, 0, tok, tok_stride, tok_off, n, c->attn_norm[0], c->d_xn, M, st)); }
+    CERB_TRY(launch_fused_norm(c, nullptr, 0, 0, tok, tok_stride, tok_off, n, c->attn_norm[0], c->d_xn, M, st, row_off)); }
   cerb_attn_args a;
   memset(&a, 0, sizeof(a));
   a.dtype = g.dtype; a.B = B; a.n = n; a.n_heads = g.n_heads; a.head_dim = g.head_dim; a.max_pages = g.max_pages;
@@ -290,13 +295,13 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
     { ProfScope ps(c, K_GEMM, st);
       CERB_TRY(gemm(c, c->d_xn, &c->tm_xn, c->wqkv[l], c->bf16 ? &c->tm_wqkv[l] : nullptr, M, 3 * HD, d, &ns, st)); }
     CERB_ORDER(oc, LO_ROPE);
-    { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_rope_append(c, l, tree->dev, c->d_part, ns, (size_t)M * 3 * HD, B, n, st)); }
+    { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_rope_append(c, l, tree->dev, c->d_part, ns, (size_t)M * 3 * HD, B, n, M, st, row_off)); }
     a.k_pool = c->k_pool + (size_t)l * c->pool_layer_bytes;
     a.v_pool = c->v_pool + (size_t)l * c->pool_layer_bytes;
     CERB_ORDER(oc, LO_ATTN);
     { ProfScope ps(c, K_ATTN, st);
       CERB_TRY(launch_tree_attention(c, &a, c->bf16 ? &c->tm_kpool[l] : nullptr, c->bf16 ? &c->tm_vpool[l] : nullptr,
-                                     c->sm_count, c->d_status, st)); }
+                                     c->sm_count, c->d_status, st, row_off)); }
     CERB_ORDER(oc, LO_GEMM_WO);
     { ProfScope ps(c, K_GEMM, st);
       CERB_TRY(gemm(c, c->d_attn, &c->tm_attn, c->wo[l], c->bf16 ? &c->tm_wo[l] : nullptr, M, d, HD, &ns, st)); }
@@ -431,6 +436,7 @@ int cerb_load(const cerb_config* cfg, const cerb_weights* w, void* workspace_dev
   c->B = 0;
   c->verified_tree = nullptr;
   c->launches = 0;
+  c->last_rows = 0;
   c->prof_on = false;
   c->prof_mode = 0;
   c->gemm_clock_used = 0;
@@ -614,6 +620,8 @@ int cerb_step(cerb_ctx* c, const cerb_tree* tree, float T, const int32_t* plant_
     if (out->S_host) out->S_host[b] = S;
     if (out->mode_host) out->mode_host[b] = hs[b];
   }
+  int n_ar = 0;
+  for (int b = 0; b < B; ++b) n_ar += hs[b] == CERB_MODE_AR;
   const cerb_tree* used = (any_par && tree->n > 1) ? tree : c->single;
   const int32_t* tok = c->d_root;                       // [B][1]: the root tokens
   if (used != c->single) {
@@ -621,11 +629,24 @@ int cerb_step(cerb_ctx* c, const cerb_tree* tree, float T, const int32_t* plant_
     CERB_TRY(launch_heads(c, tree, c->d_treetok, plant_tok_dev, nullptr, nullptr, st));
     tok = c->d_treetok;
   }
-  const int n = used->n, M = B * n;
-  CERB_TRY(forward_rows(c, used, tok, n, 0, n, st));
+  const int n = used->n;
+  // A batch whose sequences chose different modes: an auto-regressive sequence contributes one row, a drafting one
+  // n rows.  The row offsets go to the device ahead of the forward's first kernel (the staging words are free:
+  // this call has just waited for the stream).
+  int M = B * n;
+  const int32_t* row_off = nullptr;
+  if (used != c->single && n_ar > 0) {
+    int32_t* ro = hs + 3 * CERB_MAX_BATCH;
+    M = 0;
+    for (int b = 0; b < B; ++b) { ro[b] = M; M += hs[b] == CERB_MODE_AR ? 1 : n; }
+    ro[B] = M;
+    CERB_CUDA_OK(cudaMemcpyAsync(c->d_rowoff, ro, (B + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    row_off = c->d_rowoff;
+  }
+  CERB_TRY(forward_rows(c, used, tok, n, 0, n, st, M, row_off));
   CERB_TRY(lm_head_argmax(c, c->d_hidden, &c->tm_hidden, M, c->d_argmax, nullptr, st));
   { ProfScope ps(c, K_ACCEPT, st);
-    CERB_TRY(launch_accept(c, used, tok, c->d_nactive, c->d_argmax, out->n_accept_dev, c->d_path, out->tokens_dev, st)); }
+    CERB_TRY(launch_accept(c, used, tok, c->d_nactive, c->d_argmax, out->n_accept_dev, c->d_path, out->tokens_dev, st, row_off)); }
   for (int b = 0; b < B; ++b) c->h_len[b] += used->max_depth + 1;
   if (out->n_accept_host)
     CERB_CUDA_OK(cudaMemcpyAsync(out->n_accept_host, out->n_accept_dev, B * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
@@ -777,6 +798,8 @@ int cerb_profile_read(cerb_ctx* c, double* ms_out, int64_t* groups_out, void* st
 }
 
 int64_t cerb_launch_count(const cerb_ctx* c) { return c ? c->launches : -1; }
+
+int32_t cerb_last_forward_rows(const cerb_ctx* c) { return c ? c->last_rows : -1; }
 
 int cerb_set_wait_cycles(int64_t cycles) {
   if (cycles < 1000) return CERB_E_ARG;

@@ -71,6 +71,7 @@ struct AttnParams {
   const int32_t* len;
   const int32_t* n_active;
   const uint64_t* anc;
+  const int32_t* row_off;   // first row of every sequence in q / out, or null: sequence b starts at row b * n
   bf16* out;
   float* lse;
   float* partial;           // [B*H][nsplit][NQ][DH+4]
@@ -121,6 +122,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int L = p.len[b];
   const int nq_all = p.n_active ? min(p.n_active[b], p.n) : p.n;      // live nodes of this sequence
+  const size_t qrow = p.row_off ? (size_t)p.row_off[b] : (size_t)b * p.n;   // this sequence's first row of q and out
   const int nq = min(nq_all - p.row0, p.rows);                        // live query rows of this launch
   if (nq <= 0) return;
   const int kv_total = L + min(nq_all, p.row0 + p.rows);
@@ -190,8 +192,8 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
     // Q fragments straight from global memory (A operand of m16n8k16, one per 16 head-dim elements)
     uint32_t qa[DH / 16][4];
     {
-      const bf16* q0 = p.q + (((size_t)b * p.n + r0) * p.H + h) * DH;
-      const bf16* q1 = p.q + (((size_t)b * p.n + r1) * p.H + h) * DH;
+      const bf16* q0 = p.q + ((qrow + r0) * p.H + h) * DH;
+      const bf16* q1 = p.q + ((qrow + r1) * p.H + h) * DH;
 #pragma unroll
       for (int kk = 0; kk < DH / 16; ++kk) {
         int c = kk * 16 + tq * 2;
@@ -369,7 +371,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
       for (int idx = ct; idx < nq * DH; idx += nct) {
         int r = idx / DH, c = idx % DH;
         float l = mrg[(size_t)r * ROWF + DH + 1];
-        p.out[(((size_t)b * p.n + r) * p.H + h) * DH + c] = __float2bfloat16_rn(mrg[(size_t)r * ROWF + c] / l);
+        p.out[((qrow + r) * p.H + h) * DH + c] = __float2bfloat16_rn(mrg[(size_t)r * ROWF + c] / l);
       }
       if (p.lse)
         for (int r = ct; r < nq; r += nct)
@@ -413,7 +415,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
             acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
           }
           uint2 packed = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
-          *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.n + r) * p.H + h) * DH + c4 * 4) = packed;
+          *reinterpret_cast<uint2*>(p.out + ((qrow + r) * p.H + h) * DH + c4 * 4) = packed;
         }
         if (ct == 0) p.counters[b * p.H + h] = 0u;       // ready for the next launch
       }
@@ -446,7 +448,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
           acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
         }
         const float inv = 1.0f / Lsum;
-        *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.n + r) * p.H + h) * DH + c4 * 4) =
+        *reinterpret_cast<uint2*>(p.out + ((qrow + r) * p.H + h) * DH + c4 * 4) =
             make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
         if (c4 == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
       }
@@ -532,6 +534,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
   const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int L = p.len[b];
   const int nq_all = p.n_active ? min(p.n_active[b], p.n) : p.n;      // live nodes of this sequence
+  const size_t qrow = p.row_off ? (size_t)p.row_off[b] : (size_t)b * p.n;   // this sequence's first row of q and out
   const int nq = min(nq_all - p.row0, p.rows);                        // live query rows of this launch
   if (nq <= 0) return;
   const int kv_total = L + min(nq_all, p.row0 + p.rows);
@@ -702,7 +705,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     griddep_launch();
     if (g == 0) {
       // stage this row of Q (zeros past the last node) in the swizzled K-major layout
-      const uint4* src = reinterpret_cast<const uint4*>(p.q + (((size_t)b * p.n + (valid ? row : 0)) * p.H + h) * DH);
+      const uint4* src = reinterpret_cast<const uint4*>(p.q + ((qrow + (valid ? row : 0)) * p.H + h) * DH);
 #pragma unroll
       for (int c = 0; c < 16; ++c) {
         uint4 v = valid ? src[c] : make_uint4(0, 0, 0, 0);
@@ -871,7 +874,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
         const int r = idx / (DH / 4), c4 = idx % (DH / 4);
         const float inv = 1.0f / mrg[(size_t)r * ROWF + DH + 1];
         const float4 v = *reinterpret_cast<const float4*>(mrg + (size_t)r * ROWF + c4 * 4);
-        *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.n + r) * p.H + h) * DH + c4 * 4) =
+        *reinterpret_cast<uint2*>(p.out + ((qrow + r) * p.H + h) * DH + c4 * 4) =
             make_uint2(pack_bf16(v.x * inv, v.y * inv), pack_bf16(v.z * inv, v.w * inv));
       }
       if (p.lse)
@@ -913,7 +916,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
             const float w = wts[s2 * RP + r];
             acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
           }
-          *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.n + r) * p.H + h) * DH + c4 * 4) =
+          *reinterpret_cast<uint2*>(p.out + ((qrow + r) * p.H + h) * DH + c4 * 4) =
               make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
         }
         if (ct == 0) p.counters[b * p.H + h] = 0u;          // ready for the next launch
@@ -955,7 +958,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
           }
         }
         const float inv = 1.0f / Lsum;
-        *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.n + r) * p.H + h) * DH + c4 * 4) =
+        *reinterpret_cast<uint2*>(p.out + ((qrow + r) * p.H + h) * DH + c4 * 4) =
             make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
         if (c4 == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
       }
@@ -983,7 +986,7 @@ __global__ void __launch_bounds__(128) tree_attn_f32_kernel(const float* __restr
                                                             const int32_t* __restrict__ n_active,
                                                             const uint64_t* __restrict__ anc, float* __restrict__ out,
                                                             float* __restrict__ lse, int n, int H, int max_pages,
-                                                            float scale) {
+                                                            float scale, const int32_t* __restrict__ row_off) {
   constexpr int E = DH / 32;
   __shared__ float s_o[4][DH];
   __shared__ float s_m[4], s_l[4];
@@ -995,7 +998,8 @@ __global__ void __launch_bounds__(128) tree_attn_f32_kernel(const float* __restr
   const int L = len[b], warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint64_t a0 = anc[i * CERB_ANC_WORDS], a1 = anc[i * CERB_ANC_WORDS + 1], a2 = anc[i * CERB_ANC_WORDS + 2];
   float qv[E], acc[E];
-  const float* qp = q + (((size_t)b * n + i) * H + h) * DH;
+  const size_t qrow = row_off ? (size_t)row_off[b] : (size_t)b * n;
+  const float* qp = q + ((qrow + i) * H + h) * DH;
   for (int e = 0; e < E; ++e) { qv[e] = qp[lane + 32 * e]; acc[e] = 0.f; }
   float m = -INFINITY, l = 0.f;
   for (int kpos = warp; kpos < L + nq; kpos += 4) {
@@ -1023,7 +1027,7 @@ __global__ void __launch_bounds__(128) tree_attn_f32_kernel(const float* __restr
   for (int c = threadIdx.x; c < DH; c += 128) {
     float a = 0.f;
     for (int w = 0; w < 4; ++w) a += s_m[w] == -INFINITY ? 0.f : s_o[w][c] * expf(s_m[w] - M);
-    out[(((size_t)b * n + i) * H + h) * DH + c] = a / Ls;
+    out[((qrow + i) * H + h) * DH + c] = a / Ls;
   }
   if (threadIdx.x == 0 && lse) lse[((size_t)b * H + h) * n + i] = M + logf(Ls);
 }
@@ -1076,7 +1080,7 @@ constexpr int kAttnRowsPerLaunch = 128;
 
 // One launch of the bf16 kernels over query rows row0 .. row0 + rows - 1 (rows <= 128) of every sequence's tree.
 static int launch_attn_window(const cerb_attn_args* a, int row0, int rows, const CUtensorMap* tmK, const CUtensorMap* tmV,
-                              int32_t* status, cudaStream_t st) {
+                              int32_t* status, cudaStream_t st, const int32_t* row_off) {
   AttnParams p;
   const size_t row_elems = (size_t)a->n_heads * a->head_dim;
   p.q = (const bf16*)a->q + (size_t)row0 * row_elems;
@@ -1084,6 +1088,7 @@ static int launch_attn_window(const cerb_attn_args* a, int row0, int rows, const
   p.len = a->len;
   p.n_active = a->n_active;
   p.anc = a->anc + (size_t)row0 * CERB_ANC_WORDS;
+  p.row_off = row_off;
   p.out = (bf16*)a->out + (size_t)row0 * row_elems;
   p.lse = a->lse ? a->lse + row0 : nullptr;
   p.row0 = row0;
@@ -1180,18 +1185,18 @@ static int launch_attn_window(const cerb_attn_args* a, int row0, int rows, const
 }
 
 int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMap* tmK, const CUtensorMap* tmV,
-                          int sm_count, int32_t* status, cudaStream_t st) {
+                          int sm_count, int32_t* status, cudaStream_t st, const int32_t* row_off) {
   (void)sm_count;
   if (a->dtype == CERB_F32) {
     dim3 grid(a->n, a->n_heads, a->B);
     if (a->head_dim == 64)
       tree_attn_f32_kernel<64><<<grid, 128, 0, st>>>((const float*)a->q, (const float*)a->k_pool, (const float*)a->v_pool,
                                                      a->page_table, a->len, a->n_active, a->anc, (float*)a->out, a->lse,
-                                                     a->n, a->n_heads, a->max_pages, a->scale);
+                                                     a->n, a->n_heads, a->max_pages, a->scale, row_off);
     else if (a->head_dim == 128)
       tree_attn_f32_kernel<128><<<grid, 128, 0, st>>>((const float*)a->q, (const float*)a->k_pool, (const float*)a->v_pool,
                                                       a->page_table, a->len, a->n_active, a->anc, (float*)a->out, a->lse,
-                                                      a->n, a->n_heads, a->max_pages, a->scale);
+                                                      a->n, a->n_heads, a->max_pages, a->scale, row_off);
     else
       return CERB_E_SHAPE;
     CERB_LAUNCH_CHECK(c);
@@ -1205,7 +1210,7 @@ int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMa
   // whole tree, rows of the first only nodes below 128 (an ancestor has a lower index than its descendant).
   for (int row0 = 0; row0 < a->n; row0 += kAttnRowsPerLaunch) {
     const int rows = a->n - row0 < kAttnRowsPerLaunch ? a->n - row0 : kAttnRowsPerLaunch;
-    CERB_TRY(launch_attn_window(a, row0, rows, tmK, tmV, status, st));
+    CERB_TRY(launch_attn_window(a, row0, rows, tmK, tmV, status, st, row_off));
     CERB_LAUNCH_CHECK(c);
   }
   return CERB_OK;

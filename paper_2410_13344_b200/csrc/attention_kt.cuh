@@ -106,6 +106,7 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
   // everything up to the first use of Q or of this step's tree keys runs before griddep_wait().
   const int L = p.len[b];
   const int nq_all = p.n_active ? min(p.n_active[b], p.n) : p.n;      // live nodes of this sequence
+  const size_t qrow = p.row_off ? (size_t)p.row_off[b] : (size_t)b * p.n;   // this sequence's first row of q and out
   const int nq = min(nq_all - p.row0, p.rows);                        // live query rows of this launch
   if (nq <= 0) return;                                                // (uniform over a cluster)
   const int n_tree = min(nq_all, p.row0 + p.rows);                    // tree keys these rows can see
@@ -279,7 +280,7 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
 #pragma unroll
       for (int i = 0; i < PIECES; ++i) {
         const int piece = st + i * nst, row = piece >> 4, c = piece & 15;
-        v[i] = row < nq ? reinterpret_cast<const uint4*>(p.q + (((size_t)b * p.n + row) * p.H + h) * DH)[c] : make_uint4(0, 0, 0, 0);
+        v[i] = row < nq ? reinterpret_cast<const uint4*>(p.q + ((qrow + row) * p.H + h) * DH)[c] : make_uint4(0, 0, 0, 0);
       }
 #pragma unroll
       for (int i = 0; i < PIECES; ++i) {
@@ -503,7 +504,7 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
         const int rr = idx / (DH / 4), c4 = idx % (DH / 4);
         const float inv = 1.0f / mrg[(size_t)rr * ROWF + DH + 1];
         const float4 v = *reinterpret_cast<const float4*>(mrg + (size_t)rr * ROWF + c4 * 4);
-        *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.n + rr) * p.H + h) * DH + c4 * 4) =
+        *reinterpret_cast<uint2*>(p.out + ((qrow + rr) * p.H + h) * DH + c4 * 4) =
             make_uint2(pack_bf16(v.x * inv, v.y * inv), pack_bf16(v.z * inv, v.w * inv));
       }
       if (p.lse)
@@ -547,7 +548,7 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
             const float w = wts[s2 * RP + rr];
             acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
           }
-          *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.n + rr) * p.H + h) * DH + c4 * 4) =
+          *reinterpret_cast<uint2*>(p.out + ((qrow + rr) * p.H + h) * DH + c4 * 4) =
               make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
         }
         if (ct == 0) p.counters[b * p.H + h] = 0u;          // ready for the next launch
@@ -595,7 +596,7 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
           acc.x += vs[s2].x * w; acc.y += vs[s2].y * w; acc.z += vs[s2].z * w; acc.w += vs[s2].w * w;
         }
         const float inv = 1.0f / Lsum;
-        *reinterpret_cast<uint2*>(p.out + (((size_t)b * p.n + rr) * p.H + h) * DH + c4 * 4) =
+        *reinterpret_cast<uint2*>(p.out + ((qrow + rr) * p.H + h) * DH + c4 * 4) =
             make_uint2(pack_bf16(acc.x * inv, acc.y * inv), pack_bf16(acc.z * inv, acc.w * inv));
         if (c4 == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + rr] = (M + log2f(Lsum)) * LN2;
       }

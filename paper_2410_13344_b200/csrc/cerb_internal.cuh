@@ -136,6 +136,7 @@ struct cerb_ctx {
   // workspace carve-out
   int32_t *d_len, *d_len_old, *d_root, *d_nactive, *d_status, *d_lens_in, *d_mode, *d_naccept;
   int32_t *d_path, *d_outtok, *d_argmax, *d_treetok, *d_topk, *d_kper;
+  int32_t* d_rowoff;                  // [CERB_MAX_BATCH + 1] first row of every sequence when the rows of a step are ragged
   float* d_S;
   void *d_hlast, *d_x, *d_xn, *d_q, *d_attn, *d_act, *d_hidden;
   float *d_part, *d_logits, *d_hlogits;
@@ -160,6 +161,7 @@ struct cerb_ctx {
   int h_len[CERB_MAX_BATCH];          // upper bound of the committed length per sequence
   const cerb_tree* verified_tree;     // tree of the last cerb_verify not yet accepted
   int64_t launches;
+  int last_rows;                      // rows of the last forward (for accounting)
   int sm_count;
 
   // optional per-family timing (cerb_profile_*)
@@ -195,9 +197,10 @@ int launch_order_violations(int variant);
 // glue.cu
 int launch_rope_table(cerb_ctx* c, cudaStream_t st);
 int launch_fused_norm(cerb_ctx* c, const float* part, int nsplit, size_t split_stride, const int32_t* tok, int tok_stride,
-                      int tok_off, int n, const void* gain, void* out, int rows, cudaStream_t st);
+                      int tok_off, int n, const void* gain, void* out, int rows, cudaStream_t st,
+                      const int32_t* row_off = nullptr);
 int launch_rope_append(cerb_ctx* c, int layer, const TreeDev& t, const float* part, int nsplit, size_t split_stride,
-                       int B, int n, cudaStream_t st);
+                       int B, int n, int rows, cudaStream_t st, const int32_t* row_off = nullptr);
 int launch_swiglu(cerb_ctx* c, const float* part, int nsplit, size_t split_stride, void* act, int rows, cudaStream_t st);
 int launch_argmax_rows(cerb_ctx* c, const float* part, int nsplit, size_t split_stride, int rows, int V, int32_t* out,
                        float* summed, cudaStream_t st);
@@ -226,8 +229,9 @@ int init_driver_api();
 // attention.cu
 size_t attn_scratch_bytes(int B, int n, int H, int Dh);
 int make_pool_map(CUtensorMap* out, const void* pool, int n_pool_pages, int H, int Dh);
+// row_off: first row of every sequence in q / out when the rows of a batch are ragged (device, [B]); null = b * n
 int launch_tree_attention(cerb_ctx* c, const cerb_attn_args* a, const CUtensorMap* tmK, const CUtensorMap* tmV,
-                          int sm_count, int32_t* status, cudaStream_t st);
+                          int sm_count, int32_t* status, cudaStream_t st, const int32_t* row_off = nullptr);
 
 // heads.cu
 int launch_heads(cerb_ctx* c, const cerb_tree* tree, int32_t* tree_tok, const int32_t* plant, int32_t* topk_out,
@@ -236,6 +240,7 @@ int launch_heads(cerb_ctx* c, const cerb_tree* tree, int32_t* tree_tok, const in
 // gate_accept.cu
 int launch_gate(cerb_ctx* c, float T, float* S, int32_t* mode, int32_t* nactive_or_null, int n_par, cudaStream_t st);
 int launch_accept(cerb_ctx* c, const cerb_tree* tree, const int32_t* tree_tok, const int32_t* n_active,
-                  const int32_t* node_argmax, int32_t* n_accept, int32_t* path, int32_t* out_tok, cudaStream_t st);
+                  const int32_t* node_argmax, int32_t* n_accept, int32_t* path, int32_t* out_tok, cudaStream_t st,
+                  const int32_t* row_off = nullptr);
 
 }  // namespace cerb

@@ -65,7 +65,7 @@ __global__ void __launch_bounds__(CERB_MAX_NODES) accept_kernel(const int32_t* _
                                                      int32_t* __restrict__ len_old, int32_t* __restrict__ root,
                                                      const T* __restrict__ hidden, T* __restrict__ h_last, int d,
                                                      int32_t* __restrict__ n_accept, int32_t* __restrict__ path,
-                                                     int32_t* __restrict__ out_tok) {
+                                                     int32_t* __restrict__ out_tok, const int32_t* __restrict__ row_off) {
   constexpr int NWARP = CERB_MAX_NODES / 32;
   __shared__ uint32_t mword[NWARP];
   __shared__ int skey[NWARP];
@@ -75,7 +75,8 @@ __global__ void __launch_bounds__(CERB_MAX_NODES) accept_kernel(const int32_t* _
   const int b = blockIdx.x, v = threadIdx.x;
   const int na = min(n_active[b], n);
   const int32_t* tk = tok + (size_t)b * n;
-  const int32_t* am = argmax + (size_t)b * n;
+  const size_t row0 = row_off ? (size_t)row_off[b] : (size_t)b * n;      // this sequence's first row of argmax / hidden
+  const int32_t* am = argmax + row0;
   bool match = v < na && (v == 0 || tk[v] == am[parent[v]]);
   uint32_t bal = __ballot_sync(0xffffffffu, match);
   if ((v & 31) == 0) mword[v >> 5] = bal;
@@ -118,7 +119,7 @@ __global__ void __launch_bounds__(CERB_MAX_NODES) accept_kernel(const int32_t* _
     len[b] = L + cnt;
   }
   __syncthreads();
-  const T* src = hidden + ((size_t)b * n + best_s) * d;
+  const T* src = hidden + (row0 + best_s) * d;
   for (int j = threadIdx.x; j < d; j += blockDim.x) h_last[(size_t)b * d + j] = src[j];
 }
 
@@ -175,17 +176,18 @@ int launch_gate(cerb_ctx* c, float T, float* S, int32_t* mode, int32_t* nactive_
 }
 
 int launch_accept(cerb_ctx* c, const cerb_tree* tree, const int32_t* tree_tok, const int32_t* n_active,
-                  const int32_t* node_argmax, int32_t* n_accept, int32_t* path, int32_t* out_tok, cudaStream_t st) {
+                  const int32_t* node_argmax, int32_t* n_accept, int32_t* path, int32_t* out_tok, cudaStream_t st,
+                  const int32_t* row_off) {
   const cerb_config& g = c->cfg;
   const TreeDev& t = tree->dev;
   if (c->bf16)
     accept_kernel<bf16><<<c->B, CERB_MAX_NODES, 0, st>>>(tree_tok, node_argmax, n_active, t.parent, t.depth, t.anc, tree->n, c->d_len,
                                               c->d_len_old, c->d_root, (const bf16*)c->d_hidden, (bf16*)c->d_hlast,
-                                              g.d_model, n_accept, path, out_tok);
+                                              g.d_model, n_accept, path, out_tok, row_off);
   else
     accept_kernel<float><<<c->B, CERB_MAX_NODES, 0, st>>>(tree_tok, node_argmax, n_active, t.parent, t.depth, t.anc, tree->n, c->d_len,
                                                c->d_len_old, c->d_root, (const float*)c->d_hidden, (float*)c->d_hlast,
-                                               g.d_model, n_accept, path, out_tok);
+                                               g.d_model, n_accept, path, out_tok, row_off);
   CERB_LAUNCH_CHECK(c);
   if (tree->n > 1) {
     int row_bytes = g.head_dim * (int)c->esize;

@@ -24,6 +24,16 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
   return t;
 }
 
+// Which sequence and which tree node a row belongs to.  Rows are ordered [sequence][node]; with ragged rows
+// (sequences that verify a one-node tree next to sequences that verify the whole tree) sequence b starts at
+// row_off[b], otherwise at b * n.
+__device__ __forceinline__ void locate_row(int row, const int32_t* __restrict__ row_off, int B, int n, int& b, int& v) {
+  if (!row_off) { b = row / n; v = row - b * n; return; }
+  b = 0;
+  while (b + 1 < B && row_off[b + 1] <= row) ++b;
+  v = row - row_off[b];
+}
+
 // cos/sin of pos * base^(-2i/Dh), evaluated once in double precision.
 __global__ void rope_table_kernel(float2* tab, int max_pos, int half, double base) {
   int idx = blockIdx.x * blockDim.x + threadIdx.x;
@@ -68,7 +78,8 @@ __global__ void __launch_bounds__(NORM_THREADS) fused_norm_kernel(float* __restr
                                                                    size_t split_stride, const T* __restrict__ embed,
                                                                    const int32_t* __restrict__ tok, int tok_stride, int tok_off,
                                                                    const int32_t* __restrict__ n_active, int n, int V,
-                                                                   const T* __restrict__ gain, T* __restrict__ out, int d, float eps) {
+                                                                   const T* __restrict__ gain, T* __restrict__ out, int d, float eps,
+                                                                   const int32_t* __restrict__ row_off, int B) {
   __shared__ float red[32];
   const int row = blockIdx.x;
   float* xr = x + (size_t)row * d;
@@ -88,7 +99,8 @@ __global__ void __launch_bounds__(NORM_THREADS) fused_norm_kernel(float* __restr
   griddep_launch();
   const T* src = nullptr;
   if (embed) {
-    int b = row / n, v = row % n, t = 0;
+    int b, v, t = 0;
+    locate_row(row, row_off, B, n, b, v);
     if (v < n_active[b]) t = tok[(size_t)b * tok_stride + tok_off + v];
     if (t < 0 || t >= V) t = 0;
     src = embed + (size_t)t * d;
@@ -142,10 +154,13 @@ __global__ void rope_append_kernel(const float* __restrict__ part, int nsplit, s
                                    const int32_t* __restrict__ len, const int32_t* __restrict__ n_active,
                                    const int32_t* __restrict__ depth, const int32_t* __restrict__ page_table,
                                    int max_pages, const float2* __restrict__ rope, int max_pos, int n, int H, int Dh,
-                                   T* __restrict__ q, T* __restrict__ kpool, T* __restrict__ vpool) {
+                                   T* __restrict__ q, T* __restrict__ kpool, T* __restrict__ vpool,
+                                   const int32_t* __restrict__ row_off, int B) {
   // Lengths, live node counts, the tree, the page table and the rotation table are at least two kernels
   // old: the chain of dependent index loads runs before the wait for the QKV GEMM in front.
-  const int row = blockIdx.x, h = blockIdx.y, b = row / n, v = row % n;
+  const int row = blockIdx.x, h = blockIdx.y;
+  int b, v;
+  locate_row(row, row_off, B, n, b, v);          // (the row offsets come from the host, before the step's first kernel)
   const int HD = H * Dh, half = Dh >> 1;
   const bool active = v < n_active[b];
   const int L = len[b];
@@ -286,35 +301,35 @@ int launch_rope_table(cerb_ctx* c, cudaStream_t st) {
 
 // x <- embedding rows (tok != null) | x + partials (nsplit > 0) | x;  out <- RMSNorm(x) * gain (out may be null).
 int launch_fused_norm(cerb_ctx* c, const float* part, int nsplit, size_t split_stride, const int32_t* tok, int tok_stride,
-                      int tok_off, int n, const void* gain, void* out, int rows, cudaStream_t st) {
+                      int tok_off, int n, const void* gain, void* out, int rows, cudaStream_t st, const int32_t* row_off) {
   const cerb_config& g = c->cfg;
   const int d = g.d_model;
   if (d % 4 || d > NORM_THREADS * NORM_MAX_ITER * 4) return CERB_E_SHAPE;
   if (c->bf16)
     launch_pdl(fused_norm_kernel<bf16>, dim3(rows), dim3(NORM_THREADS), 0, st, (float*)c->d_x, part, nsplit, split_stride,
                tok ? (const bf16*)c->embed : (const bf16*)nullptr, tok, tok_stride, tok_off, (const int32_t*)c->d_nactive, n,
-               g.vocab, (const bf16*)gain, (bf16*)out, d, g.rms_eps);
+               g.vocab, (const bf16*)gain, (bf16*)out, d, g.rms_eps, row_off, c->B);
   else
     launch_pdl(fused_norm_kernel<float>, dim3(rows), dim3(NORM_THREADS), 0, st, (float*)c->d_x, part, nsplit, split_stride,
                tok ? (const float*)c->embed : (const float*)nullptr, tok, tok_stride, tok_off, (const int32_t*)c->d_nactive, n,
-               g.vocab, (const float*)gain, (float*)out, d, g.rms_eps);
+               g.vocab, (const float*)gain, (float*)out, d, g.rms_eps, row_off, c->B);
   CERB_LAUNCH_CHECK(c);
   return CERB_OK;
 }
 
 int launch_rope_append(cerb_ctx* c, int layer, const TreeDev& t, const float* part, int nsplit, size_t split_stride,
-                       int B, int n, cudaStream_t st) {
+                       int B, int n, int rows, cudaStream_t st, const int32_t* row_off) {
   const cerb_config& g = c->cfg;
   char* kp = c->k_pool + (size_t)layer * c->pool_layer_bytes;
   char* vp = c->v_pool + (size_t)layer * c->pool_layer_bytes;
   if (c->bf16)
-    launch_pdl(rope_append_kernel<bf16>, dim3(B * n, g.n_heads), dim3(64), 0, st, part, nsplit, split_stride,
+    launch_pdl(rope_append_kernel<bf16>, dim3(rows, g.n_heads), dim3(64), 0, st, part, nsplit, split_stride,
                (const int32_t*)c->d_len, (const int32_t*)c->d_nactive, (const int32_t*)t.depth, c->page_table, g.max_pages,
-               (const float2*)c->d_rope, c->max_pos, n, g.n_heads, g.head_dim, (bf16*)c->d_q, (bf16*)kp, (bf16*)vp);
+               (const float2*)c->d_rope, c->max_pos, n, g.n_heads, g.head_dim, (bf16*)c->d_q, (bf16*)kp, (bf16*)vp, row_off, B);
   else
-    launch_pdl(rope_append_kernel<float>, dim3(B * n, g.n_heads), dim3(64), 0, st, part, nsplit, split_stride,
+    launch_pdl(rope_append_kernel<float>, dim3(rows, g.n_heads), dim3(64), 0, st, part, nsplit, split_stride,
                (const int32_t*)c->d_len, (const int32_t*)c->d_nactive, (const int32_t*)t.depth, c->page_table, g.max_pages,
-               (const float2*)c->d_rope, c->max_pos, n, g.n_heads, g.head_dim, (float*)c->d_q, (float*)kp, (float*)vp);
+               (const float2*)c->d_rope, c->max_pos, n, g.n_heads, g.head_dim, (float*)c->d_q, (float*)kp, (float*)vp, row_off, B);
   CERB_LAUNCH_CHECK(c);
   return CERB_OK;
 }

@@ -270,31 +270,53 @@ def test_tiny_bf16_greedy_decoding_matches_oracle(cb):
         assert float(row.max() - row[g["tokens"][j]]) < 2e-2, (n, j, g, o.tokens)
 
 
-def test_batch_of_two_ragged_prompts(cb):
+@pytest.mark.parametrize("lens", [(150, 21), (33, 70, 5, 128)])
+def test_batch_with_ragged_prompts_and_mixed_modes(cb, lens):
+    """Every sequence of a batch is gated on its own (Algorithm 1 applied per sequence).  In a step where some
+    sequences draft and others decode auto-regressively, the rows of the forward are ragged: n rows for a drafting
+    sequence, one for an auto-regressive one.  Step by step and sequence by sequence: entropy, mode, accepted
+    length and tokens against the oracle's run of that sequence alone; the forward's row count against the modes."""
     ms = synth.tiny_shape("fp32")
-    rig = Rig(cb, ms, max_batch=2, max_tokens=400)
-    p0 = [int(t) for t in synth.make_prompt(ms.vocab, 150, seq=4)]      # more than one prefill chunk
-    p1 = [int(t) for t in synth.make_prompt(ms.vocab, 21, seq=5)]
-    tok = torch.zeros(2, 150, dtype=torch.int32, device="cuda")
-    tok[0, :150] = torch.tensor(p0, dtype=torch.int32)
-    tok[1, :21] = torch.tensor(p1, dtype=torch.int32)
+    B = len(lens)
+    rig = Rig(cb, ms, max_batch=B, max_tokens=400)
+    prompts = [[int(t) for t in synth.make_prompt(ms.vocab, L, seq=4 + i)] for i, L in enumerate(lens)]
+    tok = torch.zeros(B, max(lens), dtype=torch.int32, device="cuda")
+    for b, p in enumerate(prompts):
+        tok[b, :len(p)] = torch.tensor(p, dtype=torch.int32)
     eng = rig.eng
-    eng.prefill(tok, [150, 21])
+    eng.prefill(tok, list(lens))
     tree = synth.best_first_tree(16, rig.topk)
     th = eng.tree(tree)
-    truths = [orc.ar_greedy(rig.cmodel, rig.sh, p, 12) for p in (p0, p1)]
-    T = sorted(truths[0][1] + truths[1][1])[12]
-    outs = [[], []]
-    modes = set()
-    for _ in range(12):
-        eng.step(th, T)
+    n_steps = 12
+    truths = [orc.ar_greedy(rig.cmodel, rig.sh, p, n_steps + 8) for p in prompts]
+    T = orc.calibrate_threshold(sorted(sum((t[1][:n_steps] for t in truths), [])), 0.5)
+    lengths = [3, 1, 4, 2]
+    # the oracle decodes every sequence on its own, with the same planted candidates
+    oruns = [orc.cerberus_greedy(rig.cmodel, rig.sh, rig.cheads, rig.csrc, prompts[b], tree.parent, tree.head, tree.rank,
+                                 rig.topk, T, 5 * n_steps, plant=oracle_planter(tree, truths[b][0] + [0] * 64, lengths))[1]
+             for b in range(B)]
+    outs = [[] for _ in range(B)]
+    modes, mixed = set(), 0
+    for step in range(n_steps):
+        plant = torch.tensor([plant_tokens(tree, truths[b][0] + [0] * 64, len(outs[b]), lengths[step % len(lengths)])
+                              for b in range(B)], dtype=torch.int32, device="cuda")
+        eng.step(th, T, plant)
         torch.cuda.synchronize()
-        for b in range(2):
-            outs[b].extend(int(t) for t in eng.h_tokens[b, :int(eng.h_n_accept[b])])
-            modes.add(int(eng.h_mode[b]))
-    for b in range(2):
-        assert outs[b][:12] == truths[b][0][:12]
-    assert modes == {0, 1}
+        step_modes = [int(eng.h_mode[b]) for b in range(B)]
+        want_rows = sum(1 if m == cb.MODE_AR else tree.n for m in step_modes) if 0 in step_modes else B
+        assert eng.last_forward_rows() == want_rows, (step, step_modes)
+        mixed += len(set(step_modes)) == 2
+        for b in range(B):
+            o = oruns[b][step]
+            na = int(eng.h_n_accept[b])
+            assert abs(float(eng.h_S[b]) - o.S) < 1e-4 and step_modes[b] == o.mode, (step, b)
+            assert na == len(o.path) and [int(t) for t in eng.h_tokens[b, :na]] == o.tokens, (step, b)
+            outs[b].extend(o.tokens)
+            modes.add(step_modes[b])
+    for b in range(B):
+        k = min(len(outs[b]), n_steps + 8)
+        assert outs[b][:k] == truths[b][0][:k]
+    assert modes == {0, 1} and mixed >= 2
     assert eng.device_status() == 0
 
 
