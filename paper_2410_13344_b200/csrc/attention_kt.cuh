@@ -81,7 +81,7 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
   constexpr uint32_t TMEM_COLS = NQ == 64 ? 256u : 512u;           // S^T x 2 buffers, then O^T hi | lo
   constexpr uint32_t O_COL = 2u * NQ;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_u[2][NU], empty_u[NU], s_full[2], s_free[2], p_ready[PB], pv_done[PB], q_ready;
+  __shared__ __align__(8) uint64_t full_u[2][NU], empty_u[NU], s_full[2], s_free[2], p_ready[PB], pv_done[PB], q_ready, drain_bar[2];
   __shared__ __align__(8) uint64_t cl_bar[2];
   __shared__ int page_list[kMaxPagesPerCta];
   __shared__ uint32_t desc_t[CERB_MAX_NODES][4];   // per tree key: which queries of this launch see it, 32 per word
@@ -133,6 +133,8 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
       mbar_init(smem_u32(&pv_done[g]), 1);
     }
     mbar_init(smem_u32(&q_ready), NSW);
+    mbar_init(smem_u32(&drain_bar[0]), 1);
+    mbar_init(smem_u32(&drain_bar[1]), 1);
     mbar_init(smem_u32(&cl_bar[0]), (uint32_t)p.nsplit);
     mbar_init(smem_u32(&cl_bar[1]), (uint32_t)p.nsplit);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -182,20 +184,30 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
     const int box = pw + NPROD * lane;               // lanes 0 .. BOXES-1
     const int pg = box >> 1, hf = box & 1;
     const uint64_t pol = l2_policy(true);            // K/V are read once per step
+    int issued = 0;
     for (int u = 0; u < 2 * T; ++u) {
       if (u == early_units) { griddep_wait(); griddep_launch(); }
       const int slot = u % NU, t = u >> 1;
       const uint32_t fb = smem_u32(&full_u[u & 1][slot]);
+      int stop = 0;
       if (lane == 0) {
         mbar_wait_polite(smem_u32(&empty_u[slot]), ((uint32_t)(u / NU) & 1u) ^ 1u, wc, 101);
-        mbar_expect_tx(fb, KT_UNIT / NPROD);
+        stop = *aborted;
+        if (!stop) mbar_expect_tx(fb, KT_UNIT / NPROD);
       }
-      __syncwarp();
+      if (__shfl_sync(0xffffffffu, stop, 0)) break;            // a wait ran out somewhere in this CTA: issue nothing more
       if (lane < BOXES) {
         const int row = page_list[t * KT_PAGES + pg];          // out-of-range rows are zero-filled by TMA
         const uint32_t dst = ring + (uint32_t)slot * KT_UNIT + (uint32_t)hf * KT_HALF + (uint32_t)pg * (CERB_PAGE * 128);
         tma_load_2d_hint(dst, (u & 1) ? &tmV : &tmK, hf * 64, row, fb, pol);
       }
+      issued = u + 1;
+    }
+    if (lane == 0 && *aborted) {
+      // give-up path: the copies this warp has issued still land in the CTA's shared memory; see them in (the
+      // phase also needs the other producers' shares, hence a limit of its own: 10 ms)
+      for (int u = issued > NU ? issued - NU : 0; u < issued; ++u)
+        mbar_wait_drain(smem_u32(&full_u[u & 1][u % NU]), unit_parity(u), 20000000ll);
     }
     griddep_wait();      // (a lane that has waited already returns at once)
     griddep_launch();
@@ -211,6 +223,7 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
         const int u = 2 * t, slot = u % NU, sb = t & 1;
         wait_unit(u, 103);
         mbar_wait(smem_u32(&s_free[sb]), ((uint32_t)(t >> 1) & 1u) ^ 1u, wc, 104);
+        if (*aborted) break;
         tc_fence_after();
         const uint32_t kb = ring + (uint32_t)slot * KT_UNIT;
         const uint64_t k_desc0 = desc_k_sw128(kb), k_desc1 = desc_k_sw128(kb + KT_HALF);
@@ -221,6 +234,10 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
         for (int kk = 0; kk < 4; ++kk) umma_bf16(d, k_desc1 + (uint64_t)(kk * 2), q_desc1 + (uint64_t)(kk * 2), idesc_s, 1u);
         umma_commit(smem_u32(&empty_u[slot]));       // the K unit is free once these MMAs have retired
         umma_commit(smem_u32(&s_full[sb]));
+      }
+      if (*aborted) {                                // give-up path: see the MMAs already issued retire
+        umma_commit(smem_u32(&drain_bar[0]));
+        mbar_wait_drain(smem_u32(&drain_bar[0]), 0, 20000000ll);
       }
     }
   } else if (warp == W_PV) {
@@ -236,6 +253,7 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
         const int pb = t % PB;
         mbar_wait(smem_u32(&p_ready[pb]), (uint32_t)(t / PB) & 1u, wc, 105);
         wait_unit(u, 106);
+        if (*aborted) break;
         tc_fence_after();
         const uint32_t vb = ring + (uint32_t)slot * KT_UNIT;
         const uint32_t d = tmem + O_COL;
@@ -245,6 +263,10 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
                     idesc_pv, (t == 0 && ks == 0) ? 0u : 1u);
         umma_commit(smem_u32(&empty_u[slot]));
         umma_commit(smem_u32(&pv_done[pb]));
+      }
+      if (*aborted) {                                // give-up path: see the MMAs already issued retire
+        umma_commit(smem_u32(&drain_bar[1]));
+        mbar_wait_drain(smem_u32(&drain_bar[1]), 0, 20000000ll);
       }
     }
   } else {

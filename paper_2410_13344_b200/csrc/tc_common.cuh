@@ -84,12 +84,12 @@ __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const W
 // none of them outlives the CTA's shared and tensor memory.  It keeps a budget of its own (what it waits for
 // was issued and will complete; the limit only guards against the unforeseen) and reports nothing.
 constexpr long long kDrainCycles = 4000000000ll;
-__device__ __forceinline__ void mbar_wait_drain(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ void mbar_wait_drain(uint32_t bar, uint32_t parity, long long cycles = kDrainCycles) {
   const long long t0 = clock64();
   for (;;) {
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return;
-    if (clock64() - t0 > kDrainCycles) return;
+    if (clock64() - t0 > cycles) return;
   }
 }
 // Same bounded wait for a lane whose warp shares an issue port with busy warps: back off between polls.
