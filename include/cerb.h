@@ -152,7 +152,11 @@ int cerb_prefill(cerb_ctx* ctx, const int32_t* tokens_dev, const int32_t* lens_h
 /* Entropy gate (Section 4.2; Algorithm 1: P = Softmax(h_last), S = Entropy(P),
  * S > T selects auto-regressive decoding).  The softmax runs over the d_model
  * components of each sequence's last hidden state; S is in bits.
- * S_dev [B] float, mode_dev [B] int32 (CERB_MODE_*). */
+ * S_dev [B] float, mode_dev [B] int32 (CERB_MODE_*).
+ * The call only enqueues work and never reads S back, so it cannot return
+ * CERB_E_NONFINITE: a non-finite S (from a non-finite hidden state) is left in
+ * S_dev for the caller to see (a NaN compares false with T and so selects
+ * CERB_MODE_PAR); cerb_step, which reads S on the host anyway, reports it. */
 int cerb_gate(cerb_ctx* ctx, float T, float* S_dev, int32_t* mode_dev, void* stream);
 
 /* Draft (Section 4.1; Algorithm 1: Candidates = (LH[h_last], CH_0[h_last], ...)):

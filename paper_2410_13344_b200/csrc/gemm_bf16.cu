@@ -35,6 +35,8 @@
 // mbarriers; every wait is bounded and reports CERB_E_TIMEOUT through a status word.
 #include <stdlib.h>
 
+#include <mutex>
+
 #include "tc_common.cuh"
 
 namespace cerb {
@@ -394,10 +396,37 @@ EncodeTiledFn g_encode = nullptr;
 // for right afterwards: DRAM bursts twice as long.  Measured on the 7B decoding step: 4.23 -> 4.02 ms per
 // 64-node forward, 3.49 -> 3.31 ms per one-node forward (128-byte promotion and none are equal).
 
+// The last descriptors made, by their arguments.  A descriptor depends on nothing else, and the stand-alone entry
+// points (which own no context to keep maps in) are typically called again and again on the same buffers: they
+// find their maps here instead of encoding two to six of them per call.
+struct MapKey {
+  const void* base;
+  uint64_t inner, outer, row_bytes;
+  uint32_t box_inner, box_outer;
+  bool operator==(const MapKey& o) const {
+    return base == o.base && inner == o.inner && outer == o.outer && row_bytes == o.row_bytes && box_inner == o.box_inner &&
+           box_outer == o.box_outer;
+  }
+};
+constexpr int kMapCache = 32;
+std::mutex g_map_mutex;
+MapKey g_map_key[kMapCache];
+CUtensorMap g_map_val[kMapCache];
+int g_map_used = 0, g_map_next = 0;
+
 int encode_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer, uint64_t row_bytes, uint32_t box_inner,
               uint32_t box_outer) {
   if (init_driver_api() != CERB_OK) return CERB_E_CUDA;
   if (((uintptr_t)base & 15) || (row_bytes & 15)) return CERB_E_SHAPE;
+  const MapKey key{base, inner, outer, row_bytes, box_inner, box_outer};
+  {
+    std::lock_guard<std::mutex> lock(g_map_mutex);
+    for (int i = 0; i < g_map_used; ++i)
+      if (g_map_key[i] == key) {
+        *out = g_map_val[i];
+        return CERB_OK;
+      }
+  }
   cuuint64_t dims[2] = {inner, outer};
   cuuint64_t strides[1] = {row_bytes};
   cuuint32_t box[2] = {box_inner, box_outer};
@@ -405,7 +434,13 @@ int encode_2d(CUtensorMap* out, const void* base, uint64_t inner, uint64_t outer
   CUresult r = g_encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? CERB_OK : CERB_E_CUDA;
+  if (r != CUDA_SUCCESS) return CERB_E_CUDA;
+  std::lock_guard<std::mutex> lock(g_map_mutex);
+  g_map_key[g_map_next] = key;
+  g_map_val[g_map_next] = *out;
+  g_map_next = (g_map_next + 1) % kMapCache;
+  if (g_map_used < kMapCache) ++g_map_used;
+  return CERB_OK;
 }
 
 }  // namespace
