@@ -34,6 +34,7 @@
 // epilogue overlaps the next segment's MMAs.  Stages and accumulators are handed over with
 // mbarriers; every wait is bounded and reports CERB_E_TIMEOUT through a status word.
 #include <stdlib.h>
+#include <string.h>
 
 #include <mutex>
 
@@ -354,14 +355,254 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
   }
 }
 
+
+// ---------------------------------------------------------------------------------------------------------------
+// More than 128 activation rows: two CTAs of a cluster work as one (tcgen05 cta_group::2).
+//
+// With 256 activation rows per pass a single CTA's stage is half activations (32 KB of weights + 32 KB of
+// activations, three stages), so too few weight bytes are in flight per SM to cover HBM's latency, and the two
+// 256-column accumulators fill tensor memory.  A pair of CTAs shares the activation tile instead: one MMA is
+// 256 weight rows tall, 128 from each CTA's shared memory, and its 256 activation rows come half from each CTA.
+// A unit of the work list is then 512 weight rows x 64 k (two such MMA rows, hf = 0 / 1); per CTA a stage holds
+// 2 x 16 KB of weights + 16 KB of activations (four stages: 128 KB of weights in flight instead of 96), and each CTA's
+// tensor memory holds its 128 rows of both accumulators.  Every CTA fetches its own tiles (no multicast); the
+// byte counts of both CTAs' copies go to the first CTA's "landed" barrier, whose two MMA-issuing threads drive the
+// pair; their commits arrive on the "free" and "accumulator complete" barriers of both CTAs at once.  The work
+// list, the shares, the segments and the partial slots are those of the kernel above, with pairs in the place of
+// CTAs.
+// ---------------------------------------------------------------------------------------------------------------
+constexpr int PAIR_STAGES = 4;
+constexpr int PAIR_TILE = 4 * BM;                       // weight rows of a pair's unit
+constexpr uint32_t PAIR_STAGE_BYTES = 3 * A_STAGE_BYTES;  // per CTA: weights hf 0, weights hf 1, its half of the activations
+constexpr int PAIR_ACT = 2 * BM;                        // activation rows per pass (the MMA's N)
+
+__global__ void __launch_bounds__(224, 1) gemm_bf16_pair_kernel(const __grid_constant__ CUtensorMap tmW,
+                                                                const __grid_constant__ CUtensorMap tmX, const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[PAIR_STAGES];     // used in the pair's first CTA only
+  __shared__ __align__(8) uint64_t empty_bar[PAIR_STAGES];
+  __shared__ __align__(8) uint64_t acc_full, acc_empty;       // acc_empty: first CTA only, 4 epilogue warps of each CTA arrive
+  __shared__ __align__(8) uint64_t drain_bar[2];
+  __shared__ __align__(8) uint64_t meet_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ int aborted_s, meet_flag_s;
+  volatile int* aborted = &aborted_s;
+  const WaitCtx wc{p.wait_cycles, aborted, p.status, p.N + 100000 * (p.M > 999 ? 999 : p.M)};
+
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool first = rank == 0;
+  const int pair = (int)blockIdx.x >> 1;
+  const int share = pair / p.lock;
+  const int my_chunk = pair % p.lock;
+  const int u0 = share * p.per;
+  const int u1 = (u0 + p.per < p.total) ? u0 + p.per : p.total;
+
+  if (threadIdx.x == 0) {
+    aborted_s = 0;
+    meet_flag_s = 0;
+    for (int s = 0; s < PAIR_STAGES; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), 2);
+    }
+    mbar_init(smem_u32(&acc_full), 2);
+    mbar_init(smem_u32(&acc_empty), 8);
+    mbar_init(smem_u32(&drain_bar[0]), 1);
+    mbar_init(smem_u32(&drain_bar[1]), 1);
+    mbar_init(smem_u32(&meet_bar), 2);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    // each CTA allocates all 512 columns of its own tensor memory (so both get the same base)
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  cluster_start_arrive();       // the other CTA's barriers exist before anything is signalled across
+  cluster_start_wait();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const int n_units = u1 - u0;
+      const uint64_t pol_w = l2_policy(true), pol_x = l2_policy(false);
+      int w_job = u0 / p.num_kb, w_kb = u0 - w_job * p.num_kb;
+      int x_job = w_job, x_kb = w_kb;
+      auto load_w = [&](int i) {
+        const int tile = w_job % p.tiles;
+        const int s = i % PAIR_STAGES;
+        if (first) mbar_expect_tx(smem_u32(&full_bar[s]), 2 * PAIR_STAGE_BYTES);      // both CTAs' copies of this stage
+        const uint32_t fb = mapa_u32(smem_u32(&full_bar[s]), 0);
+        const uint32_t dst = smem_base + (uint32_t)s * PAIR_STAGE_BYTES;
+        const int row = tile * PAIR_TILE + (int)rank * BM;
+        tma_load_2d_pair(dst, &tmW, w_kb * BK, row, fb, pol_w);
+        tma_load_2d_pair(dst + A_STAGE_BYTES, &tmW, w_kb * BK, row + 2 * BM, fb, pol_w);
+        if (++w_kb == p.num_kb) { w_kb = 0; ++w_job; }
+      };
+      auto load_x = [&](int i) {
+        const int mchunk = p.lock > 1 ? my_chunk : x_job / p.tiles;
+        const int s = i % PAIR_STAGES;
+        const uint32_t fb = mapa_u32(smem_u32(&full_bar[s]), 0);
+        tma_load_2d_pair(smem_base + (uint32_t)s * PAIR_STAGE_BYTES + 2 * A_STAGE_BYTES, &tmX, x_kb * BK,
+                         mchunk * PAIR_ACT + (int)rank * BM, fb, pol_x);
+        if (++x_kb == p.num_kb) { x_kb = 0; ++x_job; }
+      };
+      const int pre = n_units < PAIR_STAGES ? n_units : PAIR_STAGES;
+      for (int i = 0; i < pre; ++i) load_w(i);
+      asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)&tmX) : "memory");
+      griddep_wait();
+      griddep_launch();
+      if (p.clk) atomicMin(p.clk, globaltimer_ns());
+      for (int i = 0; i < pre; ++i) load_x(i);
+      int issued = pre;
+      for (int i = pre; i < n_units; ++i) {
+        const int s = i % PAIR_STAGES;
+        const uint32_t ph = (uint32_t)(i / PAIR_STAGES) & 1u;
+        mbar_wait_cluster(smem_u32(&empty_bar[s]), ph ^ 1u, wc, 211);
+        if (*aborted) break;
+        load_w(i);
+        load_x(i);
+        issued = i + 1;
+      }
+      if (*aborted) {
+        // give-up path: this CTA's copies land in its own shared memory but are counted on the first CTA's
+        // barriers, and the two CTAs may have stopped at different units, so neither can see exactly its own
+        // copies in.  The first CTA waits for the stages it knows of (short budget); then both let the time of
+        // many memory round trips pass before they go on to the rendezvous and leave.
+        if (first)
+          for (int i = issued > PAIR_STAGES ? issued - PAIR_STAGES : 0; i < issued; ++i)
+            mbar_wait_drain(smem_u32(&full_bar[i % PAIR_STAGES]), (uint32_t)(i / PAIR_STAGES) & 1u, 2000000ll);
+        const long long t_land = clock64();
+        while (clock64() - t_land < 400000ll) __nanosleep(1000);
+      }
+    }
+  } else if (warp == 1 || warp == 6) {
+    // MMA issuers of the pair: the first CTA's warps 1 (hf 0) and 6 (hf 1)
+    const int hf = warp == 6 ? 1 : 0;
+    if (first && lane == 0) {
+      const uint32_t idesc = idesc_bf16(2 * BM, PAIR_ACT, false, false);
+      int u = u0;
+      Segment sg;
+      int i = 0, g = 0;
+      while (next_segment(u, u1, p.num_kb, sg)) {
+        mbar_wait_cluster(smem_u32(&acc_empty), ((uint32_t)g & 1u) ^ 1u, wc, 212);
+        if (*aborted) break;
+        tc_fence_after();
+        const uint32_t d = tmem_base + (uint32_t)(hf * PAIR_ACT);
+        for (int k = 0; k < sg.nkb; ++k, ++i) {
+          const int s = i % PAIR_STAGES;
+          const uint32_t ph = (uint32_t)(i / PAIR_STAGES) & 1u;
+          mbar_wait_cluster(smem_u32(&full_bar[s]), ph, wc, 213);
+          if (*aborted) break;
+          tc_fence_after();
+          const uint32_t src = smem_base + (uint32_t)s * PAIR_STAGE_BYTES;
+          const uint64_t adesc = desc_k_sw128(src + (uint32_t)hf * A_STAGE_BYTES);
+          const uint64_t bdesc = desc_k_sw128(src + 2 * A_STAGE_BYTES);
+#pragma unroll
+          for (int kk = 0; kk < BK / 16; ++kk)
+            umma_bf16_pair(d, adesc + (uint64_t)(kk * 2), bdesc + (uint64_t)(kk * 2), idesc, (k > 0 || kk > 0) ? 1u : 0u);
+          umma_commit_pair(smem_u32(&empty_bar[s]));       // the stage is free in both CTAs once these MMAs have read it
+        }
+        if (*aborted) break;
+        umma_commit_pair(smem_u32(&acc_full));
+        ++g;
+      }
+      if (*aborted) {
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(&drain_bar[hf])) : "memory");
+        mbar_wait_drain(smem_u32(&drain_bar[hf]), 0, 40000000ll);
+      }
+    }
+  } else {
+    const int quarter = warp & 3;                    // TMEM lanes 32*quarter .. +31 belong to this warp
+    griddep_wait();                                  // the kernel before this one may still be reading the partial buffer
+    const uint32_t ae = mapa_u32(smem_u32(&acc_empty), 0);
+    int u = u0;
+    Segment sg;
+    int g = 0;
+    while (next_segment(u, u1, p.num_kb, sg)) {
+      const int tile = sg.job % p.tiles, mchunk = p.lock > 1 ? my_chunk : sg.job / p.tiles;
+      mbar_wait_cluster(smem_u32(&acc_full), (uint32_t)g & 1u, wc, 214);
+      if (*aborted) break;
+      tc_fence_after();
+      const int job_u0 = sg.job * p.num_kb;
+      const int first_share = job_u0 / p.per;
+      const int last_share = (job_u0 + p.num_kb - 1) / p.per;
+      const int slot = share - first_share;
+      const int m_base = mchunk * PAIR_ACT;
+      const int m_cnt = min(PAIR_ACT, p.M - m_base);
+      const size_t ldo = (size_t)p.N;
+      for (int hf = 0; hf < 2; ++hf) {
+        const int n_out = tile * PAIR_TILE + hf * 2 * BM + (int)rank * BM + quarter * 32 + lane;
+        const bool n_ok = n_out < p.N;
+        float* o = p.out + ((size_t)slot * p.M + m_base) * ldo + (n_ok ? n_out : 0);
+        const uint32_t taddr = tmem_base + (uint32_t)(hf * PAIR_ACT) + ((uint32_t)(quarter * 32) << 16);
+        for (int c0 = 0; c0 < m_cnt; c0 += 16) {
+          uint32_t r[16];
+          tmem_ld16(taddr + (uint32_t)c0, r);
+          if (n_ok) {
+            if (c0 + 16 <= m_cnt) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) { *o = __uint_as_float(r[j]); o += ldo; }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j)
+                if (c0 + j < m_cnt) { *o = __uint_as_float(r[j]); o += ldo; }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(ae);          // (the first CTA's own warps arrive the same way)
+      if (share == last_share) {
+        for (int hf = 0; hf < 2; ++hf) {
+          const int n_out = tile * PAIR_TILE + hf * 2 * BM + (int)rank * BM + quarter * 32 + lane;
+          if (n_out >= p.N) continue;
+          for (int z = last_share - first_share + 1; z < p.nslots; ++z) {
+            float* zo = p.out + ((size_t)z * p.M + m_base) * ldo + n_out;
+            for (int m = 0; m < m_cnt; ++m) { *zo = 0.f; zo += ldo; }
+          }
+        }
+      }
+      ++g;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (p.clk && threadIdx.x == 0) atomicMax(p.clk + kGemmClockSlots, globaltimer_ns());
+  // Neither CTA leaves (nor frees its tensor memory) before the other is done: copies, commits and arrivals cross
+  // between them until then.  The rendezvous keeps a budget of its own, far above that of the other waits, so that a
+  // CTA which has given up still finds its partner.
+  if (warp == 2) {
+    const long long meet_budget = p.wait_cycles * 4 > 40000000ll ? p.wait_cycles * 4 : 40000000ll;
+    const WaitCtx wm{meet_budget, &meet_flag_s, p.status, wc.tag};
+    cluster_meet(&meet_bar, 2, lane, wm, 215);
+  }
+  __syncthreads();
+  if (warp == 1)
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+}
+
 struct GemmPlan {
   int tiles, mchunks, num_kb, per, ctas, nslots, lock;
+  bool pair;         // CTA pairs (gemm_bf16_pair_kernel): `ctas` then counts pairs, a unit is 512 weight rows
   long long total;   // checked to fit 31 bits before launch
 };
 
+// More than 128 rows go to the CTA pairs.  CERB_GEMM_PAIR=0 keeps them on single CTAs (tests, comparison).
+bool pair_enabled() {
+  static const int v = getenv("CERB_GEMM_PAIR") ? atoi(getenv("CERB_GEMM_PAIR")) : 1;
+  return v != 0;
+}
+
 GemmPlan make_plan(int sm_count, int M, int N, int K) {
   GemmPlan g;
-  const int rows_per_tile = 2 * BM;            // a unit is two weight tiles of 128 rows
+  g.pair = M > BM && pair_enabled();
+  if (g.pair) sm_count /= 2;                   // workers are pairs
+  const int rows_per_tile = g.pair ? PAIR_TILE : 2 * BM;     // a unit is two weight tiles of 128 rows (of 256 for a pair)
   g.tiles = (N + rows_per_tile - 1) / rows_per_tile;
   g.mchunks = (M + kGemmRowsPerPass - 1) / kGemmRowsPerPass;
   g.num_kb = (K + BK - 1) / BK;
@@ -496,6 +737,29 @@ int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, fl
   // the caller used (148) and simply run that many CTAs; the hardware queues what does not fit.
   GemmPlan g = make_plan(148, M, N, K);
   if (g.nslots != nsplit) return CERB_E_ARG;
+  if (g.pair) {
+    if (epi && epi->kind != 0) return CERB_E_SHAPE;
+    if (g.total >= (1ll << 30)) return CERB_E_SHAPE;
+    GemmParams q;
+    memset(&q, 0, sizeof(q));
+    q.out = out; q.status = status;
+    q.M = M; q.N = N; q.K = K;
+    q.n_mma = PAIR_ACT; q.num_kb = g.num_kb; q.tiles = g.tiles; q.per = g.per; q.total = (int)g.total; q.lock = g.lock;
+    q.nslots = g.nslots; q.stages = PAIR_STAGES; q.wait_cycles = wait_cycles(); q.acc_cols = 2u * PAIR_ACT; q.acc_bufs = 1;
+    q.tile_rows = PAIR_TILE; q.half_off = 2 * BM;
+    q.clk = clock_slot;
+    const size_t smem = (size_t)PAIR_STAGES * PAIR_STAGE_BYTES + 1024;
+    static bool pair_configured = false;
+    if (!pair_configured) {
+      CERB_CUDA_OK(cudaFuncSetAttribute(gemm_bf16_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      pair_configured = true;
+    }
+    // each CTA loads 128 of the pass's 256 activation rows: the map with 128-row boxes
+    if (launch_pdl_cluster(gemm_bf16_pair_kernel, dim3(2 * g.ctas), dim3(224), smem, st, 2u, *tmW, tmX->m[row_bucket(BM)], q) != cudaSuccess)
+      return CERB_E_CUDA;
+    CERB_LAUNCH_CHECK(c);
+    return CERB_OK;
+  }
   GemmParams p;
   int bucket = row_bucket(M < kGemmRowsPerPass ? M : kGemmRowsPerPass);
   p.out = out;

@@ -152,6 +152,33 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// The same for a pair of CTAs working as one (cta_group::2; issued by one thread of the pair's first CTA): the MMA
+// is 256 rows tall, 128 from each CTA's shared memory at the same offsets; the B operand's rows are split likewise;
+// each CTA's tensor memory receives its 128 rows of D.  The eight mask words (rows not to write) are zero.
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  const uint32_t z = 0u;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc), "r"(z)
+      : "memory");
+}
+// Arrives, once the pair's MMAs issued so far have retired, on the mbarrier at this shared-memory offset in both
+// CTAs of the pair (CTA mask 0b11).
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar), "h"(mask)
+               : "memory");
+}
+// TMA tile load of a CTA of such a pair into its own shared memory; the bytes are counted on `bar`, a
+// shared::cluster address that may lie in the other CTA of the pair.  No multicast: each CTA fetches its own tiles.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"((uint64_t)map), "r"(x), "r"(y), "r"(bar), "l"(pol)
+      : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void proxy_fence() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -224,6 +251,28 @@ __device__ __forceinline__ void cluster_meet(uint64_t* bar, int members, int idx
   for (;;) {
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait_cluster(local, 0)) return;
+    if (clock64() - t0 > budget) break;
+  }
+  wait_ran_out(w, site);
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Arrive on an mbarrier anywhere in the cluster (shared::cluster address), release at cluster scope.
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Bounded wait on an own mbarrier whose arrivals may come from another CTA of the cluster (acquire at cluster scope).
+__device__ __forceinline__ void mbar_wait_cluster(uint32_t bar, uint32_t parity, const WaitCtx& w, int site = 0) {
+  for (int i = 0; i < 8; ++i)
+    if (mbar_try_wait_cluster(bar, parity)) return;
+  const long long t0 = clock64();
+  const long long budget = *w.aborted ? kAbortedWaitCycles : w.budget;
+  for (;;) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait_cluster(bar, parity)) return;
     if (clock64() - t0 > budget) break;
   }
   wait_ran_out(w, site);
