@@ -82,7 +82,7 @@ inline cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 
 
 constexpr int kPathMax = CERB_MAX_DEPTH + 1;
 constexpr int kPrefillChunkMax = 128;   // prompt tokens per prefill chunk (a chain-shaped tree), whatever max_nodes is
-constexpr int kGemmRowsPerPass = 256;   // activation rows one tcgen05 pass covers (the MMA's N extent)
+constexpr int kGemmRowsPerPass = 256;   // activation rows one tcgen05 pass covers at most (the MMA's N extent; CTA pairs)
 constexpr int kGemmMaxSplit = 16;
 
 // Device-side copy of a tree, living in the workspace.

@@ -4,18 +4,18 @@
 //
 // A decoding step has few activation rows (tree nodes x batch) and large weight matrices, so the
 // kernel is organised around streaming W exactly once at HBM speed ("swap-AB"): a 128-row tile of
-// W is the MMA's A operand (M = 128), up to 256 activation rows are the B operand (N = rows), and
+// W is the MMA's A operand (M = 128), the activation rows are the B operand (N = rows), and
 // D[128][rows] accumulates in tensor memory and is written out transposed.
 //
-// A CTA takes 256 weight rows at a time (two MMA tiles that share one activation stage), which
-// halves the activation re-reads through L2; weight tiles carry an evict-first L2 hint, activation
-// tiles evict-last.  With 256 activation rows per pass the two accumulators fill tensor memory, so
-// the accumulator is single-buffered there; with fewer rows it is double-buffered.
+// Up to 128 activation rows (gemm_bf16_kernel): a CTA takes 256 weight rows at a time (two MMA tiles
+// that share one activation stage), which halves the activation re-reads through L2; weight tiles
+// carry an evict-first L2 hint, activation tiles evict-last; the accumulator is double-buffered.
 //
-// More than 256 rows (batched trees, prefill chunks of a batch) are cut into row chunks of 256.  The
-// chunks are not queued one after the other: the CTAs are grouped, one CTA per row chunk in a group,
-// and the CTAs of a group walk the same weight tiles side by side, so that HBM delivers each weight
-// byte once and the other chunks find it in L2.
+// More than 128 rows (batched trees, prefill chunks of a batch; gemm_bf16_pair_kernel further down):
+// two CTAs of a cluster work as one, 256 rows per pass.  More than 256 rows are cut into row chunks of
+// 256 that are not queued one after the other: the pairs are grouped, one pair per row chunk in a
+// group, and the pairs of a group walk the same weight tiles side by side, so that HBM delivers each
+// weight byte once and the other chunks find it in L2.
 //
 // The kernel is launched programmatically dependent on its predecessor: weights do not depend on
 // the previous kernel, so the producer fills the whole stage ring with weight tiles before it
@@ -59,21 +59,21 @@ struct GemmParams {
   float* out;
   int32_t* status;
   int M, N, K;
-  int n_mma;          // activation rows per pass (16..256, power of two)
+  int n_mma;          // activation rows per pass (16..128, power of two; 256 for CTA pairs)
   int num_kb;         // ceil(K / 64)
   int tiles;          // ceil(N / 128)
   int per;            // work units per CTA
-  int total;          // work units in the list: mchunks * tiles * num_kb (tiles * num_kb with lock > 1)
-  int lock;           // > 1: this many CTAs (one per row chunk) walk the same share of the (tile, k block) list side by
-                      // side, so a weight tile is fetched from HBM once and found in L2 by the others; 1: row chunks are
-                      // part of the list
+  int total;          // work units in the list: tiles * num_kb (pairs with lock == 1: row chunks * tiles * num_kb)
+  int lock;           // CTA pairs only.  > 1: this many pairs (one per chunk of 256 rows) walk the same share of the (tile,
+                      // k block) list side by side, so a weight tile is fetched from HBM once and found in L2 by the
+                      // others; 1: row chunks are part of the list
   int nslots;         // partial slots per output element
   int stages;
   long long wait_cycles;   // budget of every bounded wait, SM clock cycles
   uint32_t idesc;
   uint32_t acc_cols;  // TMEM columns of one accumulator buffer
-  int acc_bufs;       // accumulator buffers in TMEM: 2 (a segment's epilogue overlaps the next segment's MMAs), or 1 when
-                      // one accumulator already fills all 512 columns (two weight tiles x 256 activation rows)
+  int acc_bufs;       // accumulator buffers in TMEM: 2 (a segment's epilogue overlaps the next segment's MMAs); 1 for CTA
+                      // pairs, whose two 256-column accumulators fill all 512 columns
   int tile_rows;      // weight rows between the starts of consecutive tiles
   int half_off;       // weight-row offset of a wide unit's second tile from its first
   int epi;            // fused epilogue (GemmEpilogue::kind)
@@ -118,8 +118,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
   const uint32_t a_bytes = 2 * A_STAGE_BYTES;        // two weight tiles of 128 rows per unit
   const uint32_t stage_bytes = a_bytes + b_bytes;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int share = (int)blockIdx.x / p.lock;          // which contiguous share of the unit list
-  const int my_chunk = (int)blockIdx.x % p.lock;       // with lock > 1: the row chunk this CTA computes
+  const int share = (int)blockIdx.x;                   // which contiguous share of the unit list
   const int u0 = share * p.per;
   const int u1 = (u0 + p.per < p.total) ? u0 + p.per : p.total;
 
@@ -138,7 +137,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
-                 "r"((uint32_t)p.acc_bufs * p.acc_cols)
+                 "r"(2u * p.acc_cols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -151,9 +150,9 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
     if (lane == 0) {
       const int n_units = u1 - u0;
       const uint64_t pol_w = l2_policy(true), pol_x = l2_policy(false);
-      // (tile, row chunk, k block) of the unit being issued, advanced incrementally
+      // (tile, k block) of the unit being issued, advanced incrementally
       int w_job = u0 / p.num_kb, w_kb = u0 - w_job * p.num_kb;
-      int x_job = w_job, x_kb = w_kb;
+      int x_kb = w_kb;
       auto load_w = [&](int i) {
         const int tile = w_job % p.tiles;
         const int s = i % p.stages;
@@ -165,12 +164,11 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
         if (++w_kb == p.num_kb) { w_kb = 0; ++w_job; }
       };
       auto load_x = [&](int i) {
-        const int mchunk = p.lock > 1 ? my_chunk : x_job / p.tiles;
         const int s = i % p.stages;
         const uint32_t fb = smem_u32(&full_bar[s]);
         const uint32_t x_dst = smem_base + (uint32_t)s * stage_bytes + a_bytes;
-        tma_load_2d_hint(x_dst, &tmX, x_kb * BK, mchunk * kGemmRowsPerPass, fb, pol_x);
-        if (++x_kb == p.num_kb) { x_kb = 0; ++x_job; }
+        tma_load_2d_hint(x_dst, &tmX, x_kb * BK, 0, fb, pol_x);
+        if (++x_kb == p.num_kb) x_kb = 0;
       };
       // Weights do not depend on the kernel before this one: fill the whole ring with weight tiles
       // while that kernel is still finishing, then wait for it and fetch the activations.
@@ -212,8 +210,8 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
       Segment sg;
       int i = 0, g = 0;
       while (next_segment(u, u1, p.num_kb, sg)) {
-        const int buf = p.acc_bufs == 2 ? (g & 1) : 0;
-        const uint32_t use = (uint32_t)(p.acc_bufs == 2 ? g >> 1 : g);      // how often this buffer was used before
+        const int buf = g & 1;
+        const uint32_t use = (uint32_t)(g >> 1);      // how often this buffer was used before
         mbar_wait(smem_u32(&acc_empty[buf]), (use & 1u) ^ 1u, wc, 202);
         if (*aborted) break;
         tc_fence_after();
@@ -250,9 +248,9 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
     Segment sg;
     int g = 0;
     while (next_segment(u, u1, p.num_kb, sg)) {
-      const int buf = p.acc_bufs == 2 ? (g & 1) : 0;
-      const int tile = sg.job % p.tiles, mchunk = p.lock > 1 ? my_chunk : sg.job / p.tiles;
-      mbar_wait(smem_u32(&acc_full[buf]), (uint32_t)(p.acc_bufs == 2 ? g >> 1 : g) & 1u, wc, 204);
+      const int buf = g & 1;
+      const int tile = sg.job;
+      mbar_wait(smem_u32(&acc_full[buf]), (uint32_t)(g >> 1) & 1u, wc, 204);
       if (*aborted) break;                         // the launch's output is undefined from here on
       tc_fence_after();
       // slot = how many CTAs before this one also work on this job
@@ -260,8 +258,8 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
       const int first_cta = job_u0 / p.per;
       const int last_cta = (job_u0 + p.num_kb - 1) / p.per;
       const int slot = share - first_cta;
-      const int m_base = mchunk * kGemmRowsPerPass;
-      const int m_cnt = min(p.n_mma, p.M - m_base);
+      const int m_base = 0;                            // (all rows in one pass: this kernel takes up to 128)
+      const int m_cnt = p.M;
       const size_t ldo = (size_t)p.N;
       const int cnt = last_cta - first_cta + 1;        // CTAs that share this job = slots it uses
       if (p.epi == 1 && cnt == 1) {
@@ -351,7 +349,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
   __syncthreads();
   if (p.clk && threadIdx.x == 0) atomicMax(p.clk + kGemmClockSlots, globaltimer_ns());
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.acc_bufs * p.acc_cols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2u * p.acc_cols) : "memory");
   }
 }
 
@@ -592,22 +590,17 @@ struct GemmPlan {
   long long total;   // checked to fit 31 bits before launch
 };
 
-// More than 128 rows go to the CTA pairs.  CERB_GEMM_PAIR=0 keeps them on single CTAs (tests, comparison).
-bool pair_enabled() {
-  static const int v = getenv("CERB_GEMM_PAIR") ? atoi(getenv("CERB_GEMM_PAIR")) : 1;
-  return v != 0;
-}
-
+// Up to 128 rows: single CTAs, one pass over all rows.  More: CTA pairs, 256 rows per pass.
 GemmPlan make_plan(int sm_count, int M, int N, int K) {
   GemmPlan g;
-  g.pair = M > BM && pair_enabled();
+  g.pair = M > BM;
   if (g.pair) sm_count /= 2;                   // workers are pairs
   const int rows_per_tile = g.pair ? PAIR_TILE : 2 * BM;     // a unit is two weight tiles of 128 rows (of 256 for a pair)
   g.tiles = (N + rows_per_tile - 1) / rows_per_tile;
-  g.mchunks = (M + kGemmRowsPerPass - 1) / kGemmRowsPerPass;
+  g.mchunks = g.pair ? (M + PAIR_ACT - 1) / PAIR_ACT : 1;
   g.num_kb = (K + BK - 1) / BK;
-  // More than one row chunk: the (tile, k block) list of ONE chunk is cut into sm_count / mchunks shares and every
-  // share is walked by mchunks CTAs side by side, one per row chunk.  They ask for the same weight tiles at the
+  // More than one row chunk: the (tile, k block) list of ONE chunk is cut into (pairs / chunks) shares and every
+  // share is walked by `chunks` pairs side by side, one per row chunk.  They ask for the same weight tiles at the
   // same time, so HBM delivers every weight byte once instead of once per row chunk (measured at 2048 rows x
   // 22016 x 4096 before this: 1.58 GB of DRAM reads for 180 MB of weights, the kernel at 70 % of DRAM throughput).
   g.lock = (g.mchunks > 1 && g.mchunks * 2 <= sm_count) ? g.mchunks : 1;
@@ -761,7 +754,7 @@ int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, fl
     return CERB_OK;
   }
   GemmParams p;
-  int bucket = row_bucket(M < kGemmRowsPerPass ? M : kGemmRowsPerPass);
+  int bucket = row_bucket(M);                   // (M <= 128 here)
   p.out = out;
   p.status = status;
   p.M = M; p.N = N; p.K = K;
@@ -771,7 +764,7 @@ int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, fl
   p.per = g.per;
   if (g.total >= (1ll << 30)) return CERB_E_SHAPE;
   p.total = (int)g.total;
-  p.lock = g.lock;
+  p.lock = 1;
   p.nslots = g.nslots;
   p.tile_rows = 2 * BM;
   p.wait_cycles = wait_cycles();
@@ -789,7 +782,7 @@ int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, fl
   if (p.stages > MAX_STAGES) p.stages = MAX_STAGES;
   if (p.stages < 2) return CERB_E_SHAPE;
   p.acc_cols = 2u * (uint32_t)p.n_mma;            // two weight tiles side by side (at least 32 columns)
-  p.acc_bufs = 2u * p.acc_cols <= 512u ? 2 : 1;
+  p.acc_bufs = 2;                                 // 2 x (2 x 128) columns at most
   // instruction descriptor: D fp32, A and B bf16, both K-major, N = n_mma, M = 128
   p.idesc = idesc_bf16(BM, (uint32_t)p.n_mma, false, false);
   size_t smem = (size_t)p.stages * stage_bytes + 1024;

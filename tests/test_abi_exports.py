@@ -56,14 +56,18 @@ def test_threshold_from_samples_splits_the_requested_fraction():
 
 
 def _slots_by_the_stated_schedule(M, N, K, sms=148):
-    """Partial slots per output element of the bf16 GEMM, from its schedule as documented: units are (256-row weight
-    tile, 64-wide k block) pairs; rows beyond 256 form row chunks; with 2..74 chunks the unit list of ONE chunk is cut
-    into floor(148 / chunks) contiguous shares (one CTA per chunk walks each share), otherwise the list over all
-    chunks is cut into 148 shares; a share has at least min(k blocks, 4) units; a tile's slots = shares it touches."""
-    tiles, kb, chunks = -(-N // 256), -(-K // 64), -(-M // 256)
-    grouped = 1 < chunks <= sms // 2
+    """Partial slots per output element of the bf16 GEMM, from its schedule as documented.  Up to 128 rows: units are
+    (256-row weight tile, 64-wide k block) pairs, cut into 148 contiguous shares, one per CTA.  More rows: the workers
+    are the 74 CTA pairs, a tile has 512 weight rows, and the rows form chunks of 256; with 2..37 chunks the unit list
+    of ONE chunk is cut into floor(74 / chunks) shares (one pair per chunk walks each share), otherwise the list over
+    all chunks is cut into 74 shares.  A share has at least min(k blocks, 4) units; a tile's slots = shares it touches."""
+    pairs = M > 128
+    workers = sms // 2 if pairs else sms
+    tiles, kb = -(-N // (512 if pairs else 256)), -(-K // 64)
+    chunks = -(-M // 256) if pairs else 1
+    grouped = 1 < chunks <= workers // 2
     jobs = tiles if grouped else tiles * chunks
-    shares = sms // chunks if grouped else sms
+    shares = workers // chunks if grouped else workers
     per = max(-(-jobs * kb // shares), min(kb, 4))
     return max((j * kb + kb - 1) // per - (j * kb) // per + 1 for j in range(jobs))
 
@@ -80,7 +84,7 @@ def test_gemm_scratch_size_follows_the_documented_schedule():
         nb = C.c_size_t(0)
         assert L.cerb_gemm_scratch_bytes(M, N, K, C.byref(nb)) == binding.OK
         assert nb.value == 256 + _slots_by_the_stated_schedule(M, N, K) * M * N * 4, (M, N, K)
-    # weights leave HBM once at 2048 rows: 8 row chunks share 18 groups, a 64-block tile touches at most 2 shares
+    # weights leave HBM once at 2048 rows: 8 row chunks share 9 groups of pairs, a 64-block tile touches at most 2 shares
     assert _slots_by_the_stated_schedule(2048, 22016, 4096) == 2
 
 
