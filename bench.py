@@ -37,7 +37,7 @@ PROMPT_LEN = 2048
 HBM_NOMINAL_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one gemm_bf16_kernel launch (ncu --set full, M=64 N=22016 K=4096:
 # profiles/gemm_bf16_kernel_M64_N22016_K4096.md); algorithmic bytes of that launch: 183.7 MB.
-GEMM_TRAFFIC = 186.1e6
+GEMM_TRAFFIC = 186.0e6
 GEMM_TRAFFIC_NOTE = {"launch": "M=64 N=22016 K=4096", "algorithmic_bytes_per_launch": 183.7e6}
 
 
