@@ -27,7 +27,11 @@ def cb():
                                    (2048, 640, 512), (1000, 11008, 256), (129, 256, 11008),
                                    # row chunks of 256 walked side by side: 3 chunks (49 groups), 6 ragged chunks,
                                    # and more chunks than half the SMs (back to the plain unit list)
-                                   (513, 1536, 384), (1281, 300, 1024), (19201, 128, 64)])
+                                   (513, 1536, 384), (1281, 300, 1024), (19201, 128, 64),
+                                   # CTA pairs (more than 128 rows) at their edges: one short k block, a ragged last
+                                   # k block, weight rows that end inside the first CTA's / the second CTA's half of a
+                                   # 512-row unit, exactly one full unit
+                                   (130, 520, 72), (200, 1000, 688), (256, 512, 64), (255, 100, 4096), (257, 900, 136)])
 def test_gemm_bf16_matches_definition(cb, M, N, K):
     X = synth.normal(11, 1, (M, K), 1.0, dtype=torch.bfloat16, device="cuda")
     W = synth.normal(11, 2, (N, K), 0.05, dtype=torch.bfloat16, device="cuda")
