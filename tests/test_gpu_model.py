@@ -320,6 +320,77 @@ def test_batch_with_ragged_prompts_and_mixed_modes(cb, lens):
     assert eng.device_status() == 0
 
 
+def test_bf16_mixed_mode_batch_at_head_dim_128(cb):
+    """Ragged rows through the bf16 kernels (row offsets in the norm, RoPE, the keys-on-M attention kernel, argmax
+    and accept).  A mixed-mode batch is decoded twice with its sequences in a different order (other row offsets,
+    other page tables): every sequence must give the same entropies, modes, accepted lengths and tokens in both
+    runs, must emit its own auto-regressive continuation (taken from single-sequence runs, the path the other tests
+    hold against the oracle), and the forward's row count must follow the modes."""
+    ms = synth.ModelShape(2, 256, 2, 128, 512, 1024, "bf16")
+    lens = (40, 75, 9, 130)
+    B = len(lens)
+    rig = Rig(cb, ms, max_batch=B, max_tokens=400)
+    eng = rig.eng
+    tree = synth.best_first_tree(24, rig.topk)
+    th, th1 = eng.tree(tree), eng.tree(synth.single_node_tree())
+    prompts = [[int(t) for t in synth.make_prompt(ms.vocab, L, seq=40 + i)] for i, L in enumerate(lens)]
+    n_steps, lengths = 10, [3, 1, 4, 2]
+
+    def alone(b, n):
+        """n auto-regressive steps of sequence b on its own (threshold below any entropy)."""
+        eng.prefill(torch.tensor([prompts[b]], dtype=torch.int32, device="cuda"), [lens[b]])
+        Ss, out = [], []
+        for _ in range(n):
+            eng.step(th1, -1.0, None)
+            torch.cuda.synchronize()
+            assert int(eng.h_mode[0]) == cb.MODE_AR and int(eng.h_n_accept[0]) == 1
+            Ss.append(float(eng.h_S[0]))
+            out.append(int(eng.h_tokens[0, 0]))
+        return Ss, out
+
+    runs = [alone(b, 5 * n_steps) for b in range(B)]
+    truths = [r[1] + [0] * 64 for r in runs]
+    # a threshold in the widest gap of the entropies seen on those paths, so that both modes occur
+    Ss = sorted(S for r in runs for S in r[0][:n_steps])
+    g, i = max((Ss[k + 1] - Ss[k], k) for k in range(len(Ss) // 4, 3 * len(Ss) // 4))
+    T = 0.5 * (Ss[i] + Ss[i + 1])
+
+    def batch(order):
+        tok = torch.zeros(B, max(lens), dtype=torch.int32, device="cuda")
+        for pos, b in enumerate(order):
+            tok[pos, :lens[b]] = torch.tensor(prompts[b], dtype=torch.int32)
+        eng.prefill(tok, [lens[b] for b in order])
+        outs = {b: [] for b in order}
+        recs = {b: [] for b in order}
+        mixed = 0
+        for step in range(n_steps):
+            plant = torch.tensor([plant_tokens(tree, truths[b], len(outs[b]), lengths[step % len(lengths)]) for b in order],
+                                 dtype=torch.int32, device="cuda")
+            eng.step(th, T, plant)
+            torch.cuda.synchronize()
+            modes = [int(eng.h_mode[pos]) for pos in range(B)]
+            want_rows = sum(1 if m == cb.MODE_AR else tree.n for m in modes) if cb.MODE_PAR in modes else B
+            assert eng.last_forward_rows() == want_rows, (step, modes)
+            mixed += len(set(modes)) == 2
+            for pos, b in enumerate(order):
+                na = int(eng.h_n_accept[pos])
+                toks = [int(t) for t in eng.h_tokens[pos, :na]]
+                recs[b].append((float(eng.h_S[pos]), modes[pos], toks))
+                outs[b].extend(toks)
+        assert eng.device_status() == 0
+        return recs, outs, mixed
+
+    recs_a, outs_a, mixed_a = batch((0, 1, 2, 3))
+    recs_b, outs_b, mixed_b = batch((2, 0, 3, 1))
+    seen = set()
+    for b in range(B):
+        for step, (ra, rb) in enumerate(zip(recs_a[b], recs_b[b])):
+            assert ra[1] == rb[1] and ra[2] == rb[2] and abs(ra[0] - rb[0]) < 1e-5, (b, step, ra, rb)
+            seen.add(ra[1])
+        assert outs_a[b] == truths[b][:len(outs_a[b])] and len(outs_a[b]) >= n_steps, (b, outs_a[b], truths[b][:len(outs_a[b])])
+    assert seen == {cb.MODE_AR, cb.MODE_PAR} and mixed_a >= 2 and mixed_a == mixed_b, (seen, mixed_a, mixed_b, g)
+
+
 def test_batch_16_with_128_node_trees(cb):
     """Sweep corner at small width: 16 ragged sequences, a 128-node tree (two ancestor words, 2048 rows
     per forward), planted candidates; every sequence must emit its own auto-regressive continuation."""
