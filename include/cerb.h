@@ -239,6 +239,12 @@ typedef struct cerb_attn_args {
   size_t scratch_bytes;
 } cerb_attn_args;
 
+/* Errors found on the device (a bounded wait that ran out: CERB_E_TIMEOUT; max_len smaller than a
+ * sequence's len + n: CERB_E_SHAPE) are written to the four int32 status words at bytes 4080..4095 of
+ * the scratch ([0] code, [1] which wait, [2] which block, [3] which launch); the call itself only
+ * enqueues and returns CERB_OK.  A launch that finds word [0] set runs with its waits shortened to
+ * microseconds, produces nothing useful and leaves the word as it is; the caller reads the words after
+ * synchronising and clears the first 4 KB before the next use. */
 int cerb_attn_scratch_bytes(int32_t B, int32_t n, int32_t n_heads, int32_t head_dim, size_t* bytes_out);
 int cerb_tree_attention(const cerb_attn_args* args, void* stream);
 

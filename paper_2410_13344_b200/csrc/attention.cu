@@ -107,7 +107,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
   __shared__ __align__(8) uint64_t full_bar[STAGES];
   __shared__ __align__(8) uint64_t empty_bar[STAGES];
   __shared__ int page_list[kMaxPagesPerCta];
-  __shared__ int aborted_s;
+  __shared__ int aborted_s, exit_flag_s;
   __shared__ unsigned int ticket_s;
   __shared__ __align__(8) uint64_t cl_bar[2];
   volatile int* aborted = &aborted_s;
@@ -133,6 +133,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
 
   if (threadIdx.x == 0) {
     aborted_s = (*p.status != 0);
+    exit_flag_s = 0;
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(smem_u32(&full_bar[s]), 1);
       mbar_init(smem_u32(&empty_bar[s]), NW);
@@ -160,11 +161,14 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
     if (lane == 0) {
       int early = 0;
       while (t0 + early < t_end && early < STAGES && (t0 + early + 1) * TILE <= L) ++early;
+      int issued = 0;
       for (int t = t0, i = 0; t < t_end; ++t, ++i) {
         if (i == early) { griddep_wait(); griddep_launch(); }
         int s = i % STAGES;
         uint32_t ph = (uint32_t)(i / STAGES) & 1u;
         mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, wc, 301);
+        if (*aborted) break;                       // a wait ran out somewhere in this CTA: issue nothing more
+        issued = i + 1;
         uint32_t fb = smem_u32(&full_bar[s]);
         mbar_expect_tx(fb, STAGE_BYTES);
         uint32_t kdst = smem_base + (uint32_t)s * STAGE_BYTES, vdst = kdst + KV_BYTES;
@@ -178,6 +182,11 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
             tma_load_2d(vdst + off, &tmV, hf * 64, row, fb);
           }
         }
+      }
+      if (*aborted) {
+        // give-up path: the copies already issued still land in this CTA's shared memory; see each of them in
+        for (int i = issued > STAGES ? issued - STAGES : 0; i < issued; ++i)
+          mbar_wait_drain(smem_u32(&full_bar[i % STAGES]), (uint32_t)(i / STAGES) & 1u, 20000000ll);
       }
     }
     griddep_wait();      // (a lane that has waited already returns at once)
@@ -453,7 +462,7 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
         if (c4 == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
       }
       compute_bar(NW * 32);                                                          // this CTA has read all it needs
-      if (warp == 0) cluster_meet(&cl_bar[1], p.nsplit, lane, wc, 304);
+      if (warp == 0) cluster_meet_before_exit(&cl_bar[1], p.nsplit, lane, wc, &exit_flag_s, 304);
     }
     __syncthreads();                           // nobody exits before warp 0 has seen every member done
   }
@@ -509,10 +518,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
   constexpr uint32_t QHALF = (uint32_t)QROWS * 128u, TC_Q_BYTES = 2 * QHALF;
   constexpr uint32_t TC_P_BYTES = (uint32_t)QROWS * 128u;      // P: one term (hi or lo) of one softmax group
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_k[SK], empty_k[SK], full_v[SV], empty_v[SV], s_full[2], s_free[2], p_ready[2], pv_done[2], q_ready;
+  __shared__ __align__(8) uint64_t full_k[SK], empty_k[SK], full_v[SV], empty_v[SV], s_full[2], s_free[2], p_ready[2], pv_done[2], q_ready, drain_bar[2];
   __shared__ int page_list[kMaxPagesPerCta];
   __shared__ uint32_t tmem_slot;
-  __shared__ int aborted_s;
+  __shared__ int aborted_s, exit_flag_s;
   __shared__ unsigned int ticket_s;
   __shared__ __align__(8) uint64_t cl_bar[2];
   volatile int* aborted = &aborted_s;
@@ -546,6 +555,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
 
   if (threadIdx.x == 0) {
     aborted_s = (*p.status != 0);
+    exit_flag_s = 0;
     for (int s = 0; s < SK; ++s) {
       mbar_init(smem_u32(&full_k[s]), 1);
       mbar_init(smem_u32(&empty_k[s]), 1);
@@ -561,6 +571,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       mbar_init(smem_u32(&pv_done[g]), 1);
     }
     mbar_init(smem_u32(&q_ready), 4);
+    mbar_init(smem_u32(&drain_bar[0]), 1);
+    mbar_init(smem_u32(&drain_bar[1]), 1);
     mbar_init(smem_u32(&cl_bar[0]), (uint32_t)p.nsplit);
     mbar_init(smem_u32(&cl_bar[1]), (uint32_t)p.nsplit);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -597,17 +609,23 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       // (measured, 16 x 8192 and 4 x 4096 keys); with the shared ring it is 1-5 % slower, hence the other branch.
       static_assert(PAGES_PER_TILE == 4, "the lane -> box map below assumes four pages per tile");
       const int is_v = lane >> 3, pg = (lane >> 1) & 3, hf = lane & 1;
+      int issued = 0;
       for (int i = 0; i < T; ++i) {
         if (i == early) { griddep_wait(); griddep_launch(); }
         const int sk = i % SK, sv = i % SV;
         const uint32_t fk = smem_u32(&full_k[sk]), fv = smem_u32(&full_v[sv]);
+        int stop = 0;
         if (lane == 0) {
           mbar_wait_polite(smem_u32(&empty_k[sk]), ((uint32_t)(i / SK) & 1u) ^ 1u, wc, 305);
-          mbar_expect_tx(fk, TC_KV_BYTES);
           mbar_wait_polite(smem_u32(&empty_v[sv]), ((uint32_t)(i / SV) & 1u) ^ 1u, wc, 306);
-          mbar_expect_tx(fv, TC_KV_BYTES);
+          stop = *aborted;
+          if (!stop) {
+            mbar_expect_tx(fk, TC_KV_BYTES);
+            mbar_expect_tx(fv, TC_KV_BYTES);
+          }
         }
-        __syncwarp();
+        if (__shfl_sync(0xffffffffu, stop, 0)) break;          // a wait ran out somewhere in this CTA: issue nothing more
+        issued = i + 1;
         if (lane < 16) {
           const int row = page_list[i * PAGES_PER_TILE + pg];       // out-of-range rows are zero-filled by TMA
           const uint32_t dst = (is_v ? v_ring + (uint32_t)sv * TC_KV_BYTES : k_ring + (uint32_t)sk * TC_KV_BYTES) +
@@ -615,12 +633,22 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
           tma_load_2d(dst, is_v ? &tmV : &tmK, hf * 64, row, is_v ? fv : fk);
         }
       }
+      if (lane == 0 && *aborted) {
+        // give-up path: the copies already issued still land in this CTA's shared memory; see each of them in
+        for (int i = issued > SK ? issued - SK : 0; i < issued; ++i)
+          mbar_wait_drain(smem_u32(&full_k[i % SK]), (uint32_t)(i / SK) & 1u, 20000000ll);
+        for (int i = issued > SV ? issued - SV : 0; i < issued; ++i)
+          mbar_wait_drain(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, 20000000ll);
+      }
     } else if (lane == 0) {
       // K and V of a tile share the V ring's barriers (SK == SV): one wait and one arrival per tile
+      int issued = 0;
       for (int i = 0; i < T; ++i) {
         if (i == early) { griddep_wait(); griddep_launch(); }
         const int sv = i % SV;
         mbar_wait_polite(smem_u32(&empty_v[sv]), ((uint32_t)(i / SV) & 1u) ^ 1u, wc, 307);
+        if (*aborted) break;
+        issued = i + 1;
         const uint32_t fv = smem_u32(&full_v[sv]);
         mbar_expect_tx(fv, 2 * TC_KV_BYTES);
         const uint32_t kdst = k_ring + (uint32_t)sv * TC_KV_BYTES, vdst = v_ring + (uint32_t)sv * TC_KV_BYTES;
@@ -639,6 +667,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
             tma_load_2d(vdst + (uint32_t)hf * 8192u + (uint32_t)pg * (CERB_PAGE * 128), &tmV, hf * 64, row, fv);
         }
       }
+      if (*aborted)
+        for (int i = issued > SV ? issued - SV : 0; i < issued; ++i)
+          mbar_wait_drain(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, 20000000ll);
     }
     griddep_wait();      // (a lane that has waited already returns at once)
     griddep_launch();
@@ -657,6 +688,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
         if (!UNI) mbar_wait(smem_u32(&full_k[i % SK]), (uint32_t)(i / SK) & 1u, wc, 309);
         else mbar_wait(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, wc, 310);
         mbar_wait(smem_u32(&s_free[g]), ((uint32_t)k & 1u) ^ 1u, wc, 311);
+        if (*aborted) break;
         tc_fence_after();
         const uint32_t kb = k_ring + (uint32_t)(i % SK) * TC_KV_BYTES;
         const uint64_t k_desc0 = desc_k_sw128(kb), k_desc1 = desc_k_sw128(kb + 8192u);
@@ -667,6 +699,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
         for (int kk = 0; kk < 4; ++kk) umma(d, q_desc1 + (uint64_t)(kk * 2), k_desc1 + (uint64_t)(kk * 2), idesc_s, 1u);
         if (!UNI) umma_commit(smem_u32(&empty_k[i % SK]));     // the K tile is free once these MMAs have retired
         umma_commit(smem_u32(&s_full[g]));
+      }
+      if (*aborted) {                                // give-up path: see the MMAs already issued retire
+        umma_commit(smem_u32(&drain_bar[0]));
+        mbar_wait_drain(smem_u32(&drain_bar[0]), 0, 20000000ll);
       }
     }
   } else if (warp == 10) {
@@ -680,6 +716,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
         const int g = j & 1, k = j >> 1;
         mbar_wait(smem_u32(&p_ready[g]), (uint32_t)k & 1u, wc, 312);
         mbar_wait(smem_u32(&full_v[j % SV]), (uint32_t)(j / SV) & 1u, wc, 313);
+        if (*aborted) break;
         tc_fence_after();
         const uint32_t vb = v_ring + (uint32_t)(j % SV) * TC_KV_BYTES;
         const uint32_t d = tmem + 128u + (uint32_t)g * 128u;
@@ -692,6 +729,10 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
         }
         umma_commit(smem_u32(&empty_v[j % SV]));
         umma_commit(smem_u32(&pv_done[g]));
+      }
+      if (*aborted) {                                // give-up path: see the MMAs already issued retire
+        umma_commit(smem_u32(&drain_bar[1]));
+        mbar_wait_drain(smem_u32(&drain_bar[1]), 0, 20000000ll);
       }
     }
   } else {
@@ -963,7 +1004,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
         if (c4 == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + r] = (M + log2f(Lsum)) * LN2;
       }
       compute_bar(256);                                                              // this CTA has read all it needs
-      if (warp == 2) cluster_meet(&cl_bar[1], p.nsplit, lane, wc, 319);
+      if (warp == 2) cluster_meet_before_exit(&cl_bar[1], p.nsplit, lane, wc, &exit_flag_s, 319);
     }
   }
   tc_fence_before();

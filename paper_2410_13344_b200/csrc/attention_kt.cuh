@@ -90,7 +90,7 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
   __shared__ int raise_at[2][4];                   // [tile parity][query block]: 1 + the last tile at which a raise was requested
   __shared__ float l_part[4][128];                 // per lane quarter: partial row sums, added at the end
   __shared__ uint32_t tmem_slot;
-  __shared__ int aborted_s;
+  __shared__ int aborted_s, exit_flag_s;
   __shared__ unsigned int ticket_s;
   volatile int* aborted = &aborted_s;
   const WaitCtx wc{p.wait_cycles, aborted, p.status};
@@ -119,6 +119,7 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
 
   if (threadIdx.x == 0) {
     aborted_s = (*p.status != 0);
+    exit_flag_s = 0;
     for (int s = 0; s < NU; ++s) {
       mbar_init(smem_u32(&full_u[0][s]), NPROD);
       mbar_init(smem_u32(&full_u[1][s]), NPROD);
@@ -623,7 +624,7 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
         if (c4 == 0 && p.lse) p.lse[((size_t)b * p.H + h) * p.n + rr] = (M + log2f(Lsum)) * LN2;
       }
       asm volatile("bar.sync 2, %0;" ::"r"(128 * NCB) : "memory");            // this CTA has read all it needs
-      if (warp == 0) cluster_meet(&cl_bar[1], p.nsplit, lane, wc, 113);
+      if (warp == 0) cluster_meet_before_exit(&cl_bar[1], p.nsplit, lane, wc, &exit_flag_s, 113);
     }
   }
   tc_fence_before();

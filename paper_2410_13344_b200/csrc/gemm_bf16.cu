@@ -574,11 +574,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_pair_kernel(const __grid_con
   // Neither CTA leaves (nor frees its tensor memory) before the other is done: copies, commits and arrivals cross
   // between them until then.  The rendezvous keeps a budget of its own, far above that of the other waits, so that a
   // CTA which has given up still finds its partner.
-  if (warp == 2) {
-    const long long meet_budget = p.wait_cycles * 4 > 40000000ll ? p.wait_cycles * 4 : 40000000ll;
-    const WaitCtx wm{meet_budget, &meet_flag_s, p.status, wc.tag};
-    cluster_meet(&meet_bar, 2, lane, wm, 215);
-  }
+  if (warp == 2) cluster_meet_before_exit(&meet_bar, 2, lane, wc, &meet_flag_s, 215);
   __syncthreads();
   if (warp == 1)
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");

@@ -255,6 +255,14 @@ __device__ __forceinline__ void cluster_meet(uint64_t* bar, int members, int idx
   }
   wait_ran_out(w, site);
 }
+// Last rendezvous before a CTA of a cluster leaves: the others may still be reading this CTA's shared memory or about to
+// arrive on its barriers, so this wait keeps a budget of its own, far above that of the other waits (which shrink to
+// microseconds once a wait has run out): a CTA that has given up still waits for its partners here.
+__device__ __forceinline__ void cluster_meet_before_exit(uint64_t* bar, int members, int idx, const WaitCtx& w, int* flag, int site) {
+  const long long budget = w.budget * 4 > 40000000ll ? w.budget * 4 : 40000000ll;
+  const WaitCtx wx{budget, flag, w.status, w.tag};
+  cluster_meet(bar, members, idx, wx, site);
+}
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));

@@ -239,6 +239,45 @@ def test_bounded_wait_runs_out_cleanly_and_the_next_call_is_correct(cb):
     assert close(out[ri][:, ci].cpu(), ref, 0) < 2e-3          # 262144 products per element
 
 
+@pytest.mark.parametrize("B,n,H,L", [(1, 64, 32, 6000), (1, 8, 32, 6000), (1, 128, 32, 6000), (4, 64, 32, 3000)])
+def test_attention_after_a_timeout_comes_back_and_the_next_call_is_correct(cb, B, n, H, L):
+    """A wait that runs out leaves CERB_E_TIMEOUT in the status word, and every kernel that finds the word set when
+    it starts (the rest of a decoding step after a time-out) shortens its waits to microseconds, issues no copies
+    and no MMAs, lets those waits run out -- nothing fills its barriers -- and leaves, tensor memory freed and its
+    cluster partners met.  Here the caller sets the word before the launch, for the three bf16 kernels (keys-on-M
+    with a cluster of splits and with one split, warp-MMA, query-rows-on-M): the launch must come back with the word
+    still set, and the same call after the word has been cleared must match the oracle."""
+    Dh = 128
+    max_len = L + n
+    mp = (max_len + 15) // 16 + 1
+    tree = synth.random_parent_tree(n, 5, tree_id=77)
+    q = synth.normal(synth.SEED_ATTN, 801, (B, n, H, Dh), 1.0, dtype=torch.bfloat16, device="cuda")
+    kp = synth.normal(synth.SEED_ATTN, 802, (B * mp, H, 16, Dh), 1.0, dtype=torch.bfloat16, device="cuda")
+    vp = synth.normal(synth.SEED_ATTN, 803, (B * mp, H, 16, Dh), 1.0, dtype=torch.bfloat16, device="cuda")
+    pt = torch.from_numpy(np.stack([synth.shuffled_page_table(mp, mp, table_id=880 + b, first=b * mp) for b in range(B)])).cuda()
+    anc = torch.from_numpy(cb.tree_ancestors(tree.parent).view(np.int64)).cuda()
+    lens = torch.full((B,), L, dtype=torch.int32, device="cuda")
+    scale = 1.0 / math.sqrt(Dh)
+    nb = cb.C.c_size_t(0)
+    assert cb.lib().cerb_attn_scratch_bytes(B, n, H, Dh, cb.C.byref(nb)) == cb.OK
+    scratch = torch.zeros(nb.value, dtype=torch.uint8, device="cuda")
+    status = scratch[4096 - 16:4096].view(torch.int32)            # the status words of this entry point
+    status[0] = cb.E_TIMEOUT
+    cb.tree_attention(q, kp, vp, pt, lens, anc, scale, max_len, scratch=scratch)
+    torch.cuda.synchronize()
+    assert int(status[0].item()) == cb.E_TIMEOUT
+    scratch[:4096] = 0                                            # status and ticket counters, as before a first use
+    out, lse, _ = cb.tree_attention(q, kp, vp, pt, lens, anc, scale, max_len, scratch=scratch)
+    torch.cuda.synchronize()
+    assert int(status[0].item()) == 0
+    b = B - 1
+    pages = pt[b].cpu().long()
+    kc = kp.cpu()[pages].permute(0, 2, 1, 3).reshape(-1, H, Dh).double()
+    vc = vp.cpu()[pages].permute(0, 2, 1, 3).reshape(-1, H, Dh).double()
+    O, l = orc.tree_attention(q[b].cpu().double(), kc[:L], vc[:L], kc[L:L + n], vc[L:L + n], tree.parent, scale)
+    assert close(out[b], O, 0) < TOL_BF16 and close(lse[b], l, 0) < 2e-3
+
+
 def test_abi_rejects_bad_arguments(cb):
     L = cb.lib()
     assert L.cerb_tree_attention(None, None) == cb.E_ARG
