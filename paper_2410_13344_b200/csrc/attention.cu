@@ -161,14 +161,15 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
     if (lane == 0) {
       int early = 0;
       while (t0 + early < t_end && early < STAGES && (t0 + early + 1) * TILE <= L) ++early;
-      int issued = 0;
-      for (int t = t0, i = 0; t < t_end; ++t, ++i) {
+      // (the abort flag itself is looked at once, for a launch that starts after a time-out: nothing is issued then;
+      // later a wait that gives up says so in its return value, which costs the loop nothing)
+      const int t_stop = *aborted ? t0 : t_end;
+      int i = 0;
+      for (int t = t0; t < t_stop; ++t, ++i) {
         if (i == early) { griddep_wait(); griddep_launch(); }
         int s = i % STAGES;
         uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-        mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, wc, 301);
-        if (*aborted) break;                       // a wait ran out somewhere in this CTA: issue nothing more
-        issued = i + 1;
+        if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, wc, 301)) break;      // the consumers have stopped: issue nothing more
         uint32_t fb = smem_u32(&full_bar[s]);
         mbar_expect_tx(fb, STAGE_BYTES);
         uint32_t kdst = smem_base + (uint32_t)s * STAGE_BYTES, vdst = kdst + KV_BYTES;
@@ -184,9 +185,9 @@ __global__ void __launch_bounds__((WQ * WK + 1) * 32) tree_attn_bf16_kernel(cons
         }
       }
       if (*aborted) {
-        // give-up path: the copies already issued still land in this CTA's shared memory; see each of them in
-        for (int i = issued > STAGES ? issued - STAGES : 0; i < issued; ++i)
-          mbar_wait_drain(smem_u32(&full_bar[i % STAGES]), (uint32_t)(i / STAGES) & 1u, 20000000ll);
+        // give-up path: the copies already issued (units 0 .. i-1) still land in this CTA's shared memory; see each of them in
+        for (int j = i > STAGES ? i - STAGES : 0; j < i; ++j)
+          mbar_wait_drain(smem_u32(&full_bar[j % STAGES]), (uint32_t)(j / STAGES) & 1u, 20000000ll);
       }
     }
     griddep_wait();      // (a lane that has waited already returns at once)
@@ -609,23 +610,24 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       // (measured, 16 x 8192 and 4 x 4096 keys); with the shared ring it is 1-5 % slower, hence the other branch.
       static_assert(PAGES_PER_TILE == 4, "the lane -> box map below assumes four pages per tile");
       const int is_v = lane >> 3, pg = (lane >> 1) & 3, hf = lane & 1;
-      int issued = 0;
-      for (int i = 0; i < T; ++i) {
+      const int T_stop = *aborted ? 0 : T;         // a launch that starts after a time-out issues nothing
+      int i = 0;
+      for (; i < T_stop; ++i) {
         if (i == early) { griddep_wait(); griddep_launch(); }
         const int sk = i % SK, sv = i % SV;
         const uint32_t fk = smem_u32(&full_k[sk]), fv = smem_u32(&full_v[sv]);
         int stop = 0;
         if (lane == 0) {
-          mbar_wait_polite(smem_u32(&empty_k[sk]), ((uint32_t)(i / SK) & 1u) ^ 1u, wc, 305);
-          mbar_wait_polite(smem_u32(&empty_v[sv]), ((uint32_t)(i / SV) & 1u) ^ 1u, wc, 306);
-          stop = *aborted;
-          if (!stop) {
+          // (a wait that gives up says so in its return value: the consumers have stopped, nothing more is issued)
+          if (mbar_wait_polite(smem_u32(&empty_k[sk]), ((uint32_t)(i / SK) & 1u) ^ 1u, wc, 305) &&
+              mbar_wait_polite(smem_u32(&empty_v[sv]), ((uint32_t)(i / SV) & 1u) ^ 1u, wc, 306)) {
             mbar_expect_tx(fk, TC_KV_BYTES);
             mbar_expect_tx(fv, TC_KV_BYTES);
+          } else {
+            stop = 1;
           }
         }
-        if (__shfl_sync(0xffffffffu, stop, 0)) break;          // a wait ran out somewhere in this CTA: issue nothing more
-        issued = i + 1;
+        if (__any_sync(0xffffffffu, stop)) break;
         if (lane < 16) {
           const int row = page_list[i * PAGES_PER_TILE + pg];       // out-of-range rows are zero-filled by TMA
           const uint32_t dst = (is_v ? v_ring + (uint32_t)sv * TC_KV_BYTES : k_ring + (uint32_t)sk * TC_KV_BYTES) +
@@ -634,21 +636,20 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
         }
       }
       if (lane == 0 && *aborted) {
-        // give-up path: the copies already issued still land in this CTA's shared memory; see each of them in
-        for (int i = issued > SK ? issued - SK : 0; i < issued; ++i)
-          mbar_wait_drain(smem_u32(&full_k[i % SK]), (uint32_t)(i / SK) & 1u, 20000000ll);
-        for (int i = issued > SV ? issued - SV : 0; i < issued; ++i)
-          mbar_wait_drain(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, 20000000ll);
+        // give-up path: the copies already issued (tiles 0 .. i-1) still land in this CTA's shared memory; see each of them in
+        for (int j = i > SK ? i - SK : 0; j < i; ++j)
+          mbar_wait_drain(smem_u32(&full_k[j % SK]), (uint32_t)(j / SK) & 1u, 20000000ll);
+        for (int j = i > SV ? i - SV : 0; j < i; ++j)
+          mbar_wait_drain(smem_u32(&full_v[j % SV]), (uint32_t)(j / SV) & 1u, 20000000ll);
       }
     } else if (lane == 0) {
       // K and V of a tile share the V ring's barriers (SK == SV): one wait and one arrival per tile
-      int issued = 0;
-      for (int i = 0; i < T; ++i) {
+      const int T_stop = *aborted ? 0 : T;         // a launch that starts after a time-out issues nothing
+      int i = 0;
+      for (; i < T_stop; ++i) {
         if (i == early) { griddep_wait(); griddep_launch(); }
         const int sv = i % SV;
-        mbar_wait_polite(smem_u32(&empty_v[sv]), ((uint32_t)(i / SV) & 1u) ^ 1u, wc, 307);
-        if (*aborted) break;
-        issued = i + 1;
+        if (!mbar_wait_polite(smem_u32(&empty_v[sv]), ((uint32_t)(i / SV) & 1u) ^ 1u, wc, 307)) break;
         const uint32_t fv = smem_u32(&full_v[sv]);
         mbar_expect_tx(fv, 2 * TC_KV_BYTES);
         const uint32_t kdst = k_ring + (uint32_t)sv * TC_KV_BYTES, vdst = v_ring + (uint32_t)sv * TC_KV_BYTES;
@@ -668,8 +669,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
         }
       }
       if (*aborted)
-        for (int i = issued > SV ? issued - SV : 0; i < issued; ++i)
-          mbar_wait_drain(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, 20000000ll);
+        for (int j = i > SV ? i - SV : 0; j < i; ++j)
+          mbar_wait_drain(smem_u32(&full_v[j % SV]), (uint32_t)(j / SV) & 1u, 20000000ll);
     }
     griddep_wait();      // (a lane that has waited already returns at once)
     griddep_launch();
@@ -683,12 +684,12 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
       const uint32_t idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
       const uint64_t q_desc0 = desc_k_sw128(q_base), q_desc1 = desc_k_sw128(q_base + QHALF);
       mbar_wait(smem_u32(&q_ready), 0, wc, 308);
-      for (int i = 0; i < T; ++i) {
+      const int T_stop = *aborted ? 0 : T;
+      for (int i = 0; i < T_stop; ++i) {
         const int g = i & 1, k = i >> 1;
-        if (!UNI) mbar_wait(smem_u32(&full_k[i % SK]), (uint32_t)(i / SK) & 1u, wc, 309);
-        else mbar_wait(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, wc, 310);
-        mbar_wait(smem_u32(&s_free[g]), ((uint32_t)k & 1u) ^ 1u, wc, 311);
-        if (*aborted) break;
+        const bool ok_kv = !UNI ? mbar_wait(smem_u32(&full_k[i % SK]), (uint32_t)(i / SK) & 1u, wc, 309)
+                                : mbar_wait(smem_u32(&full_v[i % SV]), (uint32_t)(i / SV) & 1u, wc, 310);
+        if (!mbar_wait(smem_u32(&s_free[g]), ((uint32_t)k & 1u) ^ 1u, wc, 311) || !ok_kv) break;
         tc_fence_after();
         const uint32_t kb = k_ring + (uint32_t)(i % SK) * TC_KV_BYTES;
         const uint64_t k_desc0 = desc_k_sw128(kb), k_desc1 = desc_k_sw128(kb + 8192u);
@@ -712,11 +713,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tree_attn_tc_kernel(const __gri
     if (lane == 0) {
       // B operand (V) is MN-major, N = 128 (two 64-wide swizzle atoms, p.v_lbo bytes apart)
       const uint32_t idesc_pv = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
-      for (int j = 0; j < T; ++j) {
+      const int T_stop = *aborted ? 0 : T;
+      for (int j = 0; j < T_stop; ++j) {
         const int g = j & 1, k = j >> 1;
-        mbar_wait(smem_u32(&p_ready[g]), (uint32_t)k & 1u, wc, 312);
-        mbar_wait(smem_u32(&full_v[j % SV]), (uint32_t)(j / SV) & 1u, wc, 313);
-        if (*aborted) break;
+        if (!mbar_wait(smem_u32(&p_ready[g]), (uint32_t)k & 1u, wc, 312)) break;
+        if (!mbar_wait(smem_u32(&full_v[j % SV]), (uint32_t)(j / SV) & 1u, wc, 313)) break;
         tc_fence_after();
         const uint32_t vb = v_ring + (uint32_t)(j % SV) * TC_KV_BYTES;
         const uint32_t d = tmem + 128u + (uint32_t)g * 128u;

@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
   // dead-lock, measured).  Hence one "landed" barrier per slot and per kind of unit: full_u[kind][slot], whose
   // phases the one consumer of that kind sees in order.
   auto unit_parity = [](int u) { return (uint32_t)((NU & 1) ? (u / NU) >> 1 : u / NU) & 1u; };
-  auto wait_unit = [&](int u, int site) { mbar_wait(smem_u32(&full_u[u & 1][u % NU]), unit_parity(u), wc, site); };
+  auto wait_unit = [&](int u, int site) { return mbar_wait(smem_u32(&full_u[u & 1][u % NU]), unit_parity(u), wc, site); };
   if (warp >= NSW && warp < NSW + NPROD) {
     // ---------------- TMA producers ----------------
     // producer w issues boxes w, w + NPROD, ... of every unit (box = page * 2 + half of head_dim), one per lane
@@ -186,17 +186,19 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
     const int pg = box >> 1, hf = box & 1;
     const uint64_t pol = l2_policy(true);            // K/V are read once per step
     int issued = 0;
-    for (int u = 0; u < 2 * T; ++u) {
+    // (the abort flag itself is looked at once, for a launch that starts after a time-out: nothing is issued then;
+    // later a wait that gives up says so in its return value, which costs the loop nothing)
+    const int u_stop = *aborted ? 0 : 2 * T;
+    for (int u = 0; u < u_stop; ++u) {
       if (u == early_units) { griddep_wait(); griddep_launch(); }
       const int slot = u % NU, t = u >> 1;
       const uint32_t fb = smem_u32(&full_u[u & 1][slot]);
       int stop = 0;
       if (lane == 0) {
-        mbar_wait_polite(smem_u32(&empty_u[slot]), ((uint32_t)(u / NU) & 1u) ^ 1u, wc, 101);
-        stop = *aborted;
+        stop = !mbar_wait_polite(smem_u32(&empty_u[slot]), ((uint32_t)(u / NU) & 1u) ^ 1u, wc, 101);
         if (!stop) mbar_expect_tx(fb, KT_UNIT / NPROD);
       }
-      if (__shfl_sync(0xffffffffu, stop, 0)) break;            // a wait ran out somewhere in this CTA: issue nothing more
+      if (__shfl_sync(0xffffffffu, stop, 0)) break;            // this wait ran out (the consumers have stopped): issue nothing more
       if (lane < BOXES) {
         const int row = page_list[t * KT_PAGES + pg];          // out-of-range rows are zero-filled by TMA
         const uint32_t dst = ring + (uint32_t)slot * KT_UNIT + (uint32_t)hf * KT_HALF + (uint32_t)pg * (CERB_PAGE * 128);
@@ -220,11 +222,11 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
       constexpr uint32_t idesc_s = idesc_bf16(128, NQ, false, false);
       const uint64_t q_desc0 = desc_k_sw128(q_base), q_desc1 = desc_k_sw128(q_base + QHALF);
       mbar_wait(smem_u32(&q_ready), 0, wc, 102);
-      for (int t = 0; t < T; ++t) {
+      const int t_stop = *aborted ? 0 : T;
+      for (int t = 0; t < t_stop; ++t) {
         const int u = 2 * t, slot = u % NU, sb = t & 1;
-        wait_unit(u, 103);
-        mbar_wait(smem_u32(&s_free[sb]), ((uint32_t)(t >> 1) & 1u) ^ 1u, wc, 104);
-        if (*aborted) break;
+        if (!wait_unit(u, 103)) break;
+        if (!mbar_wait(smem_u32(&s_free[sb]), ((uint32_t)(t >> 1) & 1u) ^ 1u, wc, 104)) break;
         tc_fence_after();
         const uint32_t kb = ring + (uint32_t)slot * KT_UNIT;
         const uint64_t k_desc0 = desc_k_sw128(kb), k_desc1 = desc_k_sw128(kb + KT_HALF);
@@ -249,12 +251,12 @@ __global__ void __launch_bounds__(kt_threads(NCB), 1) tree_attn_kt_kernel(const 
       // A = V tile read M-major (M = head_dim: two 64-wide blocks KT_HALF apart; 8-key groups 1024 bytes apart),
       // B = P^T read N-major (N = hi and lo terms side by side: 2 NQ / 64 blocks KT_HALF apart)
       constexpr uint32_t idesc_pv = idesc_bf16(128, 2 * NQ, true, true);
-      for (int t = 0; t < T; ++t) {
+      const int t_stop = *aborted ? 0 : T;
+      for (int t = 0; t < t_stop; ++t) {
         const int u = 2 * t + 1, slot = u % NU;
         const int pb = t % PB;
-        mbar_wait(smem_u32(&p_ready[pb]), (uint32_t)(t / PB) & 1u, wc, 105);
-        wait_unit(u, 106);
-        if (*aborted) break;
+        if (!mbar_wait(smem_u32(&p_ready[pb]), (uint32_t)(t / PB) & 1u, wc, 105)) break;
+        if (!wait_unit(u, 106)) break;
         tc_fence_after();
         const uint32_t vb = ring + (uint32_t)slot * KT_UNIT;
         const uint32_t d = tmem + O_COL;

@@ -187,8 +187,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
       for (int i = pre; i < n_units; ++i) {
         const int s = i % p.stages;
         const uint32_t ph = (uint32_t)(i / p.stages) & 1u;
-        mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, wc, 201);
-        if (*aborted) break;                       // a wait ran out somewhere in this CTA: issue nothing more
+        if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, wc, 201)) break;     // this wait gave up (the consumers have stopped): issue nothing more
         load_w(i);
         load_x(i);
         issued = i + 1;
@@ -212,15 +211,13 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
       while (next_segment(u, u1, p.num_kb, sg)) {
         const int buf = g & 1;
         const uint32_t use = (uint32_t)(g >> 1);      // how often this buffer was used before
-        mbar_wait(smem_u32(&acc_empty[buf]), (use & 1u) ^ 1u, wc, 202);
-        if (*aborted) break;
+        if (!mbar_wait(smem_u32(&acc_empty[buf]), (use & 1u) ^ 1u, wc, 202)) break;
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)buf * p.acc_cols;
         for (int k = 0; k < sg.nkb; ++k, ++i) {
           int s = i % p.stages;
           uint32_t ph = (uint32_t)(i / p.stages) & 1u;
-          mbar_wait(smem_u32(&full_bar[s]), ph, wc, 203);
-          if (*aborted) break;
+          if (!mbar_wait(smem_u32(&full_bar[s]), ph, wc, 203)) break;
           tc_fence_after();
           uint32_t a_src = smem_base + (uint32_t)s * stage_bytes;
           uint64_t bdesc = desc_k_sw128(a_src + a_bytes);
@@ -250,8 +247,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
     while (next_segment(u, u1, p.num_kb, sg)) {
       const int buf = g & 1;
       const int tile = sg.job;
-      mbar_wait(smem_u32(&acc_full[buf]), (uint32_t)(g >> 1) & 1u, wc, 204);
-      if (*aborted) break;                         // the launch's output is undefined from here on
+      if (!mbar_wait(smem_u32(&acc_full[buf]), (uint32_t)(g >> 1) & 1u, wc, 204)) break;                         // the launch's output is undefined from here on
       tc_fence_after();
       // slot = how many CTAs before this one also work on this job
       const int job_u0 = sg.job * p.num_kb;
@@ -459,8 +455,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_pair_kernel(const __grid_con
       for (int i = pre; i < n_units; ++i) {
         const int s = i % PAIR_STAGES;
         const uint32_t ph = (uint32_t)(i / PAIR_STAGES) & 1u;
-        mbar_wait_cluster(smem_u32(&empty_bar[s]), ph ^ 1u, wc, 211);
-        if (*aborted) break;
+        if (!mbar_wait_cluster(smem_u32(&empty_bar[s]), ph ^ 1u, wc, 211)) break;
         load_w(i);
         load_x(i);
         issued = i + 1;
@@ -486,15 +481,13 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_pair_kernel(const __grid_con
       Segment sg;
       int i = 0, g = 0;
       while (next_segment(u, u1, p.num_kb, sg)) {
-        mbar_wait_cluster(smem_u32(&acc_empty), ((uint32_t)g & 1u) ^ 1u, wc, 212);
-        if (*aborted) break;
+        if (!mbar_wait_cluster(smem_u32(&acc_empty), ((uint32_t)g & 1u) ^ 1u, wc, 212)) break;
         tc_fence_after();
         const uint32_t d = tmem_base + (uint32_t)(hf * PAIR_ACT);
         for (int k = 0; k < sg.nkb; ++k, ++i) {
           const int s = i % PAIR_STAGES;
           const uint32_t ph = (uint32_t)(i / PAIR_STAGES) & 1u;
-          mbar_wait_cluster(smem_u32(&full_bar[s]), ph, wc, 213);
-          if (*aborted) break;
+          if (!mbar_wait_cluster(smem_u32(&full_bar[s]), ph, wc, 213)) break;
           tc_fence_after();
           const uint32_t src = smem_base + (uint32_t)s * PAIR_STAGE_BYTES;
           const uint64_t adesc = desc_k_sw128(src + (uint32_t)hf * A_STAGE_BYTES);
@@ -522,8 +515,7 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_pair_kernel(const __grid_con
     int g = 0;
     while (next_segment(u, u1, p.num_kb, sg)) {
       const int tile = sg.job % p.tiles, mchunk = p.lock > 1 ? my_chunk : sg.job / p.tiles;
-      mbar_wait_cluster(smem_u32(&acc_full), (uint32_t)g & 1u, wc, 214);
-      if (*aborted) break;
+      if (!mbar_wait_cluster(smem_u32(&acc_full), (uint32_t)g & 1u, wc, 214)) break;
       tc_fence_after();
       const int job_u0 = sg.job * p.num_kb;
       const int first_share = job_u0 / p.per;

@@ -67,18 +67,20 @@ __device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity
 }
 // Bounded wait: gives up after the budget.  A few plain polls first (almost every wait ends there); then the
 // budget is measured with the SM-local cycle counter, which is cheap to read, between short runs of polls
-// that each return after two microseconds at the latest.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w, int site = 0) {
+// that each return after two microseconds at the latest.  Returns false when it gave up (the hot loops test this
+// value, which costs nothing, rather than re-reading the CTA's abort flag after every wait).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& w, int site = 0) {
   for (int i = 0; i < 8; ++i)
-    if (mbar_try_wait(bar, parity)) return;
+    if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   const long long budget = *w.aborted ? kAbortedWaitCycles : w.budget;
   for (;;) {
     for (int i = 0; i < 16; ++i)
-      if (mbar_try_wait_hint(bar, parity, 2000u)) return;
+      if (mbar_try_wait_hint(bar, parity, 2000u)) return true;
     if (clock64() - t0 > budget) break;
   }
   wait_ran_out(w, site);
+  return false;
 }
 // Wait used on the way out of a CTA that has given up: for copies and MMAs that are already in flight, so that
 // none of them outlives the CTA's shared and tensor memory.  It keeps a budget of its own (what it waits for
@@ -93,19 +95,20 @@ __device__ __forceinline__ void mbar_wait_drain(uint32_t bar, uint32_t parity, l
   }
 }
 // Same bounded wait for a lane whose warp shares an issue port with busy warps: back off between polls.
-__device__ __forceinline__ void mbar_wait_polite(uint32_t bar, uint32_t parity, const WaitCtx& w, int site = 0) {
+__device__ __forceinline__ bool mbar_wait_polite(uint32_t bar, uint32_t parity, const WaitCtx& w, int site = 0) {
   for (int i = 0; i < 4; ++i)
-    if (mbar_try_wait(bar, parity)) return;
+    if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   const long long budget = *w.aborted ? kAbortedWaitCycles : w.budget;
   for (;;) {
     for (int i = 0; i < 64; ++i) {
-      if (mbar_try_wait(bar, parity)) return;
+      if (mbar_try_wait(bar, parity)) return true;
       __nanosleep(40);
     }
     if (clock64() - t0 > budget) break;
   }
   wait_ran_out(w, site);
+  return false;
 }
 
 // ---- TMA tile loads (no multicast anywhere) ----
@@ -273,17 +276,18 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 // Bounded wait on an own mbarrier whose arrivals may come from another CTA of the cluster (acquire at cluster scope).
-__device__ __forceinline__ void mbar_wait_cluster(uint32_t bar, uint32_t parity, const WaitCtx& w, int site = 0) {
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, const WaitCtx& w, int site = 0) {
   for (int i = 0; i < 8; ++i)
-    if (mbar_try_wait_cluster(bar, parity)) return;
+    if (mbar_try_wait_cluster(bar, parity)) return true;
   const long long t0 = clock64();
   const long long budget = *w.aborted ? kAbortedWaitCycles : w.budget;
   for (;;) {
     for (int i = 0; i < 64; ++i)
-      if (mbar_try_wait_cluster(bar, parity)) return;
+      if (mbar_try_wait_cluster(bar, parity)) return true;
     if (clock64() - t0 > budget) break;
   }
   wait_ran_out(w, site);
+  return false;
 }
 __device__ __forceinline__ uint32_t mapa_u32(uint32_t saddr, uint32_t rank) {
   uint32_t r;
