@@ -334,8 +334,9 @@ int cerb_set_wait_cycles(int64_t cycles);
 /* The launch sequence of the base-model forward with, per kernel, the buffers it writes and the buffers it reads
  * ahead of its dependency wait (bit masks; the paper has no counterpart, this documents the library's use of
  * programmatic dependent launch).  Writes one line per launch, "id|name|writes|reads-before-wait", for one set-up
- * launch, three layers and the tail, into buf (host).  variant 0: separate SwiGLU kernel; 1: SwiGLU inside the
- * gate-up GEMM (steps of at most 16 rows).  Returns CERB_OK when no kernel reads, ahead of its wait, a buffer
+ * launch, three layers and the tail, into buf (host).  variant 0: separate SwiGLU and RoPE kernels; 1: SwiGLU inside the
+ * gate-up GEMM (steps of at most 16 rows); 2: RoPE + cache append inside the QKV GEMM as well (such steps at
+ * head_dim 128).  Returns CERB_OK when no kernel reads, ahead of its wait, a buffer
  * that the kernel right in front of it writes, CERB_E_STATE otherwise, CERB_E_NOMEM when buf is too small. */
 int cerb_launch_order_table(int32_t variant, char* buf_host, size_t cap);
 

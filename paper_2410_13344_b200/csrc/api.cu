@@ -240,7 +240,7 @@ int gemm(cerb_ctx* c, const void* X, const ActMaps* xm, const void* W, const CUt
 struct OrderCheck {
   const int* ids;
   int n, pos;
-  explicit OrderCheck(bool fused) : pos(0) { n = launch_order_layer(fused ? 1 : 0, &ids); }
+  explicit OrderCheck(int variant) : pos(0) { n = launch_order_layer(variant, &ids); }
   bool next(int id) {
     if (id == LO_NORM_FINAL) return pos == 0;
     const bool ok = ids[pos] == id;
@@ -278,7 +278,11 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
     if (c->h_len[b] + n > c->max_pos) return CERB_E_STATE;
     if (c->h_len[b] + n > max_len) max_len = c->h_len[b] + n;
   }
-  OrderCheck oc(c->bf16 && gemm_swiglu_fusable(M, F));
+  // Steps of up to 16 rows: SwiGLU runs in the gate-up GEMM's epilogue and (head_dim 128) RoPE + cache append in the
+  // QKV GEMM's.
+  const bool fuse_swiglu = c->bf16 && gemm_swiglu_fusable(M, F);
+  const bool fuse_rope = fuse_swiglu && gemm_rope_fusable(M, g.head_dim);
+  OrderCheck oc(fuse_rope ? 2 : fuse_swiglu ? 1 : 0);
   // embedding gather fused with the first layer's attention norm
   CERB_ORDER(oc, LO_NORM_ATTN);
   { ProfScope ps(c, K_GLUE, st);
@@ -291,13 +295,24 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
   a.n_pool_pages = g.n_pool_pages; a.scratch = c->d_attn_scratch; a.scratch_bytes = c->attn_scratch_bytes;
   int ns = 1;
   for (int l = 0; l < g.n_layers; ++l) {
-    CERB_ORDER(oc, LO_GEMM_QKV);
-    { ProfScope ps(c, K_GEMM, st);
-      CERB_TRY(gemm(c, c->d_xn, &c->tm_xn, c->wqkv[l], c->bf16 ? &c->tm_wqkv[l] : nullptr, M, 3 * HD, d, &ns, st)); }
-    CERB_ORDER(oc, LO_ROPE);
-    { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_rope_append(c, l, tree->dev, c->d_part, ns, (size_t)M * 3 * HD, B, n, M, st, row_off)); }
     a.k_pool = c->k_pool + (size_t)l * c->pool_layer_bytes;
     a.v_pool = c->v_pool + (size_t)l * c->pool_layer_bytes;
+    CERB_ORDER(oc, LO_GEMM_QKV);
+    if (fuse_rope) {
+      // q, k and v leave the GEMM rotated and in place: no separate kernel, no second pass over the partial sums
+      ProfScope ps(c, K_GEMM, st);
+      const int nsl = gemm_plan_split(c->sm_count, M, 3 * HD, d);
+      if ((size_t)nsl * M * 3 * HD > c->part_floats) return CERB_E_NOMEM;
+      const RopeEpilogue re{c->d_len, c->d_nactive, tree->dev.depth, c->page_table, row_off, c->d_rope, c->d_q,
+                            (void*)a.k_pool, (void*)a.v_pool, g.max_pages, c->max_pos, n, g.n_heads, B};
+      const GemmEpilogue epi{2, nullptr, c->d_gemm_tickets, &re};
+      CERB_TRY(launch_gemm_bf16(c, &c->tm_wqkv[l], &c->tm_xn, c->d_part, M, 3 * HD, d, nsl, c->d_status, st, &epi, gemm_clock_slot(c)));
+    } else {
+      { ProfScope ps(c, K_GEMM, st);
+        CERB_TRY(gemm(c, c->d_xn, &c->tm_xn, c->wqkv[l], c->bf16 ? &c->tm_wqkv[l] : nullptr, M, 3 * HD, d, &ns, st)); }
+      CERB_ORDER(oc, LO_ROPE);
+      { ProfScope ps(c, K_GLUE, st); CERB_TRY(launch_rope_append(c, l, tree->dev, c->d_part, ns, (size_t)M * 3 * HD, B, n, M, st, row_off)); }
+    }
     CERB_ORDER(oc, LO_ATTN);
     { ProfScope ps(c, K_ATTN, st);
       CERB_TRY(launch_tree_attention(c, &a, c->bf16 ? &c->tm_kpool[l] : nullptr, c->bf16 ? &c->tm_vpool[l] : nullptr,
@@ -310,7 +325,7 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
     { ProfScope ps(c, K_GLUE, st);
       CERB_TRY(launch_fused_norm(c, c->d_part, ns, (size_t)M * d, nullptr, 0, 0, n, c->mlp_norm[l], c->d_xn, M, st)); }
     CERB_ORDER(oc, LO_GEMM_GU);
-    if (c->bf16 && gemm_swiglu_fusable(M, F)) {
+    if (fuse_swiglu) {
       // SwiGLU runs in the GEMM's epilogue: no separate kernel, no second pass over the partial sums
       ProfScope ps(c, K_GEMM, st);
       const int nsl = gemm_plan_split(c->sm_count, M, 2 * F, d);

@@ -37,6 +37,15 @@ typedef __nv_bfloat16 bf16;
 // anything the predecessor writes (or anything the predecessor may still be reading and this
 // kernel overwrites).  griddep_launch() lets the next kernel in the stream be scheduled early.
 #ifdef __CUDACC__
+// Which sequence and which node a row of the step's activation buffers belongs to: with ragged rows (sequences that
+// verify a one-node tree next to sequences that verify the whole tree) sequence b starts at row_off[b], otherwise at
+// b * n.
+__device__ __forceinline__ void locate_row(int row, const int32_t* __restrict__ row_off, int B, int n, int& b, int& v) {
+  if (!row_off) { b = row / n; v = row - b * n; return; }
+  b = 0;
+  while (b + 1 < B && row_off[b + 1] <= row) ++b;
+  v = row - row_off[b];
+}
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 #endif
@@ -189,7 +198,8 @@ constexpr int kTopkChunks = 16;     // the vocabulary is cut into this many chun
 // launch_order.cu: the forward's launch sequence and what each kernel reads ahead of its dependency wait
 enum { LO_SET_ACTIVE = 0, LO_NORM_ATTN, LO_GEMM_QKV, LO_ROPE, LO_ATTN, LO_GEMM_WO, LO_NORM_MLP, LO_GEMM_GU, LO_SWIGLU,
        LO_GEMM_DOWN, LO_NORM_FINAL, LO_GEMM_LM, LO_ARGMAX };
-int launch_order_layer(int variant, const int** ids_out);     // variant 0: separate SwiGLU kernel, 1: fused into the GEMM
+int launch_order_layer(int variant, const int** ids_out);     // variant 0: separate SwiGLU and RoPE kernels, 1: SwiGLU fused
+                                                               // into the gate-up GEMM, 2: RoPE + append fused into the QKV GEMM too
 int launch_order_violations(int variant);
 
 // ---- launch wrappers implemented across the .cu files (all asynchronous on `st`) ----
@@ -213,12 +223,24 @@ int gemm_plan_split(int sm_count, int M, int N, int K);
 // Optional fused epilogue of the bf16 GEMM.  kind 1 (SwiGLU): W is [gate rows F][up rows F]; the GEMM
 // pairs gate tile t with up tile t in one unit and the CTA that completes a tile last writes
 // act[row][f] = SiLU(gate) * up (bf16) instead of leaving the partial slots to a separate kernel.
+// kind 2 (RoPE + cache append): W is the QKV matrix [q rows | k rows | v rows] of a model with head_dim 128; the CTA
+// that completes a 256-row tile (two heads' worth of q, k or v) last sums the tile's slots in index order, rotates q
+// and k at position len + depth and writes q dense and k, v into the paged pools -- what rope_append_kernel does,
+// with the same arithmetic in the same order.  Both pay for steps of up to 16 rows only.
+struct RopeEpilogue {
+  const int32_t *len, *n_active, *depth, *page_table, *row_off;    // as for rope_append_kernel (row_off may be null)
+  const float2* rope;       // rotation table [max_pos][64]
+  void *q, *kpool, *vpool;  // bf16: q [rows][H * 128]; this layer's pools
+  int max_pages, max_pos, n, H, B;
+};
 struct GemmEpilogue {
-  int kind;                 // 0 none, 1 SwiGLU
-  void* act;                // [M][F] bf16
+  int kind;                 // 0 none, 1 SwiGLU, 2 RoPE + cache append
+  void* act;                // kind 1: [M][F] bf16
   unsigned int* tickets;    // kGemmTickets counters, zero on entry and on exit
+  const RopeEpilogue* rope; // kind 2
 };
 bool gemm_swiglu_fusable(int M, int F);
+bool gemm_rope_fusable(int M, int head_dim);
 int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, float* out, int M, int N, int K,
                      int nsplit, int32_t* status, cudaStream_t st, const GemmEpilogue* epi = nullptr,
                      unsigned long long* clock_slot = nullptr);

@@ -80,6 +80,7 @@ struct GemmParams {
   int F;              // SwiGLU: width of the gate (and of the up) block
   bf16* act;          // SwiGLU: output [M][F]
   unsigned int* tickets;
+  RopeEpilogue re;    // RoPE + cache append (epi == 2)
   unsigned long long* clk;   // measurement only: clk[0] <- min over CTAs of the time the dependency wait returned,
                              // clk[kGemmClockSlots] <- max over CTAs of the time the CTA finished (globaltimer, ns); or null
 };
@@ -334,6 +335,79 @@ __global__ void __launch_bounds__(224, 1) gemm_bf16_kernel(const __grid_constant
               uv += __ldcg(src + z * sstride + (size_t)m * ldo + p.F);
             }
             a[(size_t)m * p.F] = __float2bfloat16_rn(gv / (1.0f + expf(-gv)) * uv);
+          }
+          if (warp == 2 && lane == 0) p.tickets[sg.job] = 0u;      // ready for the next launch
+        }
+      }
+      if (p.epi == 2) {
+        // The CTA that finishes this tile last (by ticket) adds the tile's slots in index order, rotates q and k and
+        // stores q, k and v where the attention kernel expects them.  A thread owns one output column (= weight row)
+        // of each half of the unit; the other element of its rotation pair is 64 columns away in the same head.
+        __threadfence();
+        asm volatile("bar.sync 2, 128;" ::: "memory");
+        if (warp == 2 && lane == 0) ticket_s = atomicAdd(&p.tickets[sg.job], 1u);
+        asm volatile("bar.sync 2, 128;" ::: "memory");
+        if (ticket_s == (unsigned)cnt - 1u) {
+          __threadfence();
+          const RopeEpilogue& e = p.re;
+          const int HD = e.H * 128;
+          const size_t sstride = (size_t)p.M * ldo;
+          // this thread's two output columns (one per half of the unit) and their rotation partners
+          int col[2], which[2], hd[2];
+          bool col_ok[2];
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            col[hf] = tile * p.tile_rows + hf * p.half_off + quarter * 32 + lane;
+            col_ok[hf] = col[hf] < 3 * HD;
+            which[hf] = col_ok[hf] ? col[hf] / HD : 2;
+            hd[hf] = col[hf] - which[hf] * HD;
+          }
+          for (int m = 0; m < m_cnt; ++m) {
+            int b, v;
+            locate_row(m, e.row_off, e.B, e.n, b, v);
+            const int na = e.n_active[b], L = e.len[b], dep = e.depth[v];
+            // every slot value this thread needs, requested before any of them is used (one round trip to L2)
+            constexpr int ZMAX = 6;
+            float own[2][ZMAX], oth[2][ZMAX];
+            const float* src = p.out + (size_t)m * ldo;
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+              const int i = hd[hf] & 127;
+              const int partner = i < 64 ? col[hf] + 64 : col[hf] - 64;
+#pragma unroll
+              for (int z = 0; z < ZMAX; ++z) {
+                const bool take = col_ok[hf] && z < cnt;
+                own[hf][z] = take ? __ldcg(src + z * sstride + col[hf]) : 0.f;
+                oth[hf][z] = take && which[hf] < 2 ? __ldcg(src + z * sstride + partner) : 0.f;
+              }
+            }
+            const int pos = L + dep, slot = L + v;
+            const bool ok = v < na && pos < e.max_pos && slot < e.max_pos;
+            const int page = ok ? e.page_table[(size_t)b * e.max_pages + slot / CERB_PAGE] : 0;
+            float2 cs[2];
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) cs[hf] = ok && which[hf] < 2 ? e.rope[(size_t)pos * 64 + (hd[hf] & 63)] : make_float2(1.f, 0.f);
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+              if (!col_ok[hf] || !ok) continue;
+              const int i = hd[hf] & 127, h = hd[hf] >> 7;
+              float a = 0.f, o2 = 0.f;
+#pragma unroll
+              for (int z = 0; z < ZMAX; ++z) { a += own[hf][z]; o2 += oth[hf][z]; }        // slots in index order
+              for (int z = ZMAX; z < cnt; ++z) {                                          // (more slots than usual)
+                const int partner = i < 64 ? col[hf] + 64 : col[hf] - 64;
+                a += __ldcg(src + z * sstride + col[hf]);
+                if (which[hf] < 2) o2 += __ldcg(src + z * sstride + partner);
+              }
+              float val = a;
+              if (which[hf] < 2) val = i < 64 ? a * cs[hf].x - o2 * cs[hf].y : a * cs[hf].x + o2 * cs[hf].y;
+              if (which[hf] == 0) {
+                reinterpret_cast<bf16*>(e.q)[(size_t)m * HD + hd[hf]] = __float2bfloat16_rn(val);
+              } else {
+                bf16* pool = reinterpret_cast<bf16*>(which[hf] == 1 ? e.kpool : e.vpool);
+                pool[(((size_t)page * e.H + h) * CERB_PAGE + (size_t)(slot % CERB_PAGE)) * 128 + i] = __float2bfloat16_rn(val);
+              }
+            }
           }
           if (warp == 2 && lane == 0) p.tickets[sg.job] = 0u;      // ready for the next launch
         }
@@ -702,6 +776,11 @@ int make_pool_map(CUtensorMap* out, const void* pool, int n_pool_pages, int H, i
 bool gemm_swiglu_fusable(int M, int F) {
   return M >= 1 && M <= 16 && F % BM == 0;
 }
+// The same reasoning for the RoPE + cache-append epilogue of the QKV GEMM (head_dim 128: a 128-row weight tile is one
+// head, so both elements of every rotation pair lie in the tile that the finishing CTA owns).
+bool gemm_rope_fusable(int M, int head_dim) {
+  return M >= 1 && M <= 16 && head_dim == 128;
+}
 int gemm_plan_split(int sm_count, int M, int N, int K) { return make_plan(sm_count, M, N, K).nslots; }
 
 int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, float* out, int M, int N, int K,
@@ -742,6 +821,7 @@ int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, fl
     return CERB_OK;
   }
   GemmParams p;
+  memset(&p, 0, sizeof(p));
   int bucket = row_bucket(M);                   // (M <= 128 here)
   p.out = out;
   p.status = status;
@@ -764,6 +844,10 @@ int launch_gemm_bf16(cerb_ctx* c, const CUtensorMap* tmW, const ActMaps* tmX, fl
     p.epi = 1; p.F = N / 2; p.act = (bf16*)epi->act; p.tickets = epi->tickets;
     p.tile_rows = BM;            // a unit = gate tile t (rows t*128..) and up tile t (rows F + t*128..)
     p.half_off = p.F;
+  }
+  if (epi && epi->kind == 2) {
+    if (!epi->rope || !gemm_rope_fusable(M, 128) || N != 3 * epi->rope->H * 128 || g.tiles > kGemmTickets || !epi->tickets) return CERB_E_SHAPE;
+    p.epi = 2; p.tickets = epi->tickets; p.re = *epi->rope;
   }
   uint32_t stage_bytes = 2 * A_STAGE_BYTES + (uint32_t)p.n_mma * BK * 2;
   p.stages = (int)((216u * 1024u) / stage_bytes);

@@ -24,15 +24,6 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
   return t;
 }
 
-// Which sequence and which tree node a row belongs to.  Rows are ordered [sequence][node]; with ragged rows
-// (sequences that verify a one-node tree next to sequences that verify the whole tree) sequence b starts at
-// row_off[b], otherwise at b * n.
-__device__ __forceinline__ void locate_row(int row, const int32_t* __restrict__ row_off, int B, int n, int& b, int& v) {
-  if (!row_off) { b = row / n; v = row - b * n; return; }
-  b = 0;
-  while (b + 1 < B && row_off[b + 1] <= row) ++b;
-  v = row - row_off[b];
-}
 
 // cos/sin of pos * base^(-2i/Dh), evaluated once in double precision.
 __global__ void rope_table_kernel(float2* tab, int max_pos, int half, double base) {

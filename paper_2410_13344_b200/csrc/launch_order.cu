@@ -57,6 +57,14 @@ const Entry kLayer16[] = {
     {LO_GEMM_GU, "gemm gate-up + swiglu epilogue", B_PART | B_ACT, B_CONST},
     kLayer64[8],
 };
+// ... and (head_dim 128) RoPE + cache append in the QKV GEMM's epilogue.
+const Entry kLayer16r[] = {
+    kLayer64[0],
+    {LO_GEMM_QKV, "gemm qkv + rope / append epilogue", B_PART | B_Q | B_KV, B_CONST},
+    kLayer64[3], kLayer64[4], kLayer64[5],
+    {LO_GEMM_GU, "gemm gate-up + swiglu epilogue", B_PART | B_ACT, B_CONST},
+    kLayer64[8],
+};
 const Entry kTail[] = {
     {LO_NORM_FINAL, "fused_norm (residual add, final norm)", B_X | B_HIDDEN, B_X | B_CONST},
     {LO_GEMM_LM, "gemm lm_head", B_PART, B_CONST},
@@ -65,8 +73,10 @@ const Entry kTail[] = {
 
 int build(int variant, const Entry** out, int cap) {
   // set-up, three layers (enough to close the cycle between layers), tail
-  const Entry* layer = variant == 1 ? kLayer16 : kLayer64;
-  const int nl = variant == 1 ? (int)(sizeof(kLayer16) / sizeof(Entry)) : (int)(sizeof(kLayer64) / sizeof(Entry));
+  const Entry* layer = variant == 2 ? kLayer16r : variant == 1 ? kLayer16 : kLayer64;
+  const int nl = variant == 2   ? (int)(sizeof(kLayer16r) / sizeof(Entry))
+                 : variant == 1 ? (int)(sizeof(kLayer16) / sizeof(Entry))
+                                : (int)(sizeof(kLayer64) / sizeof(Entry));
   int n = 0;
   out[n++] = &kSetActive;
   for (int l = 0; l < 3; ++l)
@@ -78,14 +88,15 @@ int build(int variant, const Entry** out, int cap) {
 }  // namespace
 
 int launch_order_layer(int variant, const int** ids_out) {
-  static int ids64[16], ids16[16];
-  static int n64 = 0, n16 = 0;
+  static int ids64[16], ids16[16], ids16r[16];
+  static int n64 = 0, n16 = 0, n16r = 0;
   if (!n64) {
     for (const Entry& e : kLayer64) ids64[n64++] = e.id;
     for (const Entry& e : kLayer16) ids16[n16++] = e.id;
+    for (const Entry& e : kLayer16r) ids16r[n16r++] = e.id;
   }
-  *ids_out = variant == 1 ? ids16 : ids64;
-  return variant == 1 ? n16 : n64;
+  *ids_out = variant == 2 ? ids16r : variant == 1 ? ids16 : ids64;
+  return variant == 2 ? n16r : variant == 1 ? n16 : n64;
 }
 
 // Number of (kernel, buffer) pairs that break the rule; the tail after the last layer counts as the "next layer"
@@ -109,7 +120,7 @@ int launch_order_violations(int variant) {
 
 extern "C" int cerb_launch_order_table(int32_t variant, char* buf, size_t cap) {
   using namespace cerb;
-  if (!buf || cap < 64 || variant < 0 || variant > 1) return CERB_E_ARG;
+  if (!buf || cap < 64 || variant < 0 || variant > 2) return CERB_E_ARG;
   const Entry* seq[64];
   const int n = build(variant, seq, 64);
   size_t off = 0;

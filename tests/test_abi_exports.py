@@ -102,12 +102,12 @@ def test_no_kernel_reads_before_its_wait_what_the_kernel_in_front_writes():
     per kernel, the buffers written and the buffers read ahead of the wait; the rule is recomputed here."""
     from paper_2410_13344_b200 import binding
     CONST = 1 << 9
-    for variant in (0, 1):
+    for variant in (0, 1, 2):
         rc, rows = _launch_table(variant)
         assert rc == binding.OK
         names = [r[1] for r in rows]
         assert sum("gemm" in n for n in names) == 3 * 4 + 1 and sum(n == "tree attention" for n in names) == 3
-        assert ("swiglu" in names) == (variant == 0)
+        assert ("swiglu" in names) == (variant == 0) and ("rope_append" in names) == (variant < 2)
         for i, (_, name, _, reads) in enumerate(rows):
             for bit in range(9):
                 if not reads >> bit & 1:

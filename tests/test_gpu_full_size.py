@@ -47,13 +47,14 @@ def _engine(cb, ms, n_cheads, topk, max_tokens, max_batch=1):
     return model, layout, heads, eng
 
 
-def _two_layer_width_against_oracle(cb, ms, n_cheads, prompt_len, seq, what):
-    """Prefill, gate, draft, one 64-node verification forward, acceptance: values and decisions against the oracle."""
+def _two_layer_width_against_oracle(cb, ms, n_cheads, prompt_len, seq, what, n_nodes=64):
+    """Prefill, gate, draft, one verification forward over an n_nodes tree, acceptance: values and decisions against
+    the oracle."""
     topk = [10] * n_cheads
     model, layout, heads, eng = _engine(cb, ms, n_cheads, topk, 512)
     cmodel, cheads, sh, csrc = cpu(model), cpu(heads), oracle_shape(ms), concat_src(layout)
     prompt = [int(t) for t in synth.make_prompt(ms.vocab, prompt_len, seq=seq)]
-    tree = synth.best_first_tree(64, topk)
+    tree = synth.best_first_tree(n_nodes, topk)
     th = eng.tree(tree)
     eng.prefill(torch.tensor([prompt], dtype=torch.int32, device="cuda"), [len(prompt)])
     st = orc.prefill(cmodel, sh, prompt, 512)
@@ -80,7 +81,7 @@ def _two_layer_width_against_oracle(cb, ms, n_cheads, prompt_len, seq, what):
         assert [int(t) for t in topk_ids[0, h, :10]] == list(orc.topk_ids(hlog[0, h].cpu().double(), 10))
     want_tok = [int(roots[0])] + [int(topk_ids[0, tree.head[v], tree.rank[v]]) for v in range(1, tree.n)]
     assert [int(t) for t in tree_tok[0]] == want_tok
-    # verify: hidden states and logits of all 64 nodes, every argmax
+    # verify: hidden states and logits of all nodes, every argmax
     node_argmax, logits, hidden = eng.verify(th, tree_tok, want_logits=True, want_hidden=True)
     o_hidden, o_logits = orc.verify_tree(cmodel, sh, st, want_tok, tree.parent)
     assert_close_large(hidden[0], o_hidden, TOL, what + " hidden", outliers=OUTLIERS_HIDDEN)
@@ -98,6 +99,12 @@ def _two_layer_width_against_oracle(cb, ms, n_cheads, prompt_len, seq, what):
 
 def test_7b_width_two_layers_against_oracle(cb):
     _two_layer_width_against_oracle(cb, synth.shape_7b(n_layers=2), 4, 200, 7, "7B width, 2 layers")
+
+
+def test_7b_width_two_layers_twelve_node_tree_against_oracle(cb):
+    """Steps of up to 16 rows at head_dim 128 take other kernels for the same arithmetic: RoPE and the cache append run
+    in the QKV GEMM's epilogue, SwiGLU in the gate-up GEMM's, attention on the warp-MMA kernel."""
+    _two_layer_width_against_oracle(cb, synth.shape_7b(n_layers=2), 4, 150, 9, "7B width, 2 layers, 12 nodes", n_nodes=12)
 
 
 def test_13b_width_two_layers_against_oracle(cb):
