@@ -58,6 +58,7 @@ def _run_gpu(rig, th, T, prompt, n_new, plant_fn=None):
         toks = [int(t) for t in eng.h_tokens[0, :na]]
         recs.append(dict(S=float(eng.h_S[0]), mode=int(eng.h_mode[0]), n_accept=na, tokens=toks))
         out.extend(toks)
+    assert eng.wait_diagnosis() == [0, 0, 0, 0]        # no bounded wait ran out: code, wait, block and launch all unset
     assert eng.device_status() == 0
     return out[:n_new], recs
 
