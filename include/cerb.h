@@ -85,7 +85,7 @@ typedef struct cerb_config {
   int32_t max_pages;             /* page-table columns per sequence: capacity = 16 * max_pages tokens */
   int32_t n_pool_pages;          /* physical pages per layer in each pool */
   int32_t max_batch;             /* <= CERB_MAX_BATCH */
-  int32_t max_nodes;             /* <= CERB_MAX_NODES; prefill runs in chunks of min(max_nodes, 128) tokens */
+  int32_t max_nodes;             /* <= CERB_MAX_NODES (prefill runs in chunks of 128 tokens whatever this is) */
   int32_t n_cheads;              /* Cerberus heads CH_0 .. CH_{n_cheads-1} */
   int32_t n_levels;              /* Resblocks per head */
   /* Section 4.1 wiring: concat_src[h][j] = -1 for the plain Resblock

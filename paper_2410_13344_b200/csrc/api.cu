@@ -162,12 +162,14 @@ void init_sizes(cerb_ctx* c, const cerb_config* g, int sm_count) {
   c->cfg = *g;
   c->bf16 = g->dtype == CERB_BF16;
   c->esize = c->bf16 ? 2 : 4;
-  c->Mmax = g->max_batch * g->max_nodes;
+  // rows per sequence of one forward: the widest tree, or a prefill chunk (128 prompt tokens whatever max_nodes is)
+  const int rows_seq = g->max_nodes > kPrefillChunkMax ? g->max_nodes : kPrefillChunkMax;
+  c->Mmax = g->max_batch * rows_seq;
   c->max_pos = g->max_pages * CERB_PAGE;
   c->sm_count = sm_count;
   head_widths(g, c->head_w, &c->head_wmax);
   c->part_floats = part_floats_needed(g, c->Mmax, sm_count);
-  c->attn_scratch_bytes = attn_scratch_bytes(g->max_batch, g->max_nodes, g->n_heads, g->head_dim);
+  c->attn_scratch_bytes = attn_scratch_bytes(g->max_batch, rows_seq, g->n_heads, g->head_dim);
 }
 
 int tree_build(cerb_ctx* c, const int32_t* parent, const int32_t* head_of, const int32_t* rank_of, int n, int slot,
@@ -255,8 +257,9 @@ struct OrderCheck {
 // rows / row_off: with ragged rows (cerb_step on a batch whose sequences chose different modes) sequence b owns the
 // rows row_off[b] .. row_off[b] + n_active[b] - 1 of every activation buffer and `rows` is their total; otherwise
 // row_off is null and sequence b owns rows b * n .. b * n + n - 1.
+// need: per sequence, how many of the n rows are live (host; a prefill chunk near the end of a prompt), or null = n.
 int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok_stride, int tok_off, int n,
-                 cudaStream_t st, int rows = 0, const int32_t* row_off = nullptr) {
+                 cudaStream_t st, int rows = 0, const int32_t* row_off = nullptr, const int* need = nullptr) {
   const cerb_config& g = c->cfg;
   const int B = c->B, M = row_off ? rows : B * n, d = g.d_model, HD = g.n_heads * g.head_dim, F = g.mlp_dim;
   c->last_rows = M;
@@ -265,7 +268,8 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
   bool refreshed = false;
   int max_len = 0;
   for (int b = 0; b < B; ++b) {
-    if (c->h_len[b] + n > c->max_pos && !refreshed) {
+    const int nb = need ? need[b] : n;
+    if (c->h_len[b] + nb > c->max_pos && !refreshed) {
       int32_t tmp[CERB_MAX_BATCH];
       CERB_CUDA_OK(cudaStreamSynchronize(st));
       CERB_CUDA_OK(cudaMemcpy(tmp, c->d_len, B * sizeof(int32_t), cudaMemcpyDeviceToHost));
@@ -275,8 +279,8 @@ int forward_rows(cerb_ctx* c, const cerb_tree* tree, const int32_t* tok, int tok
       b = -1;
       continue;
     }
-    if (c->h_len[b] + n > c->max_pos) return CERB_E_STATE;
-    if (c->h_len[b] + n > max_len) max_len = c->h_len[b] + n;
+    if (c->h_len[b] + nb > c->max_pos) return CERB_E_STATE;
+    if (c->h_len[b] + nb > max_len) max_len = c->h_len[b] + nb;
   }
   // Steps of up to 16 rows: SwiGLU runs in the gate-up GEMM's epilogue and (head_dim 128) RoPE + cache append in the
   // QKV GEMM's.
@@ -487,7 +491,7 @@ int cerb_load(const cerb_config* cfg, const cerb_weights* w, void* workspace_dev
       if ((rc = make_act_maps(&c->tm_hlast, c->d_hlast, CERB_MAX_BATCH, g.d_model)) != CERB_OK) break;
     }
     if ((rc = launch_rope_table(c, 0)) != CERB_OK) break;
-    const int chunk = g.max_nodes < kPrefillChunkMax ? g.max_nodes : kPrefillChunkMax;
+    const int chunk = kPrefillChunkMax;
     std::vector<int32_t> par(chunk);
     for (int v = 0; v < chunk; ++v) par[v] = v - 1;
     // the prefill chain is deeper than an acceptable path may be: no depth limit for it
@@ -557,11 +561,16 @@ int cerb_prefill(cerb_ctx* c, const int32_t* tokens_dev, const int32_t* lens_hos
   CERB_CUDA_OK(cudaStreamSynchronize(st));
   for (int b = 0; b < B; ++b) c->h_stage[b] = lens_host[b];
   CERB_CUDA_OK(cudaMemcpyAsync(c->d_lens_in, c->h_stage, B * sizeof(int32_t), cudaMemcpyHostToDevice, st));
-  const int C = c->chain->n;          // min(max_nodes, 128) tokens per chunk
+  const int C = c->chain->n;          // 128 tokens per chunk
   for (int off = 0; off < longest; off += C) {
-    for (int b = 0; b < B; ++b) c->h_len[b] = lens_host[b] < off ? lens_host[b] : off;
+    int need[CERB_MAX_BATCH];
+    for (int b = 0; b < B; ++b) {
+      c->h_len[b] = lens_host[b] < off ? lens_host[b] : off;
+      const int left = lens_host[b] - off;
+      need[b] = left < 0 ? 0 : left < C ? left : C;
+    }
     CERB_TRY(launch_set_nactive(c, 1, off, C, st));
-    CERB_TRY(forward_rows(c, c->chain, tokens_dev, max_len, off, C, st));
+    CERB_TRY(forward_rows(c, c->chain, tokens_dev, max_len, off, C, st, 0, nullptr, need));
     CERB_TRY(launch_prefill_commit(c, C, st));
   }
   for (int b = 0; b < B; ++b) c->h_len[b] = lens_host[b];
